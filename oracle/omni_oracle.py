@@ -1,0 +1,327 @@
+"""CPU oracle for the per-chunk hot path: score -> select -> compact -> attend.
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain reference that the
+CUDA kernels are checked against.  Only the tests, the smoke check and the
+benchmark's CPU-baseline leg may import it; the product path never does.  It
+shares no code with the CUDA path and imports nothing from the package.
+
+Arithmetic: inputs are taken exactly as stored (bf16 or fp32 values widened to
+float64); every product, sum, exponential and division is float64 (numpy).
+Integer steps are plain integer arithmetic.
+
+What follows the paper and what does not
+----------------------------------------
+* compact_pack      -- eager compaction exactly as the paper defines it
+                       (Section 6, "Compaction-movement trade-off": all
+                       retained entries packed into a contiguous prefix), the
+                       allocation classes and page promotion rule of
+                       Section 6.1, the page-rounded span of Section 6.2.
+                       Pinned by the definition, by the span arithmetic the
+                       paper prints for Fig. 12 and Fig. 8, and by invariants.
+* chunk_attention   -- dense causal attention of the new chunk over the
+                       retained history (Section 2.1 prefill; Section 3 "Dense
+                       attention").  Pinned by brute force, by a library
+                       attention routine and by closed forms.
+* select_units      -- the paper's structural rules that are fixed (protected
+                       prefix, most recent events kept whole, whole-span
+                       boundaries, low watermark as a trimming target,
+                       re-indexing of survivors: Sections 5.1-5.2) plus a
+                       score-ordered greedy fill that the paper does NOT
+                       define.  PARITY UNPINNED for the greedy order; pinned
+                       only by invariants, special cases and brute force.
+* score_units       -- the paper's OmniPick collects no attention scores at
+                       run time; the statistic scored here is the one its
+                       design study measures offline (attention weight from
+                       later queries to each span, averaged; Section 5 "Key
+                       insight"), weighted per modality ("Modality-asymmetric
+                       attention").  PARITY UNPINNED by the paper; pinned only
+                       by closed forms, invariants and brute force.
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+# unit-table columns
+U_START, U_LEN, U_MOD, U_EVENT, U_GROUP, U_FLAGS = range(6)
+GRP_MUST_KEEP, GRP_SELECTED, GRP_RECENT = 0, 1, 2
+KEEP_DROPPED, KEEP_WHOLE = 0, 2          # code 1 (sink prefix only) is reserved
+PAGE_EMPTY = 255
+
+
+def _f64(a):
+    return np.asarray(a, dtype=np.float64)
+
+
+# ---------------------------------------------------------------------------
+# S -- unit scoring
+# ---------------------------------------------------------------------------
+def score_units(q, k_hist, units, w_modality, scale=None):
+    """Modality-weighted mean attention lift of the chunk's queries on each history unit.
+
+    q [T, Hq, D], k_hist [N, Hkv, D], units [U, 6] covering slots 0..N-1 in order.
+    For head h, query i, history key j:
+        s_hij = scale * <q[i,h,:], k[j, h // G, :]>,     G = Hq / Hkv
+        a_hij = softmax over j in [0, N) of s_hij        (history keys only)
+    token importance  I_j    = mean over (h, i) of a_hij            (sums to 1 over j)
+    unit mass         mass_u = sum of I_j over the unit's tokens
+    unit score        score_u = w[modality_u] * mass_u * N / len_u  (1.0*w means "uniform attention")
+    Returns (score[U], mass[U]) as float64.
+    """
+    q = _f64(q)
+    k = _f64(k_hist)
+    units = np.asarray(units)
+    T, Hq, D = q.shape
+    N, Hkv, _ = k.shape
+    G = Hq // Hkv
+    if scale is None or scale <= 0:
+        scale = 1.0 / math.sqrt(D)
+    importance = np.zeros(N, dtype=np.float64)
+    for h in range(Hq):
+        s = (q[:, h, :] @ k[:, h // G, :].T) * scale              # [T, N]
+        s -= s.max(axis=1, keepdims=True)
+        a = np.exp(s)
+        a /= a.sum(axis=1, keepdims=True)
+        importance += a.sum(axis=0)
+    importance /= float(Hq * T)
+    U = len(units)
+    mass = np.zeros(U, dtype=np.float64)
+    score = np.zeros(U, dtype=np.float64)
+    for u in range(U):
+        st, ln, mod = int(units[u, U_START]), int(units[u, U_LEN]), int(units[u, U_MOD])
+        mass[u] = importance[st:st + ln].sum()
+        score[u] = float(w_modality[mod]) * mass[u] * N / ln if ln > 0 else 0.0
+    return score, mass
+
+
+# ---------------------------------------------------------------------------
+# L -- budgeted unit selection
+# ---------------------------------------------------------------------------
+def select_units(units, scores, budget, n_recent_events=1, modality_cap=(-1, -1, -1)):
+    """Choose which whole units of the history survive.
+
+    1. Protected set: units in the must-keep group (protected system prefix,
+       Section 5.1) and every unit of the `n_recent_events` newest events
+       (recent units kept in full, never cut at a token position).
+    2. If the protected set alone reaches the budget, keep exactly it: the
+       budget is a trimming target, not a strict bound (Section 5.1).
+    3. Remaining units are candidates, visited by descending score (ties: the
+       more recent unit first; NaN scores last).  A candidate is taken iff it
+       fits the remaining budget and its modality's remaining cap; a misfit
+       does not end the walk.
+    4. Survivors are re-indexed: a kept token's new position is the number of
+       kept tokens before it (Section 5.2); unit records keep modality, event
+       and flags; group becomes must-keep / recent-context / selected-history.
+
+    `scores` is compared in float32 (the precision the CUDA path ranks in).
+    Returns dict(unit_keep[U] u8, keep_mask[N] u8, n_kept, units_out[U', 6], order[list]).
+    """
+    units = np.asarray(units, dtype=np.int64)
+    U = len(units)
+    scores = np.asarray(scores, dtype=np.float32)
+    events = units[:, U_EVENT]
+    if U > 1 and np.any(np.diff(events) < 0):
+        raise ValueError("event ids must be non-decreasing in unit order")
+    distinct = sorted(set(int(e) for e in events))
+    recent = set(distinct[len(distinct) - n_recent_events:]) if n_recent_events > 0 else set()
+
+    protected = [u for u in range(U)
+                 if units[u, U_GROUP] == GRP_MUST_KEEP or int(events[u]) in recent]
+    keep = np.zeros(U, dtype=np.uint8)
+    for u in protected:
+        keep[u] = KEEP_WHOLE
+    used = int(sum(units[u, U_LEN] for u in protected))
+    order = []
+    if used < budget:
+        cand = [u for u in range(U) if keep[u] == 0]
+
+        def key(u):
+            s = scores[u]
+            if np.isnan(s):
+                return (1, 0.0, -u)
+            return (0, -float(s), -u)
+        cand.sort(key=key)
+        order = cand
+        cap_rem = [int(c) if c >= 0 else None for c in modality_cap]
+        for u in cand:
+            ln, mod = int(units[u, U_LEN]), int(units[u, U_MOD])
+            if ln > budget - used:
+                continue
+            if cap_rem[mod] is not None and ln > cap_rem[mod]:
+                continue
+            keep[u] = KEEP_WHOLE
+            used += ln
+            if cap_rem[mod] is not None:
+                cap_rem[mod] -= ln
+
+    n_hist = int(units[:, U_LEN].sum())
+    keep_mask = np.zeros(n_hist, dtype=np.uint8)
+    units_out = []
+    pos = 0
+    for u in range(U):
+        if keep[u]:
+            st, ln = int(units[u, U_START]), int(units[u, U_LEN])
+            keep_mask[st:st + ln] = 1
+            if units[u, U_GROUP] == GRP_MUST_KEEP:
+                g = GRP_MUST_KEEP
+            elif int(events[u]) in recent:
+                g = GRP_RECENT
+            else:
+                g = GRP_SELECTED
+            units_out.append((pos, ln, int(units[u, U_MOD]), int(events[u]), g, int(units[u, U_FLAGS])))
+            pos += ln
+    units_out = np.asarray(units_out, dtype=np.int32).reshape(-1, 6)
+    return dict(unit_keep=keep, keep_mask=keep_mask, n_kept=pos, units_out=units_out, order=order)
+
+
+# ---------------------------------------------------------------------------
+# C -- eager compaction into the retention-partitioned page layout
+# ---------------------------------------------------------------------------
+def compact_pack(k_cache, v_cache, keep_mask, page_size, units_out=None):
+    """Pack every retained KV row into a contiguous prefix, order preserved.
+
+    k_cache, v_cache: [S, ...] arrays of any dtype (rows are copied bit for bit).
+    keep_mask [S_span] u8.  As-if semantics: all reads precede all writes.
+    Returns dict with
+      k, v         packed rows [n_kept, ...]
+      slot_map     [S_span] int32, destination slot or -1
+      n_kept, span_pages (= ceil(n_kept / P): the page-rounded span), rows_moved
+      part_begin   [4]: first slot of must-keep / selected-history / recent-context / end
+      page_class   [ceil(S_span / P)] u8: 0 page holds a must-keep row; else 1 if it holds P
+                   kept rows (fully packed page promoted to selected-history); else 2 if
+                   partially filled (stays recent-context); else 255 (empty, reusable).
+    `units_out` (the compacted unit table) supplies the groups for the partitions; because
+    units are in logical order and group rank grows with recency, the stable pack IS the
+    partitioned order -- this is asserted, not assumed.
+    """
+    keep_mask = np.asarray(keep_mask, dtype=np.uint8)
+    S = len(keep_mask)
+    P = int(page_size)
+    slot_map = np.full(S, -1, dtype=np.int32)
+    n = 0
+    src = []
+    for s in range(S):
+        if keep_mask[s]:
+            slot_map[s] = n
+            src.append(s)
+            n += 1
+    src = np.asarray(src, dtype=np.int64)
+    k_out = np.array(np.asarray(k_cache)[src], copy=True) if k_cache is not None else None
+    v_out = np.array(np.asarray(v_cache)[src], copy=True) if v_cache is not None else None
+    rows_moved = int(np.sum(src != np.arange(n)))
+    span_pages = (n + P - 1) // P
+
+    part_begin = np.array([0, 0, 0, n], dtype=np.int32)
+    if units_out is not None and len(units_out):
+        uo = np.asarray(units_out, dtype=np.int64)
+        groups = uo[:, U_GROUP]
+        if np.any(np.diff(groups) < 0):
+            raise ValueError("retention groups are not ordered must-keep <= selected-history <= recent-context")
+        if int(uo[:, U_LEN].sum()) != n:
+            raise ValueError("compacted unit table does not cover the kept rows")
+        n0 = int(uo[groups == GRP_MUST_KEEP, U_LEN].sum())
+        n1 = int(uo[groups == GRP_SELECTED, U_LEN].sum())
+        part_begin = np.array([0, n0, n0 + n1, n], dtype=np.int32)
+
+    n_pages = (S + P - 1) // P
+    page_class = np.full(n_pages, PAGE_EMPTY, dtype=np.uint8)
+    for p in range(n_pages):
+        lo, hi = p * P, min((p + 1) * P, n)
+        if hi <= lo:
+            continue
+        if lo < part_begin[1]:
+            page_class[p] = GRP_MUST_KEEP
+        elif hi - lo == P:
+            page_class[p] = GRP_SELECTED
+        else:
+            page_class[p] = GRP_RECENT
+    return dict(k=k_out, v=v_out, slot_map=slot_map, n_kept=n, span_pages=span_pages,
+                rows_moved=rows_moved, part_begin=part_begin, page_class=page_class)
+
+
+# ---------------------------------------------------------------------------
+# a5 -- append the chunk behind the compacted history
+# ---------------------------------------------------------------------------
+def append_chunk(units_kept, n_kept, chunk_units):
+    """New entries enter the recent-context class behind the kept history (Section 6.1)."""
+    cu = np.array(chunk_units, dtype=np.int32, copy=True).reshape(-1, 6)
+    cu[:, U_START] += int(n_kept)
+    cu[:, U_GROUP] = GRP_RECENT
+    uk = np.asarray(units_kept, dtype=np.int32).reshape(-1, 6)
+    return np.concatenate([uk, cu], axis=0)
+
+
+# ---------------------------------------------------------------------------
+# A -- GQA chunk-prefill attention
+# ---------------------------------------------------------------------------
+def chunk_attention(q, k_hist, v_hist, k_chunk, v_chunk, scale=None, rows=None):
+    """o[i,h] = sum_j softmax_j(scale * <q_ih, k_j>) v_j over the kept history rows followed by
+    chunk rows 0..i (causal inside the chunk, diagonal included); kv head of h is h // G.
+
+    rows: optional iterable of (i, h) pairs to evaluate only those outputs.
+    Returns (o [T, Hq, D] float64, lse [T, Hq] float64) or, with rows, (o [R, D], lse [R]).
+    """
+    q = _f64(q)
+    kh, vh, kc, vc = _f64(k_hist), _f64(v_hist), _f64(k_chunk), _f64(v_chunk)
+    T, Hq, D = q.shape
+    Hkv = kc.shape[1]
+    G = Hq // Hkv
+    Nh = kh.shape[0]
+    if scale is None or scale <= 0:
+        scale = 1.0 / math.sqrt(D)
+
+    if rows is not None:
+        rows = list(rows)
+        o = np.zeros((len(rows), D), dtype=np.float64)
+        lse = np.zeros(len(rows), dtype=np.float64)
+        for r, (i, h) in enumerate(rows):
+            g = h // G
+            keys = np.concatenate([kh[:, g, :], kc[:i + 1, g, :]], axis=0)
+            vals = np.concatenate([vh[:, g, :], vc[:i + 1, g, :]], axis=0)
+            s = (keys @ q[i, h, :]) * scale
+            m = s.max()
+            p = np.exp(s - m)
+            z = p.sum()
+            o[r] = (p @ vals) / z
+            lse[r] = m + math.log(z)
+        return o, lse
+
+    o = np.zeros((T, Hq, D), dtype=np.float64)
+    lse = np.zeros((T, Hq), dtype=np.float64)
+    causal = np.tril(np.ones((T, T), dtype=bool))
+    for h in range(Hq):
+        g = h // G
+        s_h = (q[:, h, :] @ kh[:, g, :].T) * scale if Nh else np.zeros((T, 0))
+        s_c = (q[:, h, :] @ kc[:, g, :].T) * scale
+        s_c = np.where(causal, s_c, -np.inf)
+        s = np.concatenate([s_h, s_c], axis=1)                    # [T, Nh + T]
+        m = s.max(axis=1, keepdims=True)
+        p = np.exp(s - m)
+        z = p.sum(axis=1, keepdims=True)
+        o[:, h, :] = (p[:, :Nh] @ vh[:, g, :] + p[:, Nh:] @ vc[:, g, :]) / z
+        lse[:, h] = (m + np.log(z))[:, 0]
+    return o, lse
+
+
+# ---------------------------------------------------------------------------
+# one pass of the whole path
+# ---------------------------------------------------------------------------
+def stream_step(q, k_cache, v_cache, units, k_chunk, v_chunk, chunk_units, w_modality, budget,
+                n_recent_events, modality_cap, page_size, scale=None, scores_override=None):
+    """score -> select -> compact -> append -> attend, for one chunk and one layer.
+    k_cache/v_cache hold exactly the history rows [N, Hkv, D]."""
+    units = np.asarray(units)
+    n_hist = int(units[:, U_LEN].sum())
+    if scores_override is None:
+        score, mass = score_units(q, k_cache[:n_hist], units, w_modality, scale)
+    else:
+        score, mass = np.asarray(scores_override), None
+    sel = select_units(units, score, budget, n_recent_events, modality_cap)
+    cp = compact_pack(k_cache[:n_hist], v_cache[:n_hist], sel["keep_mask"], page_size, sel["units_out"])
+    o, lse = chunk_attention(q, cp["k"], cp["v"], k_chunk, v_chunk, scale)
+    units_new = append_chunk(sel["units_out"], cp["n_kept"], chunk_units)
+    k_new = np.concatenate([cp["k"], np.asarray(k_chunk)], axis=0)
+    v_new = np.concatenate([cp["v"], np.asarray(v_chunk)], axis=0)
+    return dict(score=score, mass=mass, select=sel, compact=cp, o=o, lse=lse,
+                units=units_new, k_cache=k_new, v_cache=v_new)

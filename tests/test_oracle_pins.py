@@ -1,0 +1,435 @@
+"""Pins for the CPU oracle: what the paper prints, closed forms, invariants, library
+routines on special cases and brute force on tiny inputs.  No GPU needed."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import omni_oracle as oc
+from paper_2609_34653_b200 import workloads as wl
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "paper_span_arithmetic.txt")
+
+
+def _golden_rows():
+    rows = {}
+    with open(GOLDEN) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            name, useful, before, after, page, note = line.split()
+            rows[name] = (int(useful), int(before), int(after), int(page), note)
+    return rows
+
+
+# ---------------------------------------------------------------- compaction
+def test_compact_paper_span_qwen_fig12():
+    """2,778 useful cells scattered over a 3,840-slot span pack to 44 pages = 2,816 slots (Fig. 12)."""
+    useful, before, after, page, _ = _golden_rows()["qwen_32k"]
+    rng = np.random.default_rng(7)
+    mask = np.zeros(before, dtype=np.uint8)
+    idx = rng.choice(before - 1, size=useful - 1, replace=False)
+    mask[idx] = 1
+    mask[before - 1] = 1                       # the span really is `before` slots long
+    k = rng.integers(0, 2**16, size=(before, 2, 4), dtype=np.uint16)
+    res = oc.compact_pack(k, k[::-1].copy(), mask, page)
+    assert res["n_kept"] == useful
+    assert res["span_pages"] * page == after
+    assert abs(1 - after / before - 0.267) < 5e-4
+
+
+def test_compact_paper_span_minicpm_and_eager_ratio():
+    g = _golden_rows()
+    useful, before, after, page, _ = g["minicpm_32k"]
+    mask = np.zeros(before, dtype=np.uint8)
+    mask[np.linspace(0, before - 1, useful).astype(int)] = 1
+    n = int(mask.sum())
+    res = oc.compact_pack(None, None, mask, page)
+    # eager packing reaches the page-rounded optimum, which is below the paper's selective result
+    assert res["span_pages"] * page == -(-n // page) * page <= after
+    assert abs(1 - after / before - 0.10) < 1e-3
+    useful, before, after, page, _ = g["eager_60chunk"]
+    mask = np.zeros(before, dtype=np.uint8)
+    mask[np.arange(useful) * before // useful] = 1
+    res = oc.compact_pack(None, None, mask, page)
+    assert res["span_pages"] * page == after and before / after == 2.25
+
+
+def test_compact_definition_and_invariants():
+    rng = np.random.default_rng(3)
+    for S, P in [(1, 16), (17, 16), (200, 16), (1000, 64), (777, 256)]:
+        mask = (rng.random(S) < 0.37).astype(np.uint8)
+        k = rng.integers(0, 2**16, size=(S, 3, 8), dtype=np.uint16)
+        v = rng.integers(0, 2**16, size=(S, 3, 8), dtype=np.uint16)
+        res = oc.compact_pack(k, v, mask, P)
+        n = int(mask.sum())
+        assert res["n_kept"] == n and res["span_pages"] == -(-n // P)
+        # span never exceeds the kept count rounded up to a page, and wastes less than one page
+        assert 0 <= res["span_pages"] * P - n < P
+        # written out independently: the j-th kept slot lands at j, bytes intact, order preserved
+        kept_slots = [s for s in range(S) if mask[s]]
+        for j, s in enumerate(kept_slots):
+            assert res["slot_map"][s] == j
+            assert res["k"][j].tobytes() == k[s].tobytes() and res["v"][j].tobytes() == v[s].tobytes()
+        assert all(res["slot_map"][s] == -1 for s in range(S) if not mask[s])
+        assert res["rows_moved"] == sum(1 for j, s in enumerate(kept_slots) if j != s)
+        # idempotence: compacting the packed cache moves nothing
+        mask2 = np.zeros(S, dtype=np.uint8)
+        mask2[:n] = 1
+        res2 = oc.compact_pack(res["k"], res["v"], mask2[:n], P)
+        assert res2["rows_moved"] == 0 and res2["n_kept"] == n
+    # all keep = identity, none keep = empty
+    k = np.arange(40, dtype=np.float32).reshape(10, 4)
+    res = oc.compact_pack(k, k, np.ones(10, np.uint8), 4)
+    assert res["rows_moved"] == 0 and np.array_equal(res["k"], k) and res["span_pages"] == 3
+    res = oc.compact_pack(k, k, np.zeros(10, np.uint8), 4)
+    assert res["n_kept"] == 0 and res["span_pages"] == 0 and np.all(res["page_class"] == 255)
+
+
+def test_compact_partitions_and_page_classes():
+    # groups 0,1,1,2 with lens 20, 30, 14, 25 -> n = 89, P = 16
+    units_out = np.array([[0, 20, 2, 0, 0, 0], [20, 30, 0, 1, 1, 0], [50, 14, 1, 1, 1, 0],
+                          [64, 25, 0, 9, 2, 0]], dtype=np.int32)
+    mask = np.zeros(160, dtype=np.uint8)
+    mask[np.arange(89) + np.arange(89) // 3] = 1
+    res = oc.compact_pack(None, None, mask, 16, units_out)
+    assert res["part_begin"].tolist() == [0, 20, 64, 89]
+    # pages 0,1 hold must-keep rows; 2..4 are full -> promoted; page 5 partial -> recent; rest empty
+    assert res["page_class"].tolist() == [0, 0, 1, 1, 1, 2, 255, 255, 255, 255]
+    with pytest.raises(ValueError):
+        oc.compact_pack(None, None, mask, 16, units_out[[1, 0, 2, 3]])
+
+
+# ----------------------------------------------------------------- attention
+def _brute_attention(q, kh, vh, kc, vc, scale):
+    T, Hq, D = q.shape
+    G = Hq // kc.shape[1]
+    o = np.zeros((T, Hq, D))
+    lse = np.zeros((T, Hq))
+    for i in range(T):
+        for h in range(Hq):
+            g = h // G
+            keys = [kh[j, g] for j in range(kh.shape[0])] + [kc[j, g] for j in range(i + 1)]
+            vals = [vh[j, g] for j in range(vh.shape[0])] + [vc[j, g] for j in range(i + 1)]
+            s = [scale * sum(float(a) * float(b) for a, b in zip(q[i, h], kk)) for kk in keys]
+            m = max(s)
+            e = [math.exp(x - m) for x in s]
+            z = sum(e)
+            for d in range(D):
+                o[i, h, d] = sum(e[j] * float(vals[j][d]) for j in range(len(e))) / z
+            lse[i, h] = m + math.log(z)
+    return o, lse
+
+
+def test_attention_brute_force_tiny():
+    rng = np.random.default_rng(11)
+    T, Hq, Hkv, D, N = 5, 4, 2, 8, 7
+    q = rng.standard_normal((T, Hq, D)).astype(np.float32)
+    kh, vh = rng.standard_normal((2, N, Hkv, D)).astype(np.float32)
+    kc, vc = rng.standard_normal((2, T, Hkv, D)).astype(np.float32)
+    o, lse = oc.chunk_attention(q, kh, vh, kc, vc)
+    ob, lb = _brute_attention(q, kh, vh, kc, vc, 1 / math.sqrt(D))
+    assert np.allclose(o, ob, atol=1e-12) and np.allclose(lse, lb, atol=1e-12)
+    # a non-default scale and the sampled-rows form agree too
+    o2, l2 = oc.chunk_attention(q, kh, vh, kc, vc, scale=0.3, rows=[(4, 3), (0, 0), (2, 1)])
+    ob2, lb2 = _brute_attention(q, kh, vh, kc, vc, 0.3)
+    assert np.allclose(o2, [ob2[4, 3], ob2[0, 0], ob2[2, 1]], atol=1e-12)
+    assert np.allclose(l2, [lb2[4, 3], lb2[0, 0], lb2[2, 1]], atol=1e-12)
+
+
+def test_attention_equals_library_causal_attention():
+    """History + chunk attention is plain causal attention of the last T rows of the joined
+    sequence (dense attention keeps every preceding token): compare with torch SDPA."""
+    import torch
+    rng = np.random.default_rng(5)
+    T, Hq, Hkv, D, N = 33, 4, 2, 16, 70
+    q = rng.standard_normal((T, Hq, D)).astype(np.float32)
+    kh, vh = rng.standard_normal((2, N, Hkv, D)).astype(np.float32)
+    kc, vc = rng.standard_normal((2, T, Hkv, D)).astype(np.float32)
+    o, _ = oc.chunk_attention(q, kh, vh, kc, vc)
+    G = Hq // Hkv
+    K = torch.from_numpy(np.concatenate([kh, kc])).double().permute(1, 0, 2).repeat_interleave(G, 0)
+    V = torch.from_numpy(np.concatenate([vh, vc])).double().permute(1, 0, 2).repeat_interleave(G, 0)
+    Q = torch.from_numpy(q).double().permute(1, 0, 2)
+    mask = torch.ones(T, N + T, dtype=torch.bool).tril(diagonal=N)
+    ref = torch.nn.functional.scaled_dot_product_attention(Q[None], K[None], V[None], attn_mask=mask)[0]
+    assert np.allclose(o, ref.permute(1, 0, 2).numpy(), atol=1e-10)
+
+
+def test_attention_closed_forms():
+    rng = np.random.default_rng(9)
+    T, Hq, Hkv, D, N = 6, 2, 1, 8, 10
+    q = rng.standard_normal((T, Hq, D)).astype(np.float32)
+    vh = rng.standard_normal((N, Hkv, D)).astype(np.float32)
+    vc = rng.standard_normal((T, Hkv, D)).astype(np.float32)
+    kconst = rng.standard_normal(D).astype(np.float32)
+    kh = np.broadcast_to(kconst, (N, Hkv, D)).copy()
+    kc = np.broadcast_to(kconst, (T, Hkv, D)).copy()
+    o, lse = oc.chunk_attention(q, kh, vh, kc, vc)
+    # equal keys -> uniform weights -> running mean of the values; lse = s + log(count)
+    for i in range(T):
+        mean = (vh[:, 0].astype(np.float64).sum(0) + vc[:i + 1, 0].astype(np.float64).sum(0)) / (N + i + 1)
+        for h in range(Hq):
+            assert np.allclose(o[i, h], mean, atol=1e-12)
+            s = float(np.dot(q[i, h].astype(np.float64), kconst.astype(np.float64))) / math.sqrt(D)
+            assert abs(lse[i, h] - (s + math.log(N + i + 1))) < 1e-12
+    # permuting history rows does not change the output
+    kh = rng.standard_normal((N, Hkv, D)).astype(np.float32)
+    kc = rng.standard_normal((T, Hkv, D)).astype(np.float32)
+    o1, l1 = oc.chunk_attention(q, kh, vh, kc, vc)
+    perm = rng.permutation(N)
+    o2, l2 = oc.chunk_attention(q, kh[perm], vh[perm], kc, vc)
+    assert np.allclose(o1, o2, atol=1e-12) and np.allclose(l1, l2, atol=1e-12)
+    # splitting the history and merging the halves by their log-sum-exp reproduces the result
+    oa, la = oc.chunk_attention(q, kh[:4], vh[:4], kc, vc)
+    # second half: history only, no chunk -> emulate with a chunk whose keys never win
+    s_b = np.einsum("ihd,jd->ihj", q.astype(np.float64), kh[4:, 0].astype(np.float64)) / math.sqrt(D)
+    lb = np.log(np.exp(s_b).sum(-1))
+    ob = np.einsum("ihj,jd->ihd", np.exp(s_b - lb[..., None]), vh[4:, 0].astype(np.float64))
+    wa, wb = np.exp(la - np.logaddexp(la, lb)), np.exp(lb - np.logaddexp(la, lb))
+    assert np.allclose(o1, wa[..., None] * oa + wb[..., None] * ob, atol=1e-12)
+    # empty history is plain causal self-attention: row 0 returns v_chunk[0]
+    o0, _ = oc.chunk_attention(q, kh[:0], vh[:0], kc, vc)
+    assert np.allclose(o0[0, 0], vc[0, 0], atol=1e-12)
+
+
+# ------------------------------------------------------------------- scoring
+def _units(lens, mods=None, events=None, groups=None):
+    mods = mods or [0] * len(lens)
+    events = events or list(range(len(lens)))
+    u = wl.make_units(list(zip(lens, mods, events)), group_of_first=None)
+    if groups is not None:
+        u[:, 4] = groups
+    return u
+
+
+def test_score_closed_form_identical_keys():
+    rng = np.random.default_rng(2)
+    units = _units([5, 9, 2, 16], mods=[2, 0, 1, 0])
+    N = 32
+    q = rng.standard_normal((7, 4, 8)).astype(np.float32)
+    k = np.broadcast_to(rng.standard_normal(8).astype(np.float32), (N, 2, 8)).copy()
+    w = (1.0, 2.5, 0.75)
+    score, mass = oc.score_units(q, k, units, w)
+    assert np.allclose(mass, np.array([5, 9, 2, 16]) / N, atol=1e-14)
+    assert np.allclose(score, [w[2], w[0], w[1], w[0]], atol=1e-13)
+
+
+def test_score_invariants_and_permutation():
+    rng = np.random.default_rng(4)
+    lens = [5, 9, 2, 16, 7]
+    units = _units(lens, mods=[2, 0, 1, 0, 1])
+    N = sum(lens)
+    q = rng.standard_normal((6, 4, 8)).astype(np.float32)
+    k = rng.standard_normal((N, 2, 8)).astype(np.float32)
+    score, mass = oc.score_units(q, k, units, (1, 1, 1))
+    assert abs(mass.sum() - 1) < 1e-13
+    assert abs((score * np.array(lens)).sum() - N) < 1e-11
+    # re-ordering whole units permutes the scores
+    order = [3, 0, 4, 1, 2]
+    k2 = np.concatenate([k[units[u, 0]:units[u, 0] + units[u, 1]] for u in order])
+    units2 = _units([lens[u] for u in order], mods=[int(units[u, 2]) for u in order])
+    w = (1.0, 2.0, 3.0)
+    s1, m1 = oc.score_units(q, k, units, w)
+    s2, m2 = oc.score_units(q, k2, units2, w)
+    assert np.allclose(s2, s1[order], atol=1e-13) and np.allclose(m2, m1[order], atol=1e-14)
+    # one key strongly aligned with every query draws all the mass to its unit
+    qpos = np.abs(q)
+    kb = k.copy()
+    kb[20] = 50.0
+    _, mb = oc.score_units(qpos, kb, units, (1, 1, 1))
+    assert mb[3] > 1 - 1e-9
+
+
+def test_score_single_row_is_textbook_softmax():
+    from scipy.special import softmax
+    rng = np.random.default_rng(8)
+    lens = [3, 4, 6]
+    units = _units(lens)
+    q = rng.standard_normal((1, 1, 16)).astype(np.float32)
+    k = rng.standard_normal((13, 1, 16)).astype(np.float32)
+    _, mass = oc.score_units(q, k, units, (1, 1, 1))
+    a = softmax((k[:, 0].astype(np.float64) @ q[0, 0].astype(np.float64)) / 4.0)
+    assert np.allclose(mass, [a[0:3].sum(), a[3:7].sum(), a[7:13].sum()], atol=1e-14)
+
+
+def test_score_brute_force_tiny():
+    rng = np.random.default_rng(13)
+    lens = [4, 1, 7, 3]
+    mods = [2, 0, 1, 0]
+    units = _units(lens, mods=mods)
+    N, T, Hq, Hkv, D = sum(lens), 5, 4, 2, 6
+    q = rng.standard_normal((T, Hq, D)).astype(np.float32)
+    k = rng.standard_normal((N, Hkv, D)).astype(np.float32)
+    w = (1.0, 2.0, 0.5)
+    imp = [0.0] * N
+    for h in range(Hq):
+        for i in range(T):
+            s = [sum(float(q[i, h, d]) * float(k[j, h // 2, d]) for d in range(D)) / math.sqrt(D)
+                 for j in range(N)]
+            m = max(s)
+            e = [math.exp(x - m) for x in s]
+            z = sum(e)
+            for j in range(N):
+                imp[j] += e[j] / z / (Hq * T)
+    exp_score, pos = [], 0
+    for ln, mod in zip(lens, mods):
+        exp_score.append(w[mod] * sum(imp[pos:pos + ln]) * N / ln)
+        pos += ln
+    score, _ = oc.score_units(q, k, units, w)
+    assert np.allclose(score, exp_score, atol=1e-12)
+
+
+# ----------------------------------------------------------------- selection
+def _check_select_invariants(units, scores, budget, R, caps, res):
+    U = len(units)
+    keep = res["unit_keep"]
+    events = units[:, 3]
+    distinct = sorted(set(events.tolist()))
+    recent = set(distinct[-R:]) if R > 0 else set()
+    prot = [u for u in range(U) if units[u, 4] == 0 or events[u] in recent]
+    assert all(keep[u] == 2 for u in prot)                                     # I1
+    prot_len = int(units[prot, 1].sum())
+    n_kept = int(units[keep != 0, 1].sum())
+    assert res["n_kept"] == n_kept
+    if prot_len >= budget:
+        assert sorted(np.nonzero(keep)[0].tolist()) == sorted(prot)            # I2 (target, not bound)
+    else:
+        assert n_kept <= budget
+    mask = res["keep_mask"]
+    for u in range(U):                                                         # I3 no unit split
+        seg = mask[units[u, 0]:units[u, 0] + units[u, 1]]
+        assert np.all(seg == (1 if keep[u] else 0))
+    # re-indexing: new start = kept tokens before the unit; labels preserved
+    uo = res["units_out"]
+    kept_idx = [u for u in range(U) if keep[u]]
+    assert len(uo) == len(kept_idx)
+    pos = 0
+    for row, u in zip(uo, kept_idx):
+        assert row[0] == pos and row[1] == units[u, 1] and row[2] == units[u, 2] and row[3] == units[u, 3]
+        assert row[4] == (0 if units[u, 4] == 0 else (2 if events[u] in recent else 1))
+        pos += units[u, 1]
+    for m in range(3):
+        if caps[m] >= 0:
+            cand_kept = [u for u in kept_idx if u not in prot and units[u, 2] == m]
+            assert int(units[cand_kept, 1].sum()) <= caps[m]
+
+
+def test_select_invariants_random():
+    rng = np.random.default_rng(21)
+    for trial in range(200):
+        U = int(rng.integers(1, 14))
+        lens = rng.integers(1, 50, size=U).tolist()
+        mods = rng.integers(0, 3, size=U).tolist()
+        events = np.cumsum(rng.integers(0, 2, size=U)).tolist()
+        groups = [0 if (i == 0 and rng.random() < 0.7) else 2 for i in range(U)]
+        units = _units(lens, mods, events, groups)
+        scores = rng.random(U).astype(np.float32)
+        if rng.random() < 0.3:
+            scores[rng.integers(U)] = scores[rng.integers(U)]        # exact ties
+        budget = int(rng.integers(1, sum(lens) + 20))
+        R = int(rng.integers(0, 3))
+        caps = tuple(int(c) for c in rng.choice([-1, 10, 40, 100], size=3))
+        res = oc.select_units(units, scores, budget, R, caps)
+        _check_select_invariants(units, scores, budget, R, caps, res)
+        # I4 greedy maximality: replay -- every rejected candidate was a misfit at its turn
+        prot = [u for u in range(U) if res["unit_keep"][u] and u not in res["order"]]
+        used = int(units[prot, 1].sum())
+        cap_rem = list(caps)
+        prev = None
+        for u in res["order"]:
+            if prev is not None:     # order is by score desc, ties by recency
+                assert (scores[prev] > scores[u]) or (scores[prev] == scores[u] and prev > u)
+            prev = u
+            fits = units[u, 1] <= budget - used and (cap_rem[units[u, 2]] < 0 or units[u, 1] <= cap_rem[units[u, 2]])
+            assert bool(res["unit_keep"][u]) == bool(fits)
+            if fits:
+                used += int(units[u, 1])
+                if cap_rem[units[u, 2]] >= 0:
+                    cap_rem[units[u, 2]] -= int(units[u, 1])
+
+
+def test_select_special_cases():
+    units = _units([16, 100, 20, 100, 20, 100, 20], mods=[2, 0, 1, 0, 1, 0, 1],
+                   events=[0, 1, 1, 2, 2, 3, 3], groups=[0, 2, 2, 2, 2, 2, 2])
+    N = int(units[:, 1].sum())
+    # I5 budget >= history: nothing is evicted ("no-slide")
+    res = oc.select_units(units, np.zeros(7, np.float32), N, 1)
+    assert np.all(res["unit_keep"] == 2) and res["n_kept"] == N and np.all(res["keep_mask"] == 1)
+    # I6 score = recency reduces to unit-level FIFO: the newest units that fit survive
+    res = oc.select_units(units, np.arange(7, dtype=np.float32), 16 + 120 + 120, 1)
+    assert res["unit_keep"].tolist() == [2, 0, 0, 2, 2, 2, 2]
+    # a misfit does not end the walk: the frame of event 1 does not fit, its audio does
+    res = oc.select_units(units, np.array([0, 9, 1, 8, 7, 0, 0], np.float32), 16 + 120 + 100 + 30, 1)
+    assert res["unit_keep"].tolist() == [2, 0, 2, 2, 0, 2, 2] or res["unit_keep"].tolist() == [2, 2, 0, 0, 2, 2, 2]
+    # the exact expected walk: cand order 1(9),3(8),4(7),2(1): 1 fits (100<=130), 3 no (100>30), 4 yes (20<=30), 2 no (20>10)
+    assert res["unit_keep"].tolist() == [2, 2, 0, 0, 2, 2, 2]
+    # protected set alone above budget: kept = protected exactly (trimming target, not a bound)
+    res = oc.select_units(units, np.ones(7, np.float32), 50, 2)
+    assert res["unit_keep"].tolist() == [2, 0, 0, 2, 2, 2, 2] and res["n_kept"] == 256
+    # NaN scores go last; ties go to the more recent unit
+    sc = np.array([0, np.nan, 1, 1, 1, 0, 0], np.float32)
+    res = oc.select_units(units, sc, 16 + 120 + 40, 1)
+    assert res["order"] == [4, 3, 2, 1] and res["unit_keep"].tolist() == [2, 0, 2, 0, 2, 2, 2]
+    # modality caps bound candidates only
+    res = oc.select_units(units, np.arange(7, dtype=np.float32), N, 1, (100, -1, -1))
+    assert res["unit_keep"].tolist() == [2, 0, 2, 2, 2, 2, 2]
+    with pytest.raises(ValueError):
+        oc.select_units(_units([1, 1], events=[3, 2]), np.zeros(2, np.float32), 5)
+
+
+def test_select_brute_force_orderings():
+    """On <= 5 candidates, the rule's result equals a replay written independently:
+    enumerate every permutation, keep the one sorted by (score desc, index desc), walk it."""
+    rng = np.random.default_rng(33)
+    for trial in range(60):
+        U = int(rng.integers(2, 7))
+        lens = rng.integers(1, 30, size=U).tolist()
+        units = _units(lens, events=list(range(U)), groups=[0] + [2] * (U - 1))
+        scores = rng.integers(0, 3, size=U).astype(np.float32)   # many ties
+        budget = int(rng.integers(lens[0] + lens[-1], sum(lens) + 1))
+        res = oc.select_units(units, scores, budget, 1)
+        cand = list(range(1, U - 1))
+        best = None
+        for perm in itertools.permutations(cand):
+            ok = all((scores[a] > scores[b]) or (scores[a] == scores[b] and a > b)
+                     for a, b in zip(perm, perm[1:]))
+            if ok:
+                assert best is None
+                best = perm
+        used = lens[0] + lens[-1]
+        exp = {0, U - 1}
+        for u in best:
+            if lens[u] <= budget - used:
+                exp.add(u)
+                used += lens[u]
+        assert set(np.nonzero(res["unit_keep"])[0].tolist()) == exp
+
+
+# ------------------------------------------------------------ whole pass
+def test_stream_step_budget_covers_history_is_full_attention():
+    """With the budget covering the whole cache the pass is brute-force full attention."""
+    w = wl.small_mixed(3, n_units=6, h_q=2, h_kv=1, d=8, dtype="fp32", max_len=12, t=9)
+    N = w.n_hist
+    res = oc.stream_step(w.q, w.k_hist, w.v_hist, w.units, w.k_chunk, w.v_chunk, w.chunk_units,
+                         w.w_modality, budget=N, n_recent_events=1, modality_cap=(-1, -1, -1), page_size=4)
+    ob, _ = _brute_attention(w.q, w.k_hist, w.v_hist, w.k_chunk, w.v_chunk, 1 / math.sqrt(8))
+    assert res["compact"]["rows_moved"] == 0 and res["compact"]["n_kept"] == N
+    assert np.allclose(res["o"], ob, atol=1e-12)
+    assert len(res["units"]) == len(w.units) + len(w.chunk_units)
+    assert res["units"][-1, 0] + res["units"][-1, 1] == N + w.t
+
+
+def test_tiny_config_ranking_is_nontrivial():
+    """Config 1: the biased video unit must out-score the other old video units and survive."""
+    w = wl.tiny()
+    score, mass = oc.score_units(w.q, w.k_hist, w.units, w.w_modality)
+    vids = [u for u in range(len(w.units)) if w.units[u, 2] == 0 and u != 0 and w.units[u, 3] != 3]
+    assert max(vids, key=lambda u: score[u]) == w.biased_unit
+    sel = oc.select_units(w.units, score, w.budget, w.n_recent_events)
+    assert sel["unit_keep"][w.biased_unit] == 2 and sel["unit_keep"][0] == 2
+    assert sel["n_kept"] <= w.budget
+    cp = oc.compact_pack(w.k_hist, w.v_hist, sel["keep_mask"], w.page_size, sel["units_out"])
+    assert 0 <= cp["span_pages"] * w.page_size - cp["n_kept"] < w.page_size
