@@ -1,0 +1,251 @@
+/*
+ * omnitide.h -- C ABI of the B200 (sm_100a) per-chunk hot path of the OmniTide streaming loop.
+ *
+ * One pass per incoming chunk and per layer:
+ *     score units -> select units -> compact KV (OmniPage) -> append chunk -> chunk-prefill attention
+ *
+ * Conventions (all entry points)
+ *   - C99 ABI, no exceptions.  Every call returns an omni_status.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls enqueue device work on it and return; none
+ *     of them synchronises the host.  Errors the host can see (null / misaligned pointers, unsupported
+ *     geometry, capacity) are returned at once; errors found on the device (a bounded wait that ran
+ *     out, a malformed unit table) are OR-ed into a status word read with omnitide_poll_status().
+ *   - Pointers marked [dev] are device pointers, 16-byte aligned, owned by the caller.  Pointers
+ *     marked [host] are host pointers read before the call returns.  The library owns only the
+ *     context and the scratch memory it allocates inside omnitide_create().
+ *   - Counts that one step produces for the next live in device memory (`*_dev` arguments, int32).
+ *     A `*_dev` argument may be NULL, in which case the host bound `*_max` is the exact count.
+ *     `*_max` always bounds the device value and sizes the launch.
+ *   - Tensor layouts (row-major, dense):
+ *         Q        [T][h_q][d]          K/V cache  [S][h_kv][d]        O  [T][h_q][d]
+ *     One cache *row* = all KV heads of one token = h_kv*d elements.  Query head h reads KV head
+ *     h / (h_q / h_kv).  dtype 0 = bf16 storage, 1 = fp32 storage; accumulation is always fp32.
+ *   - Unit table: array of omni_unit in logical (time) order, contiguous: units[u+1].start ==
+ *     units[u].start + units[u].len, units[0].start == 0; `event` ids are non-decreasing.
+ */
+#ifndef OMNITIDE_H
+#define OMNITIDE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t omni_status;
+enum {
+    OMNI_OK = 0,
+    OMNI_ERR_INVALID_ARG = 1,
+    OMNI_ERR_UNSUPPORTED = 2,
+    OMNI_ERR_CUDA = 3,
+    OMNI_ERR_TIMEOUT = 4,
+    OMNI_ERR_CAPACITY = 5
+};
+
+/* bits of the device status word (omnitide_poll_status) */
+enum {
+    OMNI_DEV_TIMEOUT = 1,      /* a bounded on-device wait ran out */
+    OMNI_DEV_BAD_UNITS = 2,    /* unit table not contiguous / events decreasing / count above capacity */
+    OMNI_DEV_BAD_COUNT = 4     /* a device-side count exceeded its host bound */
+};
+
+enum { OMNI_DTYPE_BF16 = 0, OMNI_DTYPE_FP32 = 1 };
+enum { OMNI_MOD_VIDEO = 0, OMNI_MOD_AUDIO = 1, OMNI_MOD_TEXT = 2 };
+/* retention groups / allocation classes (Section 4 "OmniPick"; Section 6.1 "Placing entries") */
+enum { OMNI_GROUP_MUST_KEEP = 0, OMNI_GROUP_SELECTED = 1, OMNI_GROUP_RECENT = 2 };
+enum { OMNI_KEEP_DROPPED = 0, OMNI_KEEP_SINK_PREFIX = 1 /* reserved */, OMNI_KEEP_WHOLE = 2 };
+enum { OMNI_PAGE_EMPTY = 255 };
+enum { OMNI_COMPACT_PACK = 0 };
+
+typedef struct {
+    int32_t h_q, h_kv, d;
+    int32_t dtype;      /* OMNI_DTYPE_* of Q/K/V storage */
+    int32_t s_cap;      /* largest history (cache slots) any call will pass */
+    int32_t u_cap;      /* largest number of history units */
+    int32_t t_cap;      /* largest chunk (tokens) */
+} omni_geometry;
+
+/* One typed span of the stream (Section 2.1 "Streaming units"; Section 5.2 unit records). */
+typedef struct {
+    int32_t start;      /* first token: cache slot (history) or row in the chunk (chunk units) */
+    int32_t len;        /* tokens, > 0 */
+    int32_t modality;   /* OMNI_MOD_* */
+    int32_t event;      /* streaming event the span belongs to */
+    int32_t group;      /* OMNI_GROUP_* */
+    int32_t flags;      /* opaque, carried through */
+} omni_unit;
+
+typedef struct {
+    int32_t budget;             /* retained-history target in tokens (low watermark, Section 5.1) */
+    int32_t n_recent_events;    /* newest events kept whole */
+    int32_t modality_cap[3];    /* per-modality token cap on selected (non-protected) units; <0 = none */
+} omni_select_params;
+
+/* Integer results of one compaction, written to device memory. */
+typedef struct {
+    int32_t n_kept;         /* rows retained */
+    int32_t span_pages;     /* ceil(n_kept / page_size): page-rounded physical span (Section 6.2) */
+    int32_t rows_moved;     /* retained rows whose slot changed */
+    int32_t part_begin[4];  /* first slot of must-keep, selected-history, recent-context, end */
+    int32_t reserved;
+} omni_compact_info;
+
+typedef struct omnitide_ctx omnitide_ctx;
+
+/* Creates a context for one geometry on the current device and allocates its scratch memory.
+ * Returns OMNI_ERR_UNSUPPORTED for h_q % h_kv != 0, d not a multiple of 8 or > 256, or a device
+ * that is not sm_100; OMNI_ERR_CUDA if an allocation fails.  *ctx_out is NULL on failure. */
+omni_status omnitide_create(omnitide_ctx** ctx_out, const omni_geometry* geometry /*[host]*/);
+omni_status omnitide_destroy(omnitide_ctx* ctx);
+
+/* Copies the device status word (OMNI_DEV_* bits, 0 = clean) to *device_status_out [host] and
+ * clears it.  Synchronises `stream` first. */
+omni_status omnitide_poll_status(omnitide_ctx* ctx, void* stream, int32_t* device_status_out);
+
+/* Text of the last host-side error on this context (static storage inside the context). */
+const char* omnitide_last_error(const omnitide_ctx* ctx);
+
+/*
+ * (a1) Unit scoring.  For every history unit u:
+ *      s_hij  = scale * <Q[i][h], K[j][h / G]>                 i < t, j < n_hist
+ *      a_hij  = softmax over the n_hist history keys of s_hij   (chunk keys excluded)
+ *      mass_u = (1 / (h_q * t)) * sum over h, i and j in u of a_hij
+ *      score_u = w_modality[modality_u] * mass_u * n_hist / len_u
+ * This is the per-span averaged attention weight that the paper's design study measures offline
+ * (Section 5, "Key insight"), weighted per modality ("Modality-asymmetric attention"); the paper's
+ * own OmniPick is score-free, so the formula is this library's reading, not the paper's.
+ *   q [dev] t*h_q*d, k_cache [dev] rows 0..n_hist-1 used, units [dev] n_units entries,
+ *   w_modality [host] 3 floats, scale <= 0 means 1/sqrt(d),
+ *   scores_out [dev] n_units_max floats, mass_out [dev] nullable.
+ * The QK^T contraction runs on tcgen05 tensor cores for bf16 with d == 128, on CUDA cores otherwise.
+ */
+omni_status omnitide_score_units(omnitide_ctx* ctx, void* stream,
+                                 const void* q, int32_t t,
+                                 const void* k_cache, const int32_t* n_hist_dev, int32_t n_hist_max,
+                                 const omni_unit* units, const int32_t* n_units_dev, int32_t n_units_max,
+                                 const float* w_modality, float scale,
+                                 float* scores_out, float* mass_out);
+
+/*
+ * (a2) Budgeted unit selection (Section 5.1 for what the paper fixes: protected prefix, newest
+ * events kept whole, spans never cut at a token position, the budget a trimming target).
+ *   1. protected = units of group must-keep, plus every unit of the n_recent_events newest events;
+ *   2. if the protected tokens already reach the budget, exactly the protected set is kept;
+ *   3. otherwise the other units are visited by descending score (ties: later unit first, NaN last)
+ *      and one is taken iff it fits the remaining budget and its modality's remaining cap;
+ *   4. survivors are re-indexed (Section 5.2): units_out holds the kept units in order with `start`
+ *      = kept tokens before them, modality/event/flags preserved, group = must-keep if it was,
+ *      else recent-context if in a newest event, else selected-history.
+ * Outputs [dev]: unit_keep_out[n_units] (OMNI_KEEP_*), keep_mask_out[n_hist] (1 = retained),
+ * n_kept_out, units_out (capacity n_units_max), n_units_out.
+ */
+omni_status omnitide_select_units(omnitide_ctx* ctx, void* stream,
+                                  const omni_unit* units, const int32_t* n_units_dev, int32_t n_units_max,
+                                  const float* scores, const omni_select_params* params /*[host]*/,
+                                  uint8_t* unit_keep_out, uint8_t* keep_mask_out, int32_t n_hist_max,
+                                  int32_t* n_kept_out, omni_unit* units_out, int32_t* n_units_out);
+
+/*
+ * (a3) OmniPage eager compaction (Section 6, "Compaction-movement trade-off": pack every retained
+ * entry into a contiguous prefix; Section 6.1 for allocation classes and page promotion; Section 6.2
+ * for the page-rounded span and for copy semantics: reads of all sources precede all writes).
+ *   for s in [0, s_span): if keep_mask[s]: slot_map[s] = n; dst[n] = src[s]; n++   else slot_map[s] = -1
+ * Rows are copied bit for bit.  k_dst/v_dst may be different buffers (one read + one write per row,
+ * no staging) or equal to k_src/v_src (in place: rows are staged through context scratch).
+ * Because units are in time order and group rank grows with recency, the stable pack is already the
+ * retention-partitioned order must-keep | selected-history | recent-context; part_begin reports the
+ * partition starts from units_kept (the table omnitide_select_units wrote; may be NULL).
+ * page_class_out[p] for p < ceil(s_span_max / page_size): 0 if page p holds a must-keep row, else 1 if
+ * it holds page_size retained rows (promoted to selected-history), else 2 if partly filled (stays
+ * recent-context), else OMNI_PAGE_EMPTY.
+ *   slot_map_out [dev] s_span_max int32 (nullable), info_out [dev], page_class_out [dev] nullable.
+ * mode must be OMNI_COMPACT_PACK.
+ */
+omni_status omnipage_compact(omnitide_ctx* ctx, void* stream,
+                             const void* k_src, const void* v_src, void* k_dst, void* v_dst,
+                             const uint8_t* keep_mask, const int32_t* s_span_dev, int32_t s_span_max,
+                             int32_t page_size, int32_t mode,
+                             const omni_unit* units_kept, const int32_t* n_units_kept_dev, int32_t n_units_max,
+                             int32_t* slot_map_out, omni_compact_info* info_out, uint8_t* page_class_out);
+
+/*
+ * (a5) Append: new entries enter the recent-context class behind the retained history
+ * (Section 6.1).  Copies the chunk's t K/V rows to cache slots [n_kept, n_kept + t), appends the
+ * chunk's units to `units` with start += n_kept and group = recent-context, and writes
+ * *n_hist_out = n_kept + t, *n_units_out = n_units + n_chunk_units.
+ *   n_kept_dev, n_units_dev [dev] in; chunk_units [dev]; n_hist_out / n_units_out [dev] may alias
+ *   the inputs.  s_cap / u_cap overflow sets OMNI_DEV_BAD_COUNT and copies nothing.
+ */
+omni_status omnipage_append(omnitide_ctx* ctx, void* stream,
+                            void* k_cache, void* v_cache, const int32_t* n_kept_dev,
+                            const void* k_chunk, const void* v_chunk, int32_t t,
+                            omni_unit* units, const int32_t* n_units_dev,
+                            const omni_unit* chunk_units, int32_t n_chunk_units,
+                            int32_t* n_hist_out, int32_t* n_units_out);
+
+/*
+ * (a4) GQA chunk-prefill attention (Section 2.1 prefill; Section 3 "Dense attention"):
+ *      O[i][h] = sum_j softmax_j(scale * <Q[i][h], k_j>) v_j
+ * over j in history rows [0, n_hist) followed by chunk rows [0, i] (causal inside the chunk,
+ * diagonal included).  k_chunk/v_chunk may point into the cache behind the history.
+ *   o_out [dev] t*h_q*d of out_dtype (OMNI_DTYPE_*), lse_out [dev] t*h_q floats, nullable
+ *   (natural-log sum of exponentials of the scaled logits).
+ * bf16 with d == 128 runs on tcgen05 tensor cores (TMA-fed, TMEM accumulators); other geometries
+ * run on CUDA cores in fp32.
+ */
+omni_status omnitide_chunk_attention(omnitide_ctx* ctx, void* stream,
+                                     const void* q, int32_t t,
+                                     const void* k_hist, const void* v_hist,
+                                     const int32_t* n_hist_dev, int32_t n_hist_max,
+                                     const void* k_chunk, const void* v_chunk,
+                                     float scale, void* o_out, int32_t out_dtype, float* lse_out);
+
+/*
+ * One whole pass (a1..a5 in order) for one layer with every tensor resident on the device.
+ * State in: k_cache/v_cache rows [0, *n_hist_dev), units[0, *n_units_dev).  State out: the compacted
+ * history plus the chunk in k_cache_out/v_cache_out (must be different buffers), units_out, and the
+ * updated counts in n_hist_out / n_units_out.  Work buffers for scores, masks and the slot map come
+ * from the context.  o_out as in omnitide_chunk_attention; info_out nullable.
+ */
+omni_status omnitide_chunk_step(omnitide_ctx* ctx, void* stream,
+                                const void* q, const void* k_chunk, const void* v_chunk, int32_t t,
+                                const omni_unit* chunk_units, int32_t n_chunk_units,
+                                const void* k_cache, const void* v_cache,
+                                const int32_t* n_hist_dev, int32_t n_hist_max,
+                                const omni_unit* units, const int32_t* n_units_dev, int32_t n_units_max,
+                                const float* w_modality, const omni_select_params* params, int32_t page_size,
+                                float scale,
+                                void* k_cache_out, void* v_cache_out, omni_unit* units_out,
+                                int32_t* n_hist_out, int32_t* n_units_out,
+                                void* o_out, int32_t out_dtype, omni_compact_info* info_out);
+
+/*
+ * The same pass for a caller whose chunk lives in host memory: q/k_chunk/v_chunk/chunk_units are
+ * HOST pointers (pinned memory recommended) copied to context staging buffers on `stream`, and the
+ * attention output is copied back to o_host (out_dtype elements).  The call returns after the
+ * copies and kernels are enqueued; synchronise the stream before reading o_host.
+ */
+omni_status omnitide_chunk_step_host(omnitide_ctx* ctx, void* stream,
+                                     const void* q_host, const void* k_chunk_host, const void* v_chunk_host, int32_t t,
+                                     const omni_unit* chunk_units_host, int32_t n_chunk_units,
+                                     const void* k_cache, const void* v_cache,
+                                     const int32_t* n_hist_dev, int32_t n_hist_max,
+                                     const omni_unit* units, const int32_t* n_units_dev, int32_t n_units_max,
+                                     const float* w_modality, const omni_select_params* params, int32_t page_size,
+                                     float scale,
+                                     void* k_cache_out, void* v_cache_out, omni_unit* units_out,
+                                     int32_t* n_hist_out, int32_t* n_units_out,
+                                     void* o_host, int32_t out_dtype, omni_compact_info* info_out);
+
+/* Options.  OMNI_OPT_FORCE_CUDA_CORES != 0 routes scoring and attention through the fp32 CUDA-core
+ * kernels even where the tensor-core kernels apply (a second implementation for cross-checks). */
+enum { OMNI_OPT_FORCE_CUDA_CORES = 1 };
+omni_status omnitide_set_option(omnitide_ctx* ctx, int32_t option, int32_t value);
+
+/* Number of kernels this library has launched on this context since creation (for accounting). */
+int64_t omnitide_launch_count(const omnitide_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OMNITIDE_H */

@@ -1,0 +1,219 @@
+// Context life cycle, dispatch between the tensor-core and CUDA-core paths, and the whole-pass calls.
+#include "common.cuh"
+
+#include <new>
+
+namespace {
+
+bool tc_geometry(const omnitide_ctx* ctx) {
+    return ctx->g.dtype == OMNI_DTYPE_BF16 && ctx->g.d == 128 && !ctx->force_cuda_cores;
+}
+
+template <typename T>
+cudaError_t alloc(T** p, size_t n) {
+    *p = nullptr;
+    return cudaMalloc(reinterpret_cast<void**>(p), n ? n * sizeof(T) : sizeof(T));
+}
+
+void free_all(omnitide_ctx* c) {
+    void* ptrs[] = {c->status_dev, c->score_part, c->score_tile_mass, c->score_mass64, c->inplace_k, c->inplace_v,
+                    c->ws_scores, c->ws_unit_keep, c->ws_keep_mask, c->ws_slot_map, c->ws_counts, c->ws_info, c->st_q,
+                    c->st_k, c->st_v, c->st_o, c->st_units, c->attn_part_o, c->attn_part_ml};
+    for (void* p : ptrs)
+        if (p) cudaFree(p);
+}
+
+}  // namespace
+
+extern "C" omni_status omnitide_create(omnitide_ctx** ctx_out, const omni_geometry* g) {
+    if (!ctx_out) return OMNI_ERR_INVALID_ARG;
+    *ctx_out = nullptr;
+    if (!g) return OMNI_ERR_INVALID_ARG;
+    if (g->h_q <= 0 || g->h_kv <= 0 || g->h_q % g->h_kv != 0 || g->d <= 0 || g->d % 8 != 0 || g->d > 256 ||
+        (g->dtype != OMNI_DTYPE_BF16 && g->dtype != OMNI_DTYPE_FP32) || g->s_cap <= 0 || g->u_cap <= 0 || g->t_cap <= 0)
+        return OMNI_ERR_UNSUPPORTED;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return OMNI_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return OMNI_ERR_CUDA;
+    if (prop.major != 10) return OMNI_ERR_UNSUPPORTED;      // built for sm_100a only
+    omnitide_ctx* c = new (std::nothrow) omnitide_ctx();
+    if (!c) return OMNI_ERR_CUDA;
+    memset(c, 0, sizeof(*c));
+    c->g = *g;
+    c->device = dev;
+    c->sm_count = prop.multiProcessorCount;
+    c->es = g->dtype == OMNI_DTYPE_BF16 ? 2 : 4;
+    c->row_bytes = (size_t)g->h_kv * g->d * c->es;
+    const size_t row_tiles = ((size_t)g->t_cap + 127) / 128 * g->h_q;
+    const size_t q_elems = (size_t)g->t_cap * g->h_q * g->d;
+    bool ok = true;
+    ok &= alloc(&c->status_dev, 1) == cudaSuccess;
+    ok &= alloc(&c->score_part, row_tiles * g->u_cap * 128) == cudaSuccess;
+    ok &= alloc(&c->score_tile_mass, row_tiles * g->u_cap) == cudaSuccess;
+    ok &= alloc(&c->score_mass64, (size_t)g->u_cap) == cudaSuccess;
+    ok &= alloc(&c->ws_scores, (size_t)g->u_cap) == cudaSuccess;
+    ok &= alloc(&c->ws_unit_keep, (size_t)g->u_cap + 16) == cudaSuccess;
+    ok &= alloc(&c->ws_keep_mask, (size_t)g->s_cap + 16) == cudaSuccess;
+    ok &= alloc(&c->ws_slot_map, (size_t)g->s_cap + 16) == cudaSuccess;
+    ok &= alloc(&c->ws_counts, 4) == cudaSuccess;
+    ok &= alloc(&c->ws_info, 1) == cudaSuccess;
+    ok &= cudaMalloc(&c->st_q, q_elems * c->es) == cudaSuccess;
+    ok &= cudaMalloc(&c->st_k, (size_t)g->t_cap * c->row_bytes) == cudaSuccess;
+    ok &= cudaMalloc(&c->st_v, (size_t)g->t_cap * c->row_bytes) == cudaSuccess;
+    ok &= cudaMalloc(&c->st_o, q_elems * 4) == cudaSuccess;
+    ok &= alloc(&c->st_units, 64) == cudaSuccess;
+    if (ok) ok = cudaMemset(c->status_dev, 0, sizeof(int32_t)) == cudaSuccess;
+    if (ok) {
+        cudaDriverEntryPointQueryResult qres;
+        void* fn = nullptr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            c->encode_tiled = fn;
+        else
+            ok = false;
+    }
+    if (!ok) {
+        cudaGetLastError();
+        free_all(c);
+        delete c;
+        return OMNI_ERR_CUDA;
+    }
+    *ctx_out = c;
+    return OMNI_OK;
+}
+
+extern "C" omni_status omnitide_destroy(omnitide_ctx* ctx) {
+    if (!ctx) return OMNI_ERR_INVALID_ARG;
+    cudaDeviceSynchronize();
+    free_all(ctx);
+    delete ctx;
+    return OMNI_OK;
+}
+
+extern "C" omni_status omnitide_poll_status(omnitide_ctx* ctx, void* stream, int32_t* out) {
+    if (!ctx || !out) return OMNI_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    OMNI_CUDA(ctx, cudaMemcpyAsync(out, ctx->status_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    OMNI_CUDA(ctx, cudaMemsetAsync(ctx->status_dev, 0, sizeof(int32_t), st));
+    OMNI_CUDA(ctx, cudaStreamSynchronize(st));
+    return OMNI_OK;
+}
+
+extern "C" const char* omnitide_last_error(const omnitide_ctx* ctx) { return ctx ? ctx->err : "null context"; }
+extern "C" int64_t omnitide_launch_count(const omnitide_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+extern "C" omni_status omnitide_set_option(omnitide_ctx* ctx, int32_t option, int32_t value) {
+    if (!ctx) return OMNI_ERR_INVALID_ARG;
+    if (option == OMNI_OPT_FORCE_CUDA_CORES) { ctx->force_cuda_cores = value != 0; return OMNI_OK; }
+    OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "unknown option %d", option);
+}
+
+extern "C" omni_status omnitide_score_units(omnitide_ctx* ctx, void* stream, const void* q, int32_t t,
+                                            const void* k_cache, const int32_t* n_hist_dev, int32_t n_hist_max,
+                                            const omni_unit* units, const int32_t* n_units_dev, int32_t n_units_max,
+                                            const float* w_modality, float scale, float* scores_out, float* mass_out) {
+    if (!ctx) return OMNI_ERR_INVALID_ARG;
+    if (!q || !k_cache || !units || !w_modality || !scores_out) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "score: null pointer");
+    if (t <= 0 || t > ctx->g.t_cap) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "score: t %d outside (0, t_cap]", t);
+    if (n_hist_max <= 0 || n_hist_max > ctx->g.s_cap) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "score: n_hist_max outside (0, s_cap]");
+    if (n_units_max <= 0 || n_units_max > ctx->g.u_cap) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "score: n_units_max outside (0, u_cap]");
+    if (!omni_aligned16(q) || !omni_aligned16(k_cache)) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "score: q/k_cache must be 16-byte aligned");
+    if (scale <= 0.f) scale = 1.0f / sqrtf((float)ctx->g.d);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (tc_geometry(ctx))
+        return omni_score_tc(ctx, st, q, t, k_cache, n_hist_dev, n_hist_max, units, n_units_dev, n_units_max, w_modality,
+                             scale, scores_out, mass_out);
+    return omni_score_simple(ctx, st, q, t, k_cache, n_hist_dev, n_hist_max, units, n_units_dev, n_units_max, w_modality,
+                             scale, scores_out, mass_out);
+}
+
+extern "C" omni_status omnitide_chunk_attention(omnitide_ctx* ctx, void* stream, const void* q, int32_t t,
+                                                const void* k_hist, const void* v_hist, const int32_t* n_hist_dev,
+                                                int32_t n_hist_max, const void* k_chunk, const void* v_chunk, float scale,
+                                                void* o_out, int32_t out_dtype, float* lse_out) {
+    if (!ctx) return OMNI_ERR_INVALID_ARG;
+    if (!q || !k_chunk || !v_chunk || !o_out) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "attention: null pointer");
+    if (n_hist_max > 0 && (!k_hist || !v_hist)) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "attention: history pointers are null");
+    if (t <= 0 || t > ctx->g.t_cap) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "attention: t %d outside (0, t_cap]", t);
+    if (n_hist_max < 0 || n_hist_max > ctx->g.s_cap) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "attention: n_hist_max outside [0, s_cap]");
+    if (out_dtype != OMNI_DTYPE_BF16 && out_dtype != OMNI_DTYPE_FP32) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "attention: bad out_dtype");
+    if (!omni_aligned16(q) || !omni_aligned16(k_hist) || !omni_aligned16(v_hist) || !omni_aligned16(k_chunk) ||
+        !omni_aligned16(v_chunk) || !omni_aligned16(o_out))
+        OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "attention: pointers must be 16-byte aligned");
+    if (scale <= 0.f) scale = 1.0f / sqrtf((float)ctx->g.d);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (tc_geometry(ctx))
+        return omni_attention_tc(ctx, st, q, t, k_hist, v_hist, n_hist_dev, n_hist_max, k_chunk, v_chunk, scale, o_out,
+                                 out_dtype, lse_out);
+    return omni_attention_simple(ctx, st, q, t, k_hist, v_hist, n_hist_dev, n_hist_max, k_chunk, v_chunk, scale, o_out,
+                                 out_dtype, lse_out);
+}
+
+extern "C" omni_status omnitide_chunk_step(omnitide_ctx* ctx, void* stream, const void* q, const void* k_chunk,
+                                           const void* v_chunk, int32_t t, const omni_unit* chunk_units,
+                                           int32_t n_chunk_units, const void* k_cache, const void* v_cache,
+                                           const int32_t* n_hist_dev, int32_t n_hist_max, const omni_unit* units,
+                                           const int32_t* n_units_dev, int32_t n_units_max, const float* w_modality,
+                                           const omni_select_params* params, int32_t page_size, float scale,
+                                           void* k_cache_out, void* v_cache_out, omni_unit* units_out, int32_t* n_hist_out,
+                                           int32_t* n_units_out, void* o_out, int32_t out_dtype,
+                                           omni_compact_info* info_out) {
+    if (!ctx) return OMNI_ERR_INVALID_ARG;
+    if (!k_cache_out || !v_cache_out || k_cache_out == k_cache || v_cache_out == v_cache)
+        OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "chunk_step: output caches must be distinct buffers");
+    if (!units_out || !n_hist_out || !n_units_out || !params) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "chunk_step: null pointer");
+    int32_t* n_kept = ctx->ws_counts;
+    int32_t* n_units_kept = ctx->ws_counts + 1;
+    omni_compact_info* info = info_out ? info_out : ctx->ws_info;
+    omni_status s;
+    s = omnitide_score_units(ctx, stream, q, t, k_cache, n_hist_dev, n_hist_max, units, n_units_dev, n_units_max,
+                             w_modality, scale, ctx->ws_scores, nullptr);
+    if (s) return s;
+    s = omnitide_select_units(ctx, stream, units, n_units_dev, n_units_max, ctx->ws_scores, params, ctx->ws_unit_keep,
+                              ctx->ws_keep_mask, n_hist_max, n_kept, units_out, n_units_kept);
+    if (s) return s;
+    s = omnipage_compact(ctx, stream, k_cache, v_cache, k_cache_out, v_cache_out, ctx->ws_keep_mask, n_hist_dev,
+                         n_hist_max, page_size, OMNI_COMPACT_PACK, units_out, n_units_kept, n_units_max, ctx->ws_slot_map,
+                         info, nullptr);
+    if (s) return s;
+    s = omnitide_chunk_attention(ctx, stream, q, t, k_cache_out, v_cache_out, n_kept, n_hist_max, k_chunk, v_chunk, scale,
+                                 o_out, out_dtype, nullptr);
+    if (s) return s;
+    return omnipage_append(ctx, stream, k_cache_out, v_cache_out, n_kept, k_chunk, v_chunk, t, units_out, n_units_kept,
+                           chunk_units, n_chunk_units, n_hist_out, n_units_out);
+}
+
+extern "C" omni_status omnitide_chunk_step_host(omnitide_ctx* ctx, void* stream, const void* q_host,
+                                                const void* k_chunk_host, const void* v_chunk_host, int32_t t,
+                                                const omni_unit* chunk_units_host, int32_t n_chunk_units,
+                                                const void* k_cache, const void* v_cache, const int32_t* n_hist_dev,
+                                                int32_t n_hist_max, const omni_unit* units, const int32_t* n_units_dev,
+                                                int32_t n_units_max, const float* w_modality,
+                                                const omni_select_params* params, int32_t page_size, float scale,
+                                                void* k_cache_out, void* v_cache_out, omni_unit* units_out,
+                                                int32_t* n_hist_out, int32_t* n_units_out, void* o_host, int32_t out_dtype,
+                                                omni_compact_info* info_out) {
+    if (!ctx) return OMNI_ERR_INVALID_ARG;
+    if (!q_host || !k_chunk_host || !v_chunk_host || !o_host || (n_chunk_units > 0 && !chunk_units_host))
+        OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "chunk_step_host: null pointer");
+    if (t <= 0 || t > ctx->g.t_cap) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "chunk_step_host: t %d outside (0, t_cap]", t);
+    if (n_chunk_units < 0 || n_chunk_units > 64) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "chunk_step_host: more than 64 chunk units");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t q_bytes = (size_t)t * ctx->g.h_q * ctx->g.d * ctx->es;
+    const size_t kv_bytes = (size_t)t * ctx->row_bytes;
+    OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->st_q, q_host, q_bytes, cudaMemcpyHostToDevice, st));
+    OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->st_k, k_chunk_host, kv_bytes, cudaMemcpyHostToDevice, st));
+    OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->st_v, v_chunk_host, kv_bytes, cudaMemcpyHostToDevice, st));
+    if (n_chunk_units)
+        OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->st_units, chunk_units_host, sizeof(omni_unit) * n_chunk_units,
+                                       cudaMemcpyHostToDevice, st));
+    omni_status s = omnitide_chunk_step(ctx, stream, ctx->st_q, ctx->st_k, ctx->st_v, t, ctx->st_units, n_chunk_units,
+                                        k_cache, v_cache, n_hist_dev, n_hist_max, units, n_units_dev, n_units_max,
+                                        w_modality, params, page_size, scale, k_cache_out, v_cache_out, units_out,
+                                        n_hist_out, n_units_out, ctx->st_o, out_dtype, info_out);
+    if (s) return s;
+    const size_t o_bytes = (size_t)t * ctx->g.h_q * ctx->g.d * (out_dtype == OMNI_DTYPE_FP32 ? 4 : 2);
+    OMNI_CUDA(ctx, cudaMemcpyAsync(o_host, ctx->st_o, o_bytes, cudaMemcpyDeviceToHost, st));
+    return OMNI_OK;
+}

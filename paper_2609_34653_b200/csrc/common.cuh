@@ -1,0 +1,85 @@
+// Shared host-side definitions of the library: the context, error helpers, launch accounting.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "../../include/omnitide.h"
+
+struct omnitide_ctx {
+    omni_geometry g;
+    int device;
+    int sm_count;
+    int es;                       // element size of the storage dtype
+    size_t row_bytes;             // h_kv * d * es : one cache row
+    int32_t* status_dev;          // device status word (OMNI_DEV_* bits)
+    // ---- scratch owned by the context -------------------------------------------------
+    float2* score_part;           // [row tiles][u_cap][128] per-(row, unit) (max, sum) partials
+    float* score_tile_mass;       // [row tiles][u_cap] per-tile unit mass
+    double* score_mass64;         // [u_cap] accumulator of the CUDA-core scoring path
+    int32_t* score_seg;           // unit boundaries per key block (built per call)
+    void* inplace_k;              // staging for in-place compaction, allocated on first use
+    void* inplace_v;
+    size_t inplace_rows;
+    // work buffers of omnitide_chunk_step
+    float* ws_scores;             // [u_cap]
+    uint8_t* ws_unit_keep;        // [u_cap]
+    uint8_t* ws_keep_mask;        // [s_cap]
+    int32_t* ws_slot_map;         // [s_cap]
+    int32_t* ws_counts;           // {n_kept, n_units_kept}
+    omni_compact_info* ws_info;
+    // staging of omnitide_chunk_step_host
+    void* st_q; void* st_k; void* st_v; void* st_o; omni_unit* st_units;
+    // attention split-KV partials
+    float* attn_part_o;           // allocated on first use
+    float* attn_part_ml;
+    size_t attn_part_cap;
+    // -----------------------------------------------------------------------------------
+    void* encode_tiled;           // cuTensorMapEncodeTiled, resolved through the runtime
+    int64_t launches;
+    bool force_cuda_cores;        // OMNI_OPT_FORCE_CUDA_CORES
+    char err[256];
+};
+
+#define OMNI_FAIL(ctx, code, ...)                                   \
+    do {                                                            \
+        if (ctx) snprintf((ctx)->err, sizeof((ctx)->err), __VA_ARGS__); \
+        return (code);                                              \
+    } while (0)
+
+#define OMNI_CUDA(ctx, expr)                                                          \
+    do {                                                                              \
+        cudaError_t e__ = (expr);                                                     \
+        if (e__ != cudaSuccess)                                                       \
+            OMNI_FAIL(ctx, OMNI_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e__)); \
+    } while (0)
+
+#define OMNI_CHECK_LAUNCH(ctx, name)                                                   \
+    do {                                                                               \
+        cudaError_t e__ = cudaGetLastError();                                          \
+        if (e__ != cudaSuccess)                                                        \
+            OMNI_FAIL(ctx, OMNI_ERR_CUDA, "launch %s: %s", name, cudaGetErrorString(e__)); \
+        (ctx)->launches++;                                                             \
+    } while (0)
+
+static inline bool omni_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+// internal entry points implemented per file
+omni_status omni_attention_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q, int t, const void* k_hist,
+                              const void* v_hist, const int32_t* n_hist_dev, int n_hist_max, const void* k_chunk,
+                              const void* v_chunk, float scale, void* o_out, int out_dtype, float* lse_out);
+omni_status omni_score_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q, int t, const void* k_cache,
+                          const int32_t* n_hist_dev, int n_hist_max, const omni_unit* units,
+                          const int32_t* n_units_dev, int n_units_max, const float* w, float scale,
+                          float* scores_out, float* mass_out);
+omni_status omni_attention_simple(omnitide_ctx* ctx, cudaStream_t st, const void* q, int t, const void* k_hist,
+                                  const void* v_hist, const int32_t* n_hist_dev, int n_hist_max, const void* k_chunk,
+                                  const void* v_chunk, float scale, void* o_out, int out_dtype, float* lse_out);
+omni_status omni_score_simple(omnitide_ctx* ctx, cudaStream_t st, const void* q, int t, const void* k_cache,
+                              const int32_t* n_hist_dev, int n_hist_max, const omni_unit* units,
+                              const int32_t* n_units_dev, int n_units_max, const float* w, float scale,
+                              float* scores_out, float* mass_out);

@@ -1,0 +1,380 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, element by element."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import omni_oracle as oc
+from paper_2609_34653_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+ATT_MAX_ABS, ATT_MEAN_ABS = 1e-2, 1e-3       # attention tolerance on fp32 outputs
+SCORE_REL = 1e-3                              # unit scores, relative
+TIE_REL = 1e-4                                # score gap below which the selected set may differ
+
+
+@pytest.fixture(scope="module")
+def H():
+    from tests import gpu_helpers
+    return gpu_helpers
+
+
+@pytest.fixture(scope="module")
+def ob():
+    from paper_2609_34653_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def cfg2():
+    return wl.layer_8b()
+
+
+# ------------------------------------------------------------------------------------ compaction
+@pytest.mark.parametrize("S,rowshape,dtype,page,density", [
+    (1, (1, 64), torch.float32, 16, 1.0),
+    (17, (1, 64), torch.float32, 16, 0.5),
+    (2048, (1, 64), torch.float32, 16, 0.5),
+    (1000, (8, 128), torch.bfloat16, 64, 0.3),
+    (5000, (2, 64), torch.bfloat16, 256, 0.9),
+    (16384, (8, 128), torch.bfloat16, 64, 0.25),
+    (80000, (8, 128), torch.bfloat16, 64, 0.1),
+])
+@pytest.mark.parametrize("in_place", [False, True])
+def test_compact_bit_exact(H, ob, S, rowshape, dtype, page, density, in_place):
+    rng = np.random.default_rng(S + 7 * in_place)
+    mask = (rng.random(S) < density).astype(np.uint8)
+    es = 2 if dtype == torch.bfloat16 else 4
+    raw = rng.integers(0, 256, size=(2, S, rowshape[0] * rowshape[1] * es), dtype=np.uint8)
+    k = torch.from_numpy(raw[0]).cuda().view(dtype).view(S, *rowshape).contiguous()
+    v = torch.from_numpy(raw[1]).cuda().view(dtype).view(S, *rowshape).contiguous()
+    exp = oc.compact_pack(raw[0], raw[1], mask, page)
+    ctx = ob.Context(4 * rowshape[0], rowshape[0], rowshape[1], "bf16" if es == 2 else "fp32", S + 64, 8, 16)
+    got = H.gpu_compact(ctx, k, v, mask, page, in_place=in_place, s_span_max=S + 40)
+    n = exp["n_kept"]
+    assert (got["n_kept"], got["span_pages"], got["rows_moved"]) == (n, exp["span_pages"], exp["rows_moved"])
+    assert np.array_equal(got["slot_map"], exp["slot_map"])
+    assert np.array_equal(H.bytes_of(got["k"][:n]).reshape(n, -1), exp["k"])
+    assert np.array_equal(H.bytes_of(got["v"][:n]).reshape(n, -1), exp["v"])
+    n_pages = (S + 40 + page - 1) // page
+    exp_pc = np.full(n_pages, 255, np.uint8)
+    exp_pc[:len(exp["page_class"])] = exp["page_class"]
+    assert np.array_equal(got["page_class"], exp_pc)
+    ctx.close()
+
+
+def test_compact_edges_and_partitions(H, ob):
+    rng = np.random.default_rng(1)
+    S = 300
+    k = torch.from_numpy(rng.standard_normal((S, 2, 64)).astype(np.float32)).cuda()
+    v = torch.from_numpy(rng.standard_normal((S, 2, 64)).astype(np.float32)).cuda()
+    ctx = ob.Context(4, 2, 64, "fp32", 512, 16, 16)
+    # none kept / all kept
+    got = H.gpu_compact(ctx, k, v, np.zeros(S, np.uint8), 16)
+    assert (got["n_kept"], got["span_pages"], got["rows_moved"]) == (0, 0, 0) and np.all(got["slot_map"] == -1)
+    assert np.all(got["page_class"] == 255)
+    got = H.gpu_compact(ctx, k, v, np.ones(S, np.uint8), 16)
+    assert (got["n_kept"], got["span_pages"], got["rows_moved"]) == (S, 19, 0)
+    assert torch.equal(got["k"], k) and torch.equal(got["v"], v)
+    # partitions and page classes from the compacted unit table
+    units_out = np.array([[0, 20, 2, 0, 0, 0], [20, 30, 0, 1, 1, 0], [50, 14, 1, 1, 1, 0], [64, 25, 0, 9, 2, 0]], np.int32)
+    mask = np.zeros(S, np.uint8)
+    mask[np.arange(89) + np.arange(89) // 3] = 1
+    exp = oc.compact_pack(H.bytes_of(k).reshape(S, -1), H.bytes_of(v).reshape(S, -1), mask, 16, units_out)
+    got = H.gpu_compact(ctx, k, v, mask, 16, units_out_np=units_out)
+    assert got["part_begin"] == exp["part_begin"].tolist() == [0, 20, 64, 89]
+    assert np.array_equal(got["page_class"], exp["page_class"])
+    # idempotence: compacting the packed cache moves nothing
+    mask2 = np.zeros(S, np.uint8)
+    mask2[:89] = 1
+    got2 = H.gpu_compact(ctx, got["k"], got["v"], mask2, 16)
+    assert got2["rows_moved"] == 0 and torch.equal(got2["k"][:89], got["k"][:89])
+    # determinism: same inputs twice give identical bytes
+    got3 = H.gpu_compact(ctx, k, v, mask, 16, units_out_np=units_out)
+    assert torch.equal(got3["k"][:89], got["k"][:89]) and np.array_equal(got3["slot_map"], got["slot_map"])
+    # host-side argument errors
+    with pytest.raises(ob.OmniTideError):
+        ctx.compact(k, v, k, v, None, None, S, 16, None, None, 1, None, None, None)
+    with pytest.raises(ob.OmniTideError):
+        ctx.compact(k, v, torch.empty_like(k), torch.empty_like(v), torch.zeros(4096, dtype=torch.uint8, device="cuda"),
+                    None, 4000, 16, None, None, 1, None, None, None)      # above s_cap
+    ctx.close()
+
+
+# ------------------------------------------------------------------------------------- selection
+def _random_table(rng, U):
+    lens = rng.integers(1, 400, size=U)
+    mods = rng.integers(0, 3, size=U)
+    events = np.cumsum(rng.integers(0, 2, size=U))
+    spans = list(zip(lens.tolist(), mods.tolist(), events.tolist()))
+    units = wl.make_units(spans, group_of_first=0 if rng.random() < 0.7 else None)
+    return units
+
+
+def test_select_exact_given_scores(H, ob):
+    rng = np.random.default_rng(77)
+    ctx = ob.Context(4, 2, 64, "bf16", 1 << 20, 2048, 16)
+    for trial in range(60):
+        U = int(rng.choice([1, 2, 3, 7, 31, 32, 33, 100, 257, 1500]))
+        units = _random_table(rng, U)
+        scores = rng.random(U).astype(np.float32)
+        if trial % 3 == 0:
+            scores = np.round(scores * 4) / 4                   # many exact ties
+        if trial % 5 == 0:
+            scores[rng.integers(U)] = np.nan
+            scores[rng.integers(U)] = -0.0
+        n = int(units[:, 1].sum())
+        budget = int(rng.integers(1, n + 50))
+        R = int(rng.integers(0, 4))
+        caps = tuple(int(c) for c in rng.choice([-1, 200, 1000, 5000], size=3))
+        exp = oc.select_units(units, scores, budget, R, caps)
+        got = H.gpu_select(ctx, units, scores, budget, R, caps)
+        assert got["status"] == 0
+        assert np.array_equal(got["unit_keep"], exp["unit_keep"]), (trial, U)
+        assert got["n_kept"] == exp["n_kept"] and got["n_units_out"] == len(exp["units_out"])
+        assert np.array_equal(got["keep_mask"], exp["keep_mask"])
+        assert np.array_equal(got["units_out"], exp["units_out"])
+    # malformed tables are reported, not trusted
+    bad = wl.make_units([(5, 0, 3), (5, 0, 2)], group_of_first=None)
+    got = H.gpu_select(ctx, bad, np.zeros(2, np.float32), 5, 1, (-1, -1, -1))
+    assert got["status"] & ob.DEV_BAD_UNITS
+    ctx.close()
+
+
+# -------------------------------------------------------------------------------------- attention
+def _check_attention(o, lse, o_ref, lse_ref):
+    err = np.abs(o - o_ref)
+    assert np.isfinite(o).all()
+    assert err.max() <= ATT_MAX_ABS, err.max()
+    assert err.mean() <= ATT_MEAN_ABS, err.mean()
+    if lse is not None:
+        assert np.abs(lse - lse_ref).max() <= 2e-3
+
+
+def test_attention_tiny_fp32(H, ob):
+    w = wl.tiny()
+    ctx = H.make_ctx(w)
+    kh, vh = ob.to_device(w.k_hist, "fp32"), ob.to_device(w.v_hist, "fp32")
+    for n in (1024, 1000, 0):
+        o, lse = H.gpu_attention(ctx, w, kh[:max(n, 1)], vh[:max(n, 1)], n)
+        o_ref, lse_ref = oc.chunk_attention(w.q, w.k_hist[:n], w.v_hist[:n], w.k_chunk, w.v_chunk)
+        _check_attention(o, lse, o_ref, lse_ref)
+    ctx.close()
+
+
+@pytest.mark.parametrize("seed,d,t,n_hist", [(1, 64, 200, None), (2, 32, 77, None), (3, 256, 40, None)])
+def test_attention_cuda_core_bf16(H, ob, seed, d, t, n_hist):
+    w = wl.small_mixed(seed, d=d, t=t)
+    ctx = H.make_ctx(w)
+    kh, vh = ob.to_device(w.k_hist, "bf16"), ob.to_device(w.v_hist, "bf16")
+    o, lse = H.gpu_attention(ctx, w, kh, vh, w.n_hist)
+    o_ref, lse_ref = oc.chunk_attention(w.q, w.k_hist, w.v_hist, w.k_chunk, w.v_chunk)
+    _check_attention(o, lse, o_ref, lse_ref)
+    ctx.close()
+
+
+@pytest.mark.parametrize("t,n_hist,h_q,h_kv", [
+    (128, 128, 4, 2),       # one full tile, one full history block
+    (50, 77, 4, 1),         # ragged everything, single pair with one active tile
+    (300, 1000, 8, 2),      # 3 tiles (second pair half empty), ragged history tail
+    (256, 0, 4, 4),         # no history: plain causal self-attention
+    (690, 4080, 8, 2),      # config-2 chunk and kept-history sizes
+    (1, 1, 4, 2),
+])
+def test_attention_tensor_core(H, ob, t, n_hist, h_q, h_kv):
+    rng = np.random.default_rng(t * 7 + n_hist)
+    units = wl.make_units([(max(n_hist, 1), 0, 0)], group_of_first=None)
+    chunk_units = wl.make_units([(t, 0, 1)], group_of_first=None)
+    q, kh, vh, kc, vc = wl.random_layer_inputs(rng, units, chunk_units, h_q, h_kv, 128, "bf16")
+    kh, vh = kh[:n_hist], vh[:n_hist]
+    w = wl.Workload("tc", h_q, h_kv, 128, "bf16", units, chunk_units, 1, 64, 1, q=q, k_hist=kh, v_hist=vh,
+                    k_chunk=kc, v_chunk=vc)
+    ctx = ob.Context(h_q, h_kv, 128, "bf16", n_hist + 300, 8, t)
+    # device buffers longer than the history, tail poisoned with NaN: must not leak into the output
+    pad = 200
+    khd = torch.full((n_hist + pad, h_kv, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    vhd = torch.full((n_hist + pad, h_kv, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    if n_hist:
+        khd[:n_hist] = ob.to_device(kh, "bf16")
+        vhd[:n_hist] = ob.to_device(vh, "bf16")
+    o_ref, lse_ref = oc.chunk_attention(q, kh, vh, kc, vc)
+    o, lse = H.gpu_attention(ctx, w, khd, vhd, n_hist, n_hist_max=n_hist + pad)
+    _check_attention(o, lse, o_ref, lse_ref)
+    # bf16 output is the fp32 result rounded to nearest even
+    o16, _ = H.gpu_attention(ctx, w, khd, vhd, n_hist, out_fp32=False, n_hist_max=n_hist + pad)
+    assert np.array_equal(o16, wl.round_to_bf16(o))
+    # the CUDA-core kernels agree as a second implementation
+    ctx.set_option(ob.OPT_FORCE_CUDA_CORES, 1)
+    o2, lse2 = H.gpu_attention(ctx, w, khd, vhd, n_hist, n_hist_max=n_hist + pad)
+    _check_attention(o2, lse2, o_ref, lse_ref)
+    ctx.close()
+
+
+# ---------------------------------------------------------------------------------------- scoring
+def _check_scores(score, mass, score_ref, mass_ref):
+    assert np.isfinite(score).all()
+    assert np.abs(mass - mass_ref).max() <= SCORE_REL * max(mass_ref.max(), 1e-30)
+    rel = np.abs(score - score_ref) / np.maximum(np.abs(score_ref), 1e-3 * np.abs(score_ref).max())
+    assert rel.max() <= SCORE_REL, rel.max()
+    assert abs(mass.sum() - 1.0) < 1e-4
+
+
+def test_score_tiny_and_small(H, ob):
+    w = wl.tiny()
+    ctx = H.make_ctx(w)
+    s, m = H.gpu_score(ctx, w)
+    s_ref, m_ref = oc.score_units(w.q, w.k_hist, w.units, w.w_modality)
+    _check_scores(s, m, s_ref, m_ref)
+    ctx.close()
+    for seed, d in [(4, 64), (5, 128), (6, 128)]:
+        w = wl.small_mixed(seed, d=d, n_units=11, max_len=500, t=333)
+        ctx = H.make_ctx(w)
+        s, m = H.gpu_score(ctx, w, use_dev_counts=(seed % 2 == 0))
+        s_ref, m_ref = oc.score_units(w.q, w.k_hist, w.units, w.w_modality)
+        _check_scores(s, m, s_ref, m_ref)
+        ctx.close()
+
+
+def test_score_closed_form_identical_keys(H, ob):
+    """All history keys equal: every unit's score is exactly its modality weight."""
+    w = wl.small_mixed(9, d=128, n_units=7, max_len=300, t=130)
+    w.k_hist[:] = w.k_hist[0:1]
+    ctx = H.make_ctx(w)
+    wm = (1.0, 2.5, 0.75)
+    s, m = H.gpu_score(ctx, w, w_mod=wm)
+    exp = np.array([wm[mod] for mod in w.units[:, 2]])
+    assert np.abs(s - exp).max() < 1e-3
+    ctx.close()
+
+
+def test_score_config2(H, ob, cfg2):
+    w = cfg2
+    ctx = H.make_ctx(w)
+    s, m = H.gpu_score(ctx, w)
+    s_ref, m_ref = oc.score_units(w.q, w.k_hist, w.units, w.w_modality)
+    _check_scores(s, m, s_ref, m_ref)
+    ctx.close()
+
+
+# ------------------------------------------------------------------------------ the whole pass
+def _selection_matches(units, gpu_keep, gpu_scores, ref_scores, budget, R, caps):
+    """The selected set equals the oracle's, except where the oracle's score gap at a decision is
+    below TIE_REL: (i) the oracle's integer rule applied to the GPU's scores reproduces the GPU set
+    exactly, and (ii) the two rankings differ only by swaps of units whose oracle scores are
+    within TIE_REL of each other."""
+    again = oc.select_units(units, gpu_scores, budget, R, caps)
+    assert np.array_equal(again["unit_keep"], gpu_keep)
+    ref = oc.select_units(units, ref_scores.astype(np.float32), budget, R, caps)
+    if np.array_equal(ref["unit_keep"], gpu_keep):
+        return
+    pos_ref = {u: i for i, u in enumerate(ref["order"])}
+    for a, b in zip(again["order"], again["order"][1:]):
+        if pos_ref[a] > pos_ref[b]:
+            gap = abs(ref_scores[a] - ref_scores[b]) / max(abs(ref_scores[a]), abs(ref_scores[b]), 1e-30)
+            assert gap < TIE_REL, (a, b, gap)
+
+
+def _run_step(H, ob, w, host=False):
+    N, T, U = w.n_hist, w.t, len(w.units)
+    s_cap = N + T + 64
+    u_cap = U + len(w.chunk_units) + 4
+    ctx = ob.Context(w.h_q, w.h_kv, w.d, w.dtype, s_cap, u_cap, T)
+    tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    kc_in = torch.zeros((s_cap, w.h_kv, w.d), dtype=tdt, device="cuda")
+    vc_in = torch.zeros_like(kc_in)
+    kc_in[:N] = ob.to_device(w.k_hist, w.dtype)
+    vc_in[:N] = ob.to_device(w.v_hist, w.dtype)
+    kc_out = torch.full_like(kc_in, float("nan"))
+    vc_out = torch.full_like(vc_in, float("nan"))
+    units_in = ob.units_to_device(w.units, u_cap)
+    units_out = torch.zeros((u_cap, 6), dtype=torch.int32, device="cuda")
+    n_hist_out, n_units_out = H.i32(-1), H.i32(-1)
+    info = torch.zeros((8,), dtype=torch.int32, device="cuda")
+    params = ob.select_params(w.budget, w.n_recent_events, w.modality_cap)
+    if host:
+        conv = (lambda a: torch.from_numpy(a).to(tdt).contiguous().pin_memory())
+        q, kc, vc = conv(w.q), conv(w.k_chunk), conv(w.v_chunk)
+        cu = np.ascontiguousarray(w.chunk_units, dtype=np.int32)
+        o = torch.empty((T, w.h_q, w.d), dtype=torch.float32).pin_memory()
+        ctx.chunk_step_host(q, kc, vc, T, cu, len(cu), kc_in, vc_in, H.i32(N), N, units_in, H.i32(U), U, w.w_modality,
+                            params, w.page_size, 0.0, kc_out, vc_out, units_out, n_hist_out, n_units_out, o,
+                            ob.DTYPE_FP32, info_out=info)
+    else:
+        q, kc, vc = (ob.to_device(a, w.dtype) for a in (w.q, w.k_chunk, w.v_chunk))
+        cu = ob.units_to_device(w.chunk_units)
+        o = torch.full((T, w.h_q, w.d), float("nan"), dtype=torch.float32, device="cuda")
+        ctx.chunk_step(q, kc, vc, T, cu, len(w.chunk_units), kc_in, vc_in, H.i32(N), N, units_in, H.i32(U), U,
+                       w.w_modality, params, w.page_size, 0.0, kc_out, vc_out, units_out, n_hist_out, n_units_out, o,
+                       ob.DTYPE_FP32, info_out=info)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    res = dict(o=o.cpu().numpy(), info=ob.info_to_dict(info), n_hist=int(n_hist_out.item()),
+               n_units=int(n_units_out.item()), k=kc_out, v=vc_out, units=units_out.cpu().numpy(),
+               scores=None, launches=ctx.launch_count())
+    # the work buffers are not part of the ABI; re-run the scoring call to look at the scores
+    res["scores"], _ = H.gpu_score(ctx, w)
+    ctx.close()
+    return res
+
+
+def _check_step(H, ob, w, res):
+    s_ref, _ = oc.score_units(w.q, w.k_hist, w.units, w.w_modality)
+    n_new = res["n_hist"] - w.t
+    nu = res["n_units"] - len(w.chunk_units)
+    kept_units = res["units"][:nu]
+    again = oc.select_units(w.units, res["scores"], w.budget, w.n_recent_events, w.modality_cap)
+    assert np.array_equal(again["units_out"], kept_units)
+    gpu_keep = again["unit_keep"]
+    _selection_matches(w.units, gpu_keep, res["scores"], s_ref, w.budget, w.n_recent_events, w.modality_cap)
+    # compaction: bit-exact given the GPU's keep mask
+    es = 2 if w.dtype == "bf16" else 4
+    raw_k = H.bytes_of(ob.to_device(w.k_hist, w.dtype)).reshape(w.n_hist, -1)
+    raw_v = H.bytes_of(ob.to_device(w.v_hist, w.dtype)).reshape(w.n_hist, -1)
+    cp = oc.compact_pack(raw_k, raw_v, again["keep_mask"], w.page_size, again["units_out"])
+    assert res["info"]["n_kept"] == cp["n_kept"] == n_new
+    assert res["info"]["span_pages"] == cp["span_pages"] and res["info"]["rows_moved"] == cp["rows_moved"]
+    assert res["info"]["part_begin"] == cp["part_begin"].tolist()
+    assert res["info"]["span_pages"] * w.page_size - n_new < w.page_size
+    assert np.array_equal(H.bytes_of(res["k"][:n_new]).reshape(n_new, -1), cp["k"])
+    assert np.array_equal(H.bytes_of(res["v"][:n_new]).reshape(n_new, -1), cp["v"])
+    # appended chunk rows and units
+    kc_bytes = H.bytes_of(res["k"][n_new:n_new + w.t]).reshape(w.t, -1)
+    assert np.array_equal(kc_bytes.view(np.uint16 if es == 2 else np.uint32).reshape(w.t, w.h_kv, w.d),
+                          (wl.bf16_bits(w.k_chunk) if es == 2 else w.k_chunk.view(np.uint32)))
+    assert np.array_equal(res["units"][:res["n_units"]], oc.append_chunk(again["units_out"], n_new, w.chunk_units))
+    # attention over the GPU's retained set
+    keep_rows = again["keep_mask"].astype(bool)
+    o_ref, _ = oc.chunk_attention(w.q, w.k_hist[keep_rows], w.v_hist[keep_rows], w.k_chunk, w.v_chunk)
+    _check_attention(res["o"], None, o_ref, None)
+
+
+def test_chunk_step_tiny(H, ob):
+    w = wl.tiny()
+    res = _run_step(H, ob, w)
+    _check_step(H, ob, w, res)
+    assert res["launches"] >= 5
+
+
+def test_chunk_step_small_mixed_and_host_entry(H, ob):
+    for seed, d in [(11, 64), (12, 128)]:
+        w = wl.small_mixed(seed, d=d, n_units=12, max_len=400, t=300)
+        _check_step(H, ob, w, _run_step(H, ob, w))
+        _check_step(H, ob, w, _run_step(H, ob, w, host=True))
+
+
+def test_chunk_step_config2(H, ob, cfg2):
+    res = _run_step(H, ob, cfg2)
+    _check_step(H, ob, cfg2, res)
+    assert res["info"]["n_kept"] <= cfg2.budget
+
+
+def test_budget_covers_history_is_full_attention(H, ob):
+    """No eviction when the budget covers the cache: output equals dense causal attention."""
+    w = wl.small_mixed(21, d=128, n_units=8, max_len=300, t=260)
+    w.budget = w.n_hist
+    res = _run_step(H, ob, w)
+    assert res["info"]["rows_moved"] == 0 and res["info"]["n_kept"] == w.n_hist
+    o_ref, _ = oc.chunk_attention(w.q, w.k_hist, w.v_hist, w.k_chunk, w.v_chunk)
+    _check_attention(res["o"], None, o_ref, None)
