@@ -124,7 +124,7 @@ def select_units(units, scores, budget, n_recent_events=1, modality_cap=(-1, -1,
     if U > 1 and np.any(np.diff(events) < 0):
         raise ValueError("event ids must be non-decreasing in unit order")
     distinct = sorted(set(int(e) for e in events))
-    recent = set(distinct[len(distinct) - n_recent_events:]) if n_recent_events > 0 else set()
+    recent = set(distinct[max(0, len(distinct) - n_recent_events):]) if n_recent_events > 0 else set()
 
     protected = [u for u in range(U)
                  if units[u, U_GROUP] == GRP_MUST_KEEP or int(events[u]) in recent]

@@ -330,7 +330,7 @@ def test_select_invariants_random():
         if rng.random() < 0.3:
             scores[rng.integers(U)] = scores[rng.integers(U)]        # exact ties
         budget = int(rng.integers(1, sum(lens) + 20))
-        R = int(rng.integers(0, 3))
+        R = int(rng.integers(0, 5))
         caps = tuple(int(c) for c in rng.choice([-1, 10, 40, 100], size=3))
         res = oc.select_units(units, scores, budget, R, caps)
         _check_select_invariants(units, scores, budget, R, caps, res)
@@ -369,6 +369,10 @@ def test_select_special_cases():
     # protected set alone above budget: kept = protected exactly (trimming target, not a bound)
     res = oc.select_units(units, np.ones(7, np.float32), 50, 2)
     assert res["unit_keep"].tolist() == [2, 0, 0, 2, 2, 2, 2] and res["n_kept"] == 256
+    # fewer events than the recent window: every event is recent, nothing is evicted
+    two = _units([26, 178], mods=[2, 0], events=[0, 1], groups=[2, 2])
+    res = oc.select_units(two, np.array([0.8, 0.5], np.float32), 92, 3)
+    assert res["unit_keep"].tolist() == [2, 2] and res["n_kept"] == 204
     # NaN scores go last; ties go to the more recent unit
     sc = np.array([0, np.nan, 1, 1, 1, 0, 0], np.float32)
     res = oc.select_units(units, sc, 16 + 120 + 40, 1)
