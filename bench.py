@@ -1,0 +1,351 @@
+#!/usr/bin/env python
+"""Benchmark of the per-chunk hot path (score -> select -> compact -> attend -> append) on B200.
+
+A "step" is one pass of the whole path for one layer over one synthetic chunk of the long-stream
+workload (80,000-token history, 2,354-token chunk, budget 8,192, 32/8 heads, head dim 128, bf16).
+Prints ONE JSON line.  `--impl reference` times the CPU oracle on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "chunk-prefill attn TFLOP/s + compaction GB/s (% roofline); stream-loop ms/chunk"
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS if k in p}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def make_workload(name):
+    from paper_2609_34653_b200 import workloads as wl
+    if name == "long_stream":
+        return wl.long_stream()
+    if name == "layer_8b":
+        return wl.layer_8b()
+    if name == "tiny":
+        return wl.tiny()
+    raise SystemExit(f"unknown workload {name}")
+
+
+def algorithmic_work(w, n_kept):
+    """FLOPs and bytes of one step, as defined for the roofline (masked work not counted)."""
+    N, T = w.n_hist, w.t
+    es = 2 if w.dtype == "bf16" else 4
+    row = w.h_kv * w.d * es
+    return {
+        "score_flop": 2.0 * w.d * w.h_q * T * N,
+        "attn_flop": 4.0 * w.d * w.h_q * (T * n_kept + T * (T + 1) / 2.0),
+        "compact_bytes": 2.0 * n_kept * 2 * row + N + 4.0 * N,        # rows (R+W, K and V) + mask + slot map
+        "select_bytes": 24.0 * len(w.units) + 5.0 * N,
+        "append_bytes": 2.0 * T * 2 * row,
+    }
+
+
+class ClockSampler:
+    def __init__(self, device_index):
+        self.path = tempfile.mktemp(suffix=".csv")
+        self.proc = None
+        self.idx = device_index
+
+    def start(self):
+        q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), f"--query-gpu={q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 7:
+                    continue
+                try:
+                    sm.append(float(f[0])); mx.append(float(f[1]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out = {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                   "samples": len(sm)}
+        return out
+
+
+def run_reference(args, rank, world):
+    """CPU oracle timed on a bounded sample of the same workload (rank 0 only)."""
+    if rank != 0:
+        return
+    from oracle import omni_oracle as oc
+    import threadpoolctl
+    w = make_workload(args.workload)
+    # sample: the attention step of one KV group (G query heads) over a history of `budget` kept rows
+    G = w.h_q // w.h_kv
+    n_kept = min(w.budget, w.n_hist)
+    q = w.q[:, :G]
+    kh, vh = w.k_hist[:n_kept, :1], w.v_hist[:n_kept, :1]
+    kc, vc = w.k_chunk[:, :1], w.v_chunk[:, :1]
+    flop = 4.0 * w.d * G * (w.t * n_kept + w.t * (w.t + 1) / 2.0)
+    times = []
+    for it in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        oc.chunk_attention(q, kh, vh, kc, vc)
+        dt = time.perf_counter() - t0
+        if it >= args.warmup:
+            times.append(dt)
+    dt = float(np.mean(times))
+    cores = max([p.get("num_threads", 1) for p in threadpoolctl.threadpool_info()] + [1])
+    val = flop / dt / 1e12
+    sample = f"attention of 1 of {w.h_kv} KV groups ({G} query heads), T={w.t}, kept history {n_kept}"
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "sample": sample},
+            "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="long_stream")
+    ap.add_argument("--sets", type=int, default=8, help="distinct cache sets rotated so the working set exceeds L2")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2609_34653_b200 import build as _b
+    _b.build()
+    from paper_2609_34653_b200 import binding as ob
+
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # every rank processes its own independent stream (layer replicas): no data-path collective
+    w = make_workload(args.workload)
+    N, T, U = w.n_hist, w.t, len(w.units)
+    s_cap = ((N + T + 255) // 256) * 256
+    u_cap = U + len(w.chunk_units) + 8
+    tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    ctx = ob.Context(w.h_q, w.h_kv, w.d, w.dtype, s_cap, u_cap, T)
+    R = args.sets
+    g = torch.Generator(device="cuda").manual_seed(1234 + rank)
+    base_k, base_v = ob.to_device(w.k_hist, w.dtype), ob.to_device(w.v_hist, w.dtype)
+    sets = []
+    for r in range(R):
+        k_in = torch.empty((s_cap, w.h_kv, w.d), dtype=tdt, device="cuda")
+        v_in = torch.empty_like(k_in)
+        k_in[:N], v_in[:N] = base_k, base_v
+        if r:   # distinct bytes per set, same distribution: permute rows within units is overkill; flip V sign
+            v_in[:N].neg_()
+        sets.append(dict(k_in=k_in, v_in=v_in, k_out=torch.empty_like(k_in), v_out=torch.empty_like(v_in),
+                         q=ob.to_device(w.q, w.dtype).clone(), kc=ob.to_device(w.k_chunk, w.dtype).clone(),
+                         vc=ob.to_device(w.v_chunk, w.dtype).clone(),
+                         o=torch.empty((T, w.h_q, w.d), dtype=torch.float32, device="cuda")))
+    del base_k, base_v
+    units_in = ob.units_to_device(w.units, u_cap)
+    units_out = torch.zeros((u_cap, 6), dtype=torch.int32, device="cuda")
+    chunk_units = ob.units_to_device(w.chunk_units)
+    cnt = lambda v: torch.tensor([v], dtype=torch.int32, device="cuda")
+    n_hist_dev, n_units_dev = cnt(N), cnt(U)
+    n_kept, n_units_kept, n_hist_out, n_units_out = cnt(0), cnt(0), cnt(0), cnt(0)
+    scores = torch.zeros(u_cap, dtype=torch.float32, device="cuda")
+    unit_keep = torch.zeros(u_cap + 16, dtype=torch.uint8, device="cuda")
+    keep_mask = torch.zeros(s_cap + 16, dtype=torch.uint8, device="cuda")
+    slot_map = torch.zeros(s_cap + 16, dtype=torch.int32, device="cuda")
+    info = torch.zeros(8, dtype=torch.int32, device="cuda")
+    params = ob.select_params(w.budget, w.n_recent_events, w.modality_cap)
+    names = ["score", "select", "compact", "attention", "append"]
+
+    def one_step(s, ev=None):
+        rec = (lambda i: ev[i].record()) if ev is not None else (lambda i: None)
+        rec(0)
+        ctx.score_units(s["q"], T, s["k_in"], n_hist_dev, N, units_in, n_units_dev, U, w.w_modality, 0.0, scores)
+        rec(1)
+        ctx.select_units(units_in, n_units_dev, U, scores, params, unit_keep, keep_mask, N, n_kept, units_out, n_units_kept)
+        rec(2)
+        ctx.compact(s["k_in"], s["v_in"], s["k_out"], s["v_out"], keep_mask, n_hist_dev, N, w.page_size, units_out,
+                    n_units_kept, U, slot_map, info, None)
+        rec(3)
+        ctx.chunk_attention(s["q"], T, s["k_out"], s["v_out"], n_kept, N, s["kc"], s["vc"], 0.0, s["o"], ob.DTYPE_FP32)
+        rec(4)
+        ctx.append(s["k_out"], s["v_out"], n_kept, s["kc"], s["vc"], T, units_out, n_units_kept, chunk_units,
+                   len(w.chunk_units), n_hist_out, n_units_out)
+        rec(5)
+
+    for i in range(args.warmup):
+        one_step(sets[i % R])
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0, "device status word not clean after warm-up"
+    kept = int(n_kept.item())
+    work = algorithmic_work(w, kept)
+
+    launches0 = ctx.launch_count()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    start.record()
+    for i in range(args.steps):
+        one_step(sets[(args.warmup + i) % R], evs[i])
+    end.record()
+    barrier()
+    clocks = sampler.stop()
+    gpu_launches = ctx.launch_count() - launches0
+    total_ms = start.elapsed_time(end)
+    per = {n: float(np.mean([evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(args.steps)]))
+           for j, n in enumerate(names)}
+    assert ctx.poll_status() == 0, "device status word not clean after the timed region"
+
+    # ---- end to end through the host-buffer entry point: chunk H2D and output D2H inside the timed region
+    hq = torch.from_numpy(w.q).to(tdt).contiguous().pin_memory()
+    hk = torch.from_numpy(w.k_chunk).to(tdt).contiguous().pin_memory()
+    hv = torch.from_numpy(w.v_chunk).to(tdt).contiguous().pin_memory()
+    ho = torch.empty((T, w.h_q, w.d), dtype=torch.float32).pin_memory()
+    hcu = np.ascontiguousarray(w.chunk_units, dtype=np.int32)
+    e2e_steps = max(3, min(args.steps, 20))
+
+    def e2e_step(s):
+        ctx.chunk_step_host(hq, hk, hv, T, hcu, len(hcu), s["k_in"], s["v_in"], n_hist_dev, N, units_in, n_units_dev, U,
+                            w.w_modality, params, w.page_size, 0.0, s["k_out"], s["v_out"], units_out, n_hist_out,
+                            n_units_out, ho, ob.DTYPE_FP32)
+        torch.cuda.current_stream().synchronize()       # the caller reads o_host after every step
+
+    for i in range(3):
+        e2e_step(sets[i % R])
+    barrier()
+    t0 = time.perf_counter()
+    e2e_start, e2e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2e_start.record()
+    for i in range(e2e_steps):
+        e2e_step(sets[(3 + i) % R])
+    e2e_end.record()
+    barrier()
+    e2e_ms = e2e_start.elapsed_time(e2e_end) / e2e_steps
+    h2d = hq.numel() * hq.element_size() + 2 * hk.numel() * hk.element_size() + hcu.nbytes
+    d2h = ho.numel() * ho.element_size()
+
+    # ---- max over ranks
+    ms_per_step = total_ms / args.steps
+    vec = torch.tensor([ms_per_step, per["attention"], per["compact"], per["score"], per["select"], per["append"], e2e_ms],
+                       dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(vec, op=dist.ReduceOp.MAX)
+    ms_per_step, att_ms, cp_ms, sc_ms, sel_ms, app_ms, e2e_ms = [float(x) for x in vec.tolist()]
+
+    peaks, peak_kind = load_peaks()
+    tensor_peak = peaks["bf16_tflops_sustained"] if "bf16_tflops_sustained" in peaks else peaks["bf16_tflops"]
+    att_tf = work["attn_flop"] / (att_ms * 1e-3) / 1e12
+    sc_tf = work["score_flop"] / (sc_ms * 1e-3) / 1e12
+    cp_gbs = work["compact_bytes"] / (cp_ms * 1e-3) / 1e9
+    kernels = {
+        "attention": {"bound": "tensor", "achieved": att_tf, "peak": tensor_peak, "unit": "TFLOP/s",
+                      "frac": att_tf / tensor_peak, "frac_of_burst_peak": att_tf / peaks["bf16_tflops"],
+                      "frac_of_nominal": att_tf / NOMINAL["bf16_tflops"], "ms": att_ms, "traffic": None},
+        "score": {"bound": "tensor", "achieved": sc_tf, "peak": tensor_peak, "unit": "TFLOP/s",
+                  "frac": sc_tf / tensor_peak, "ms": sc_ms, "traffic": None},
+        "compact": {"bound": "hbm", "achieved": cp_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": cp_gbs / peaks["hbm_gbs"], "frac_of_nominal": cp_gbs / NOMINAL["hbm_gbs"], "ms": cp_ms,
+                    "traffic": None},
+        "select": {"bound": "latency", "ms": sel_ms, "achieved": work["select_bytes"] / (sel_ms * 1e-3) / 1e9, "unit": "GB/s"},
+        "append": {"bound": "hbm", "ms": app_ms, "achieved": work["append_bytes"] / (app_ms * 1e-3) / 1e9,
+                   "peak": peaks["hbm_gbs"], "unit": "GB/s"},
+    }
+    dominant = max(("attention", "score", "compact"), key=lambda n: kernels[n]["ms"])
+    roofline = {k: kernels[dominant][k] for k in ("bound", "achieved", "peak", "unit", "frac", "traffic")}
+    roofline.update(kernel=dominant, peak_source=f"{peak_kind} ({'sustained' if 'bf16_tflops_sustained' in peaks else 'burst'} bf16 matmul / copy bandwidth)")
+
+    line = {
+        "metric": METRIC, "value": att_tf * world, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": args.workload, "h_q": w.h_q, "h_kv": w.h_kv, "head_dim": w.d, "n_hist": N, "chunk": T,
+                   "budget": w.budget, "kept": kept, "page": w.page_size, "units": U,
+                   "l2_policy": f"{R} distinct cache sets rotated ({R * 4 * s_cap * w.h_kv * w.d * 2 / 1e9:.1f} GB > L2)",
+                   "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
+        "attention_tflops": att_tf * world, "compaction_gbs": cp_gbs * world, "score_tflops": sc_tf * world,
+        "ms_per_chunk": ms_per_step, "span_slots": ((kept + w.page_size - 1) // w.page_size) * w.page_size,
+        "kept_rows": kept,
+        "kernels": kernels, "roofline": roofline, "clocks": clocks, "gpu_launches": int(gpu_launches),
+        "e2e": {"value": work["attn_flop"] * world / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_chunk": e2e_ms,
+                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                "note": "attention FLOPs of the step over the whole host-buffer pass (copies + 5 stages)"},
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import omni_oracle as oc
+        import threadpoolctl
+        G = w.h_q // w.h_kv
+        t0 = time.perf_counter()
+        oc.chunk_attention(w.q[:, :G], w.k_hist[:kept, :1], w.v_hist[:kept, :1], w.k_chunk[:, :1], w.v_chunk[:, :1])
+        dt = time.perf_counter() - t0
+        cores = max([p.get("num_threads", 1) for p in threadpoolctl.threadpool_info()] + [1])
+        line["cpu_baseline"] = {"value": work["attn_flop"] / w.h_kv / dt / 1e12, "unit": "TFLOP/s", "cores": cores,
+                                "kind": "oracle", "seconds": dt,
+                                "sample": f"attention of 1 of {w.h_kv} KV groups ({G} query heads), T={T}, kept history {kept}"}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

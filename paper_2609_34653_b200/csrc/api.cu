@@ -49,7 +49,7 @@ extern "C" omni_status omnitide_create(omnitide_ctx** ctx_out, const omni_geomet
     const size_t q_elems = (size_t)g->t_cap * g->h_q * g->d;
     bool ok = true;
     ok &= alloc(&c->status_dev, 1) == cudaSuccess;
-    ok &= alloc(&c->score_part, row_tiles * g->u_cap * 128) == cudaSuccess;
+    ok &= alloc(&c->score_part, row_tiles * ((size_t)g->u_cap + 64) * 128) == cudaSuccess;   // + split boundaries
     ok &= alloc(&c->score_tile_mass, row_tiles * g->u_cap) == cudaSuccess;
     ok &= alloc(&c->score_mass64, (size_t)g->u_cap) == cudaSuccess;
     ok &= alloc(&c->ws_scores, (size_t)g->u_cap) == cudaSuccess;

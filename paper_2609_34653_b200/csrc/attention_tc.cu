@@ -266,8 +266,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 for (int i = 0; i < 16; ++i) {
                     const float p0 = tc::ex2_approx(fmaf(__uint_as_float(sv[c][2 * i]), p.scale_log2, neg_m));
                     const float p1 = tc::ex2_approx(fmaf(__uint_as_float(sv[c][2 * i + 1]), p.scale_log2, neg_m));
-                    rs += p0 + p1;
                     pk[i] = tc::pack_bf16x2(p0, p1);
+                    // the normaliser sums the ROUNDED weights the tensor core will use, so that the
+                    // weights of a row sum to one exactly and the rounding of a dominant weight cancels
+                    rs += __uint_as_float(pk[i] << 16) + __uint_as_float(pk[i] & 0xffff0000u);
                 }
                 tc::tmem_st16(s_tmem + c * 16, pk);
             }

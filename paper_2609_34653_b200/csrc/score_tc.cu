@@ -1,10 +1,380 @@
 // Unit scoring on tcgen05 tensor cores (bf16, head dim 128).
+//
+// score_u needs, for every query row, the softmax mass that falls on each history unit.  One pass
+// over QK^T is enough: a CTA owns a pair of 128-row query tiles of one head and one contiguous range
+// of 128-key blocks ("split"); for every row a thread keeps a running max m and the sum of
+// exp2(c*(s - m)) over the keys of the CURRENT unit, and when the unit (or the split) ends it
+// writes the pair (m, sum) -- a flash-style partial -- to scratch.  A second kernel merges a row's
+// partials into its normaliser and per-unit masses and reduces them over the 128 rows of a tile; a
+// third sums the tiles in a fixed order.  Everything is deterministic (no floating-point atomics).
+//
+//   warp 9      TMA producer: Q tiles once, then K blocks through a 4-stage shared-memory ring
+//   warp 8      one thread issues tcgen05.mma S_t = Q_t K_j^T into TMEM, two S buffers per tile
+//   warps 0-3   row sums of tile 0 (one thread per row, S read from TMEM in 32-column chunks)
+//   warps 4-7   row sums of tile 1
+// TMEM map (512 columns): S0 buffers [0,128) [128,256), S1 buffers [256,384) [384,512).
 #include "common.cuh"
+#include "tc_ptx.cuh"
+
+namespace {
+
+constexpr int BLK = 128;
+constexpr int HD = 128;
+constexpr int TILE_BYTES = BLK * HD * 2;
+constexpr int HALF_BYTES = TILE_BYTES / 2;
+constexpr int NSTAGE = 4;
+constexpr int SC_THREADS = 320;
+constexpr int MAX_SPLITS = 64;
+constexpr uint32_t IDESC_QK = tc::umma_idesc_bf16(128, 128, false, false);
+
+struct ScoreParams {
+    int t, h_q, h_kv;
+    const int32_t* n_hist_dev; int n_hist_max;
+    const omni_unit* units; const int32_t* n_units_dev; int n_units_max;
+    float scale_log2;
+    float2* part;             // [tile][seg_cap][128]
+    int seg_cap;
+    int n_pairs, n_row_tiles, n_splits;
+    int32_t* status;
+};
+
+struct Barriers {
+    uint64_t q_full;
+    uint64_t k_full[NSTAGE];
+    uint64_t k_empty[NSTAGE];
+    uint64_t s_full[2][2];
+    uint64_t s_empty[2][2];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+constexpr int SMEM_FIXED = 2 * TILE_BYTES + NSTAGE * TILE_BYTES + 1024 + 256;
+
+__device__ __forceinline__ int blocks_per_split(int nkb, int n_splits) { return (nkb + n_splits - 1) / n_splits; }
+
+__global__ void __launch_bounds__(SC_THREADS, 1)
+score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, const ScoreParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - tc::smem_u32(smem_raw));
+    const uint32_t q_smem = smem_base;
+    const uint32_t k_smem = smem_base + 2 * TILE_BYTES;
+    Barriers* bars = reinterpret_cast<Barriers*>(smem_gen + 2 * TILE_BYTES + NSTAGE * TILE_BYTES);
+    int* unit_end = reinterpret_cast<int*>(smem_gen + 2 * TILE_BYTES + NSTAGE * TILE_BYTES + 256);   // [n_units_max]
+    volatile int* abort_flag = &bars->abort_flag;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    const int per_split = p.n_pairs * p.h_q;
+    const int split = blockIdx.x / per_split;
+    const int rem = blockIdx.x % per_split;
+    const int pair = rem / p.h_q;
+    const int head = rem % p.h_q;
+    const int kvh = head / (p.h_q / p.h_kv);
+
+    int n_units = p.n_units_dev ? *p.n_units_dev : p.n_units_max;
+    n_units = max(0, min(n_units, p.n_units_max));
+    int n_hist = 0;
+    if (n_units > 0) n_hist = p.units[n_units - 1].start + p.units[n_units - 1].len;
+    if (n_hist > p.n_hist_max || (p.n_hist_dev && *p.n_hist_dev != n_hist)) {
+        if (threadIdx.x == 0) atomicOr(p.status, OMNI_DEV_BAD_COUNT);
+        return;
+    }
+    const int nkb = (n_hist + BLK - 1) / BLK;
+    const int bps = blocks_per_split(nkb, p.n_splits);
+    const int b0 = split * bps, b1 = min(nkb, b0 + bps);
+    const int nb = b1 - b0;
+    if (nb <= 0) return;
+    bool active[2];
+#pragma unroll
+    for (int tt = 0; tt < 2; ++tt) active[tt] = (2 * pair + tt) * BLK < p.t;
+
+    for (int u = threadIdx.x; u < n_units; u += SC_THREADS) unit_end[u] = p.units[u].start + p.units[u].len;
+    if (threadIdx.x == 0) {
+        tc::mbar_init(tc::smem_u32(&bars->q_full), 1);
+        for (int s = 0; s < NSTAGE; ++s) {
+            tc::mbar_init(tc::smem_u32(&bars->k_full[s]), 1);
+            tc::mbar_init(tc::smem_u32(&bars->k_empty[s]), 1);
+        }
+        for (int tt = 0; tt < 2; ++tt)
+            for (int b = 0; b < 2; ++b) {
+                tc::mbar_init(tc::smem_u32(&bars->s_full[tt][b]), 1);
+                tc::mbar_init(tc::smem_u32(&bars->s_empty[tt][b]), 128);
+            }
+        bars->abort_flag = 0;
+        tc::fence_barrier_init();
+    }
+    if (warp == 8) tc::tmem_alloc<512>(tc::smem_u32(&bars->tmem_base));
+    tc::tcgen05_fence_before();
+    __syncthreads();
+    tc::tcgen05_fence_after();
+    const uint32_t tmem = bars->tmem_base;
+
+    if (warp == 9) {
+        if (lane == 0) {
+            tc::tma_prefetch_desc(&tm_q);
+            tc::tma_prefetch_desc(&tm_k);
+            const int n_active = (int)active[0] + (int)active[1];
+            tc::mbar_expect_tx(tc::smem_u32(&bars->q_full), n_active * TILE_BYTES);
+            for (int tt = 0; tt < 2; ++tt) {
+                if (!active[tt]) continue;
+                const int row0 = (2 * pair + tt) * BLK;
+                tc::tma_load_2d(q_smem + tt * TILE_BYTES, &tm_q, head * HD, row0, tc::smem_u32(&bars->q_full));
+                tc::tma_load_2d(q_smem + tt * TILE_BYTES + HALF_BYTES, &tm_q, head * HD + 64, row0, tc::smem_u32(&bars->q_full));
+            }
+            int issued = 0;
+            for (int j = 0; j < nb; ++j) {
+                const int stage = j % NSTAGE, use = j / NSTAGE;
+                if (!tc::mbar_wait(tc::smem_u32(&bars->k_empty[stage]), (use & 1) ^ 1, abort_flag)) break;
+                const uint32_t full = tc::smem_u32(&bars->k_full[stage]);
+                tc::mbar_expect_tx(full, TILE_BYTES);
+                const uint32_t dst = k_smem + stage * TILE_BYTES;
+                tc::tma_load_2d(dst, &tm_k, kvh * HD, (b0 + j) * BLK, full);
+                tc::tma_load_2d(dst + HALF_BYTES, &tm_k, kvh * HD + 64, (b0 + j) * BLK, full);
+                issued = j + 1;
+            }
+            if (*abort_flag) {
+                for (int j = max(0, issued - NSTAGE); j < issued; ++j) {
+                    const long long t0 = clock64();
+                    while (!tc::mbar_try_wait(tc::smem_u32(&bars->k_full[j % NSTAGE]), (j / NSTAGE) & 1) &&
+                           clock64() - t0 < (1ll << 24)) {}
+                }
+            }
+        }
+    } else if (warp == 8) {
+        if (lane == 0) {
+            bool ok = tc::mbar_wait(tc::smem_u32(&bars->q_full), 0, abort_flag);
+            for (int j = 0; j < nb && ok; ++j) {
+                const int stage = j % NSTAGE, buf = j & 1, use = j >> 1;
+                ok = tc::mbar_wait(tc::smem_u32(&bars->k_full[stage]), (j / NSTAGE) & 1, abort_flag);
+                for (int tt = 0; tt < 2 && ok; ++tt) {
+                    if (!active[tt]) continue;
+                    ok = tc::mbar_wait(tc::smem_u32(&bars->s_empty[tt][buf]), (use & 1) ^ 1, abort_flag);
+                    tc::tcgen05_fence_after();
+                    const uint32_t a0 = q_smem + tt * TILE_BYTES, bb = k_smem + stage * TILE_BYTES;
+#pragma unroll
+                    for (int kk = 0; kk < HD / 16; ++kk) {
+                        const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
+                        tc::umma_ss(tmem + tt * 256 + buf * 128, tc::umma_smem_desc(a0 + off, 16, 1024),
+                                    tc::umma_smem_desc(bb + off, 16, 1024), IDESC_QK, kk > 0);
+                    }
+                    tc::umma_commit(tc::smem_u32(&bars->s_full[tt][buf]));
+                }
+                tc::umma_commit(tc::smem_u32(&bars->k_empty[stage]));
+            }
+        }
+    } else {
+        const int tt = warp >> 2;
+        if (active[tt]) {
+            const int r = (warp & 3) * 32 + lane;
+            const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+            const int tile = head * p.n_row_tiles + 2 * pair + tt;
+            float2* part = p.part + (size_t)tile * p.seg_cap * BLK + r;
+            const float c = p.scale_log2;
+            // unit that holds the first key of this split
+            int key = b0 * BLK;
+            int u = 0;
+            {
+                int lo = 0, hi = n_units - 1;          // smallest u with unit_end[u] > key
+                while (lo < hi) {
+                    const int mid = (lo + hi) >> 1;
+                    if (unit_end[mid] > key) hi = mid; else lo = mid + 1;
+                }
+                u = lo;
+            }
+            int u_end = unit_end[u];
+            float m = -INFINITY, acc = 0.f;
+            bool ok = true;
+            for (int j = 0; j < nb && ok; ++j) {
+                const int buf = j & 1;
+                ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&bars->s_full[tt][buf]), (j >> 1) & 1, abort_flag));
+                tc::tcgen05_fence_after();
+                const uint32_t s_tmem = tmem + tt * 256 + buf * 128 + lane_addr;
+#pragma unroll 1
+                for (int ch = 0; ch < 4; ++ch) {
+                    uint32_t sv[32];
+                    tc::tmem_ld32(s_tmem + ch * 32, sv);
+                    tc::tmem_wait_ld();
+                    const int k0 = key + ch * 32;
+                    const int n_valid = min(32, n_hist - k0);           // <= 0 past the end of the history
+                    if (n_valid <= 0) break;
+                    if (n_valid < 32) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (i >= n_valid) sv[i] = 0xff800000u;
+                    }
+                    float cm = __uint_as_float(sv[0]);
+#pragma unroll
+                    for (int i = 1; i < 32; ++i) cm = fmaxf(cm, __uint_as_float(sv[i]));
+                    const float m_new = fmaxf(m, cm);
+                    acc *= tc::ex2_approx((m - m_new) * c);             // exp2(-inf) = 0 on the first chunk
+                    m = m_new;
+                    const float neg_m = -m * c;
+                    if (k0 + 32 <= u_end) {
+                        // the whole chunk lies inside the current unit
+                        float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                        for (int i = 0; i < 32; i += 2) {
+                            s0 += tc::ex2_approx(fmaf(__uint_as_float(sv[i]), c, neg_m));
+                            s1 += tc::ex2_approx(fmaf(__uint_as_float(sv[i + 1]), c, neg_m));
+                        }
+                        acc += s0 + s1;
+                        if (k0 + 32 == u_end && k0 + 32 < n_hist) {
+                            part[(size_t)(u + split) * BLK] = make_float2(m, acc);
+                            acc = 0.f;
+                            ++u;
+                            u_end = unit_end[u];
+                        }
+                    } else {
+                        // one or more unit boundaries inside the chunk (same columns for every row)
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            if (k0 + i == u_end && k0 + i < n_hist) {
+                                part[(size_t)(u + split) * BLK] = make_float2(m, acc);
+                                acc = 0.f;
+                                ++u;
+                                u_end = unit_end[u];
+                            }
+                            acc += tc::ex2_approx(fmaf(__uint_as_float(sv[i]), c, neg_m));
+                        }
+                    }
+                }
+                tc::tcgen05_fence_before();
+                tc::mbar_arrive(tc::smem_u32(&bars->s_empty[tt][buf]));
+                key += BLK;
+            }
+            // the split (or the history) ends inside unit u
+            if (ok) part[(size_t)(u + split) * BLK] = make_float2(m, acc);
+        }
+    }
+
+    tc::tcgen05_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, OMNI_DEV_TIMEOUT);
+    if (warp == 8) {
+        tc::tcgen05_fence_after();
+        tc::tmem_dealloc<512>(tmem);
+    }
+}
+
+// Merge the partials of each row, reduce over the 128 rows of a tile: tile_mass[tile][u].
+__global__ void __launch_bounds__(128) score_combine_kernel(const ScoreParams p, float* tile_mass) {
+    __shared__ float red[4];
+    const int tile = blockIdx.x;
+    const int row_tile = tile % p.n_row_tiles;
+    const int r = threadIdx.x, lane = r & 31, wid = r >> 5;
+    int n_units = p.n_units_dev ? *p.n_units_dev : p.n_units_max;
+    n_units = max(0, min(n_units, p.n_units_max));
+    if (n_units == 0) return;
+    const int n_hist = p.units[n_units - 1].start + p.units[n_units - 1].len;
+    if (n_hist > p.n_hist_max) return;
+    const int nkb = (n_hist + BLK - 1) / BLK;
+    const int bps = blocks_per_split(nkb, p.n_splits);
+    const bool valid = row_tile * BLK + r < p.t;
+    const float2* part = p.part + (size_t)tile * p.seg_cap * BLK + r;
+    const float c = p.scale_log2;
+    float M = -INFINITY, Z = 0.f;
+    if (valid) {
+        for (int u = 0; u < n_units; ++u) {
+            const omni_unit un = p.units[u];
+            const int s_first = (un.start / BLK) / bps, s_last = ((un.start + un.len - 1) / BLK) / bps;
+            for (int s = s_first; s <= s_last; ++s) {
+                const float2 ml = part[(size_t)(u + s) * BLK];
+                const float m_new = fmaxf(M, ml.x);
+                Z = Z * exp2f((M - m_new) * c) + ml.y * exp2f((ml.x - m_new) * c);
+                M = m_new;
+            }
+        }
+    }
+    const float inv_z = valid ? 1.f / Z : 0.f;
+    for (int u = 0; u < n_units; ++u) {
+        const omni_unit un = p.units[u];
+        float v = 0.f;
+        if (valid) {
+            const int s_first = (un.start / BLK) / bps, s_last = ((un.start + un.len - 1) / BLK) / bps;
+            for (int s = s_first; s <= s_last; ++s) {
+                const float2 ml = part[(size_t)(u + s) * BLK];
+                v += ml.y * exp2f((ml.x - M) * c);
+            }
+            v *= inv_z;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) red[wid] = v;
+        __syncthreads();
+        if (r == 0) tile_mass[(size_t)tile * p.n_units_max + u] = (red[0] + red[1]) + (red[2] + red[3]);
+        __syncthreads();
+    }
+}
+
+// mass_u = sum over tiles (fixed order) / rows;  score_u = w[modality] * mass_u * N / len_u
+__global__ void __launch_bounds__(128) score_finalize_kernel(const float* tile_mass, int n_tiles, const omni_unit* units,
+                                                             const int32_t* n_units_dev, int n_units_max, float w0, float w1,
+                                                             float w2, float inv_rows, float* scores, float* mass) {
+    __shared__ float red[128];
+    int n_units = n_units_dev ? *n_units_dev : n_units_max;
+    n_units = max(0, min(n_units, n_units_max));
+    const int u = blockIdx.x;
+    if (u >= n_units) return;
+    float v = 0.f;
+    for (int t = threadIdx.x; t < n_tiles; t += 128) v += tile_mass[(size_t)t * n_units_max + u];
+    red[threadIdx.x] = v;
+    __syncthreads();
+    for (int s = 64; s > 0; s >>= 1) {
+        if (threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        const int n_hist = units[n_units - 1].start + units[n_units - 1].len;
+        const omni_unit un = units[u];
+        const float mu = red[0] * inv_rows;
+        const int mod = min(max(un.modality, 0), 2);
+        const float w = mod == 0 ? w0 : (mod == 1 ? w1 : w2);
+        scores[u] = w * mu * (float)n_hist / (float)un.len;
+        if (mass) mass[u] = mu;
+    }
+}
+
+}  // namespace
 
 omni_status omni_score_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q, int t, const void* k_cache,
                           const int32_t* n_hist_dev, int n_hist_max, const omni_unit* units,
                           const int32_t* n_units_dev, int n_units_max, const float* w, float scale,
                           float* scores_out, float* mass_out) {
-    return omni_score_simple(ctx, st, q, t, k_cache, n_hist_dev, n_hist_max, units, n_units_dev, n_units_max, w, scale,
-                             scores_out, mass_out);
+    const omni_geometry& g = ctx->g;
+    CUtensorMap tm_q, tm_k;
+    bool ok = omni_make_map_bf16(ctx->encode_tiled, &tm_q, q, t, (uint64_t)g.h_q * HD, BLK);
+    ok &= omni_make_map_bf16(ctx->encode_tiled, &tm_k, k_cache, n_hist_max, (uint64_t)g.h_kv * HD, BLK);
+    if (!ok) OMNI_FAIL(ctx, OMNI_ERR_CUDA, "score: cuTensorMapEncodeTiled failed");
+    ScoreParams p;
+    p.t = t; p.h_q = g.h_q; p.h_kv = g.h_kv; p.n_hist_dev = n_hist_dev; p.n_hist_max = n_hist_max;
+    p.units = units; p.n_units_dev = n_units_dev; p.n_units_max = n_units_max;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.part = ctx->score_part; p.seg_cap = g.u_cap + MAX_SPLITS;
+    p.n_pairs = (t + 2 * BLK - 1) / (2 * BLK);
+    p.n_row_tiles = (t + BLK - 1) / BLK;
+    p.status = ctx->status_dev;
+    // split the key range so that the grid fills whole waves of SMs and a split keeps >= 8 key blocks
+    const int nkb_max = (n_hist_max + BLK - 1) / BLK;
+    const int base_items = p.n_pairs * g.h_q;
+    int best = 1;
+    double best_eff = 0.0;
+    for (int ks = 1; ks <= MAX_SPLITS && (ks == 1 || nkb_max / ks >= 8); ++ks) {
+        const long long items = (long long)base_items * ks;
+        const long long waves = (items + ctx->sm_count - 1) / ctx->sm_count;
+        const double eff = (double)items / (double)(waves * ctx->sm_count);
+        if (eff > best_eff + 1e-3) { best_eff = eff; best = ks; }
+    }
+    p.n_splits = best;
+    const int smem = SMEM_FIXED + n_units_max * (int)sizeof(int);
+    if (smem > 227 * 1024) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "score: too many units for one CTA's shared memory");
+    OMNI_CUDA(ctx, cudaFuncSetAttribute(score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    score_tc_kernel<<<base_items * p.n_splits, SC_THREADS, smem, st>>>(tm_q, tm_k, p);
+    OMNI_CHECK_LAUNCH(ctx, "score_tc_kernel");
+    const int n_tiles = p.n_row_tiles * g.h_q;
+    score_combine_kernel<<<n_tiles, 128, 0, st>>>(p, ctx->score_tile_mass);
+    OMNI_CHECK_LAUNCH(ctx, "score_combine_kernel");
+    score_finalize_kernel<<<n_units_max, 128, 0, st>>>(ctx->score_tile_mass, n_tiles, units, n_units_dev, n_units_max,
+                                                       w[0], w[1], w[2], 1.0f / ((float)t * g.h_q), scores_out, mass_out);
+    OMNI_CHECK_LAUNCH(ctx, "score_finalize_kernel");
+    return OMNI_OK;
 }

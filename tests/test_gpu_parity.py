@@ -150,7 +150,9 @@ def _check_attention(o, lse, o_ref, lse_ref):
     assert err.max() <= ATT_MAX_ABS, err.max()
     assert err.mean() <= ATT_MEAN_ABS, err.mean()
     if lse is not None:
-        assert np.abs(lse - lse_ref).max() <= 2e-3
+        # the tensor-core path normalises with the bf16-rounded weights it multiplies by, so its
+        # log-sum-exp carries their rounding (2^-9 relative on a dominant weight)
+        assert np.abs(lse - lse_ref).max() <= 5e-3
 
 
 def test_attention_tiny_fp32(H, ob):
