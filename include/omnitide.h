@@ -237,6 +237,36 @@ omni_status omnitide_chunk_step_host(omnitide_ctx* ctx, void* stream,
                                      int32_t* n_hist_out, int32_t* n_units_out,
                                      void* o_host, int32_t out_dtype, omni_compact_info* info_out);
 
+/*
+ * Unit scoring for callers that cannot allocate.  (The paper has no counterpart: this is a
+ * packaging variant of omnitide_score_units, same formula, computed by the fp32 CUDA-core kernel.)
+ *
+ * Some hosts of this library may not call cudaMalloc at all: a serving runtime that hands every
+ * byte of HBM to its own KV-cache pool at start-up, so that a later cudaMalloc fails or takes memory
+ * the pool believes it owns; or a latency-critical loop in which cudaMalloc/cudaFree, which
+ * synchronise the whole device, would stall every other stream.  Such callers cannot create an
+ * omnitide_ctx (creation allocates scratch).  This entry point needs no context and allocates
+ * nothing: the per-unit accumulators it needs live in a fixed array of
+ * OMNITIDE_NOALLOC_MAX_UNITS doubles (8 KiB) inside the library's device image, present on every
+ * GPU that loads the library until the process exits.
+ *
+ *   - n_units above OMNITIDE_NOALLOC_MAX_UNITS is refused with OMNI_ERR_CAPACITY (nothing is launched).
+ *   - Counts are host values here (n_hist, n_units); q, k_cache, units, scores_out, mass_out are
+ *     device pointers owned by the caller as in omnitide_score_units; mass_out may be NULL.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *     that device current); make that first call outside any stream capture.
+ *   - Every call on a device shares the one array.  The call clears the accumulators it uses before
+ *     adding into them, so back-to-back calls on one stream are independent; two calls whose kernels
+ *     can overlap on the GPU (different streams, no ordering between them) race on the array and
+ *     must be serialised by the caller.
+ */
+#define OMNITIDE_NOALLOC_MAX_UNITS 1024
+omni_status omnitide_score_units_noalloc(void* stream, int32_t h_q, int32_t h_kv, int32_t d, int32_t dtype,
+                                         const void* q, int32_t t, const void* k_cache, int32_t n_hist,
+                                         const omni_unit* units, int32_t n_units,
+                                         const float* w_modality, float scale,
+                                         float* scores_out, float* mass_out);
+
 /* Options.  OMNI_OPT_FORCE_CUDA_CORES != 0 routes scoring and attention through the fp32 CUDA-core
  * kernels even where the tensor-core kernels apply (a second implementation for cross-checks). */
 enum { OMNI_OPT_FORCE_CUDA_CORES = 1 };

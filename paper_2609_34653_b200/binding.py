@@ -39,8 +39,9 @@ EXPORTS = [
     "omnitide_create", "omnitide_destroy", "omnitide_poll_status", "omnitide_last_error",
     "omnitide_score_units", "omnitide_select_units", "omnipage_compact", "omnipage_append",
     "omnitide_chunk_attention", "omnitide_chunk_step", "omnitide_chunk_step_host",
-    "omnitide_set_option", "omnitide_launch_count",
+    "omnitide_set_option", "omnitide_launch_count", "omnitide_score_units_noalloc",
 ]
+NOALLOC_MAX_UNITS = 1024
 
 
 def load_library(path: str = LIB_PATH) -> C.CDLL:
@@ -63,6 +64,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.omnipage_compact.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, i32, vp, vp, vp]
     lib.omnipage_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, i32, vp, vp]
     lib.omnitide_chunk_attention.argtypes = [vp, vp, vp, i32, vp, vp, vp, i32, vp, vp, f32, vp, i32, vp]
+    lib.omnitide_score_units_noalloc.argtypes = [vp, i32, i32, i32, i32, vp, i32, vp, i32, vp, i32, C.POINTER(f32), f32,
+                                                 vp, vp]
     step = [vp, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp, i32, vp, vp, i32, C.POINTER(f32),
             C.POINTER(SelectParams), i32, f32, vp, vp, vp, vp, vp, vp, i32, vp]
     lib.omnitide_chunk_step.argtypes = step
@@ -201,6 +204,23 @@ class Context:
 
     def chunk_step_host(self, *a, info_out=None):
         self._step(self.lib.omnitide_chunk_step_host, "omnitide_chunk_step_host", _host_ptr, *a, info_out)
+
+
+def score_units_noalloc(h_q, h_kv, d, dtype, q, t, k_cache, n_hist, units, n_units, w_modality, scale, scores_out,
+                        mass_out=None, lib=None):
+    """Context-free scoring for hosts that may not call cudaMalloc: the accumulators live in a fixed
+    array inside the library (at most NOALLOC_MAX_UNITS units).  Calls sharing a device must not
+    overlap on the GPU.  Argument marshalling only."""
+    lib = lib or load_library()
+    w = (C.c_float * 3)(*[float(x) for x in w_modality])
+    st = lib.omnitide_score_units_noalloc(_stream(), h_q, h_kv, d, DTYPE_BF16 if dtype in ("bf16", DTYPE_BF16) else DTYPE_FP32,
+                                          _ptr(q), t, _ptr(k_cache), n_hist, _ptr(units), n_units, w, float(scale),
+                                          _ptr(scores_out), _ptr(mass_out))
+    if st == ERR_CAPACITY:
+        raise OmniTideError(f"omnitide_score_units_noalloc: CAPACITY: {n_units} units exceed the fixed scratch of "
+                            f"{NOALLOC_MAX_UNITS} units")
+    if st != OK:
+        raise OmniTideError(f"omnitide_score_units_noalloc: {_STATUS_NAMES.get(st, st)}")
 
 
 # ---- small helpers for tests and the benchmark (device memory plumbing only) -------------------

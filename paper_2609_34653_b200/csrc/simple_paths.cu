@@ -208,3 +208,83 @@ omni_status omni_score_simple(omnitide_ctx* ctx, cudaStream_t st, const void* q,
     OMNI_CHECK_LAUNCH(ctx, "score_finalize64_kernel");
     return OMNI_OK;
 }
+
+// ------------------------------------------------------------------------------------------------
+// Scoring without any allocation, for callers that have no context and may not call cudaMalloc.
+// The per-unit accumulator that the CUDA-core scoring kernel adds into lives in a fixed array in
+// device global memory that is part of the library image (every device that loads the library
+// carries these few KB until the process exits).
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int NOALLOC_MAX_UNITS = OMNITIDE_NOALLOC_MAX_UNITS;
+constexpr int NOALLOC_MAX_DEVICES = 64;
+
+static __device__ __align__(256) double g_noalloc_mass[NOALLOC_MAX_UNITS];
+static __device__ __align__(256) int32_t g_noalloc_status[64];
+
+// Device addresses of the two arrays, looked up once per device.  The array names above are only
+// host-side handles here: a kernel must be given the address that cudaGetSymbolAddress returns
+// while that device is current.
+struct NoallocDevice {
+    double* mass;
+    int32_t* status;
+    bool ready;
+};
+NoallocDevice g_noalloc_dev[NOALLOC_MAX_DEVICES];
+
+omni_status noalloc_setup(int dev, NoallocDevice** out) {
+    if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return OMNI_ERR_UNSUPPORTED;
+    NoallocDevice& d = g_noalloc_dev[dev];
+    if (!d.ready) {
+        void* p_mass = nullptr;
+        void* p_status = nullptr;
+        if (cudaGetSymbolAddress(&p_mass, g_noalloc_mass) != cudaSuccess) return OMNI_ERR_CUDA;
+        if (cudaGetSymbolAddress(&p_status, g_noalloc_status) != cudaSuccess) return OMNI_ERR_CUDA;
+        d.mass = static_cast<double*>(p_mass);
+        d.status = static_cast<int32_t*>(p_status);
+        d.ready = true;
+    }
+    *out = &d;
+    return OMNI_OK;
+}
+
+}  // namespace
+
+extern "C" omni_status omnitide_score_units_noalloc(void* stream, int32_t h_q, int32_t h_kv, int32_t d, int32_t dtype,
+                                                    const void* q, int32_t t, const void* k_cache, int32_t n_hist,
+                                                    const omni_unit* units, int32_t n_units, const float* w_modality,
+                                                    float scale, float* scores_out, float* mass_out) {
+    if (!q || !k_cache || !units || !w_modality || !scores_out) return OMNI_ERR_INVALID_ARG;
+    if (h_q <= 0 || h_kv <= 0 || h_q % h_kv != 0 || d <= 0 || d % 8 != 0 || d > 256 ||
+        (dtype != OMNI_DTYPE_BF16 && dtype != OMNI_DTYPE_FP32))
+        return OMNI_ERR_UNSUPPORTED;
+    if (t <= 0 || n_hist <= 0 || n_units <= 0) return OMNI_ERR_INVALID_ARG;
+    if (n_units > NOALLOC_MAX_UNITS) return OMNI_ERR_CAPACITY;       // the fixed accumulator array is full
+    if (!omni_aligned16(q) || !omni_aligned16(k_cache)) return OMNI_ERR_INVALID_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return OMNI_ERR_CUDA;
+    NoallocDevice* nd = nullptr;
+    omni_status s = noalloc_setup(dev, &nd);
+    if (s != OMNI_OK) return s;
+    if (scale <= 0.f) scale = 1.0f / sqrtf((float)d);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the array still holds the sums of the previous call: the accumulators must start at zero
+    if (cudaMemsetAsync(nd->mass, 0, sizeof(double) * (size_t)n_units, st) != cudaSuccess) return OMNI_ERR_CUDA;
+    const long long rows = (long long)t * h_q;
+    const int grid = (int)((rows + SP_WARPS - 1) / SP_WARPS);
+    if (dtype == OMNI_DTYPE_FP32)
+        score_rows_kernel<float><<<grid, SP_WARPS * 32, 0, st>>>((const float*)q, t, h_q, h_kv, d, (const float*)k_cache,
+                                                                 nullptr, n_hist, units, nullptr, n_units, scale, nd->mass,
+                                                                 nd->status);
+    else
+        score_rows_kernel<__nv_bfloat16><<<grid, SP_WARPS * 32, 0, st>>>(
+            (const __nv_bfloat16*)q, t, h_q, h_kv, d, (const __nv_bfloat16*)k_cache, nullptr, n_hist, units, nullptr,
+            n_units, scale, nd->mass, nd->status);
+    if (cudaGetLastError() != cudaSuccess) return OMNI_ERR_CUDA;
+    score_finalize64_kernel<<<(n_units + 255) / 256, 256, 0, st>>>(nd->mass, units, nullptr, n_units, w_modality[0],
+                                                                   w_modality[1], w_modality[2], 1.0f / (float)rows,
+                                                                   scores_out, mass_out);
+    if (cudaGetLastError() != cudaSuccess) return OMNI_ERR_CUDA;
+    return OMNI_OK;
+}
