@@ -63,6 +63,9 @@ extern "C" omni_status omnitide_create(omnitide_ctx** ctx_out, const omni_geomet
     ok &= cudaMalloc(&c->st_v, (size_t)g->t_cap * c->row_bytes) == cudaSuccess;
     ok &= cudaMalloc(&c->st_o, q_elems * 4) == cudaSuccess;
     ok &= alloc(&c->st_units, 64) == cudaSuccess;
+    // split-item partials of the attention kernel: [SM][2 slots][2 tiles][128 rows] x (128 floats, (max, sum))
+    ok &= alloc(&c->attn_part_o, (size_t)c->sm_count * 4 * 128 * 128) == cudaSuccess;
+    ok &= alloc(&c->attn_part_ml, (size_t)c->sm_count * 4 * 128 * 2) == cudaSuccess;
     if (ok) ok = cudaMemset(c->status_dev, 0, sizeof(int32_t)) == cudaSuccess;
     if (ok) {
         cudaDriverEntryPointQueryResult qres;
