@@ -1,6 +1,6 @@
 // GQA chunk-prefill attention on tcgen05 tensor cores (bf16, head dim 128).
 //
-// Work unit: one 128-key KV block of one "item" = (pair of 128-row query tiles, head).  The KV sequence
+// Work unit: one 64-key KV block of one "item" = (pair of 128-row query tiles, head).  The KV sequence
 // of an item is the history blocks followed by the causal chunk blocks.  The kernel is persistent, one
 // CTA per SM: the units of all items are laid end to end and cut into equal contiguous shares, so every
 // SM gets the same amount of tensor work whatever the number of items.  A share is a list of "parts"
@@ -9,29 +9,37 @@
 // second kernel merges them.
 //
 // Inside a CTA:
-//   warp 9      TMA producer: the part's Q tiles, then K_j / V_j tiles through a 4-stage shared-memory ring
-//   warp 8      one thread issues tcgen05.mma: S_t = Q_t K_j^T (operands in shared memory) and
-//               O_t += P_t V_j (P read from tensor memory, V as an MN-major shared-memory operand)
+//   warp 10     TMA producer: the part's Q tiles, then K / V tiles (64 keys) through an 8-stage ring
+//   warps 8, 9  MMA issuer of tile 0 / tile 1 (one elected lane, warp-uniform code): S_t = Q_t K_j^T
+//               (operands in shared memory) and O_t += P_t V_j (P read from tensor memory, V as an
+//               MN-major shared-memory operand).  One issuer per tile: issuing is the scarce resource.
 //   warps 0-3   softmax of tile 0, one thread per query row: S from TMEM, running max with lazy
 //   warps 4-7   rescale of O, exp2, P written back to TMEM as bf16 over the S columns; same for tile 1
-// The two tiles alternate on the tensor pipe, so one tile's softmax overlaps the other's MMAs.
-// TMEM map (512 columns): S0/P0 [0,128)  S1/P1 [128,256)  O0 [256,384)  O1 [384,512).
+// S is double-buffered per tile, and QK^T runs two blocks ahead of PV, so the softmax of block j never
+// waits for the tensor pipe: S_{j+1} is already in tensor memory when block j is done.
+// TMEM map (512 columns): tile t: S/P buffer 0 [128t, 128t+64)  buffer 1 [128t+64, 128t+128);  O_t [256+128t, +128).
 #include "common.cuh"
 #include "tc_ptx.cuh"
 
+#include <algorithm>
+
 namespace {
 
-constexpr int BLK = 128;                 // rows per query tile and keys per KV block
+constexpr int BQ = 128;                  // rows per query tile
+constexpr int BK = 64;                   // keys per KV block
 constexpr int HD = 128;                  // head dim
-constexpr int TILE_BYTES = BLK * HD * 2; // 32 KiB, stored as two 64-column halves of 16 KiB
-constexpr int HALF_BYTES = TILE_BYTES / 2;
-constexpr int NSTAGE = 4;
-constexpr int ATT_THREADS = 320;
-constexpr int SMEM_BYTES = 2 * TILE_BYTES + NSTAGE * TILE_BYTES + 1024 /*alignment*/ + 256 /*barriers*/;
-constexpr float RESCALE_THRESHOLD = 8.0f;   // log2 units: P stays below 2^8
+constexpr int Q_TILE_BYTES = BQ * HD * 2;    // 32 KiB, two 64-column halves of 16 KiB
+constexpr int Q_HALF_BYTES = Q_TILE_BYTES / 2;
+constexpr int KV_TILE_BYTES = BK * HD * 2;   // 16 KiB, two 64-column halves of 8 KiB
+constexpr int KV_HALF_BYTES = KV_TILE_BYTES / 2;
+constexpr int NSTAGE = 8;
+constexpr int ATT_THREADS = 352;
+constexpr int SMEM_BYTES = 2 * Q_TILE_BYTES + NSTAGE * KV_TILE_BYTES + 1024 /*alignment*/ + 512 /*barriers*/;
+// O is rescaled only when the row max grows by more than this many log2 units (P stays below 2^8).
+constexpr float RESCALE_THRESHOLD = 8.0f;
 
-constexpr uint32_t IDESC_QK = tc::umma_idesc_bf16(128, 128, false, false);
-constexpr uint32_t IDESC_PV = tc::umma_idesc_bf16(128, 128, false, true);
+constexpr uint32_t IDESC_QK = tc::umma_idesc_bf16(128, BK, false, false);
+constexpr uint32_t IDESC_PV = tc::umma_idesc_bf16(128, HD, false, true);
 
 struct AttnParams {
     int t, h_q, h_kv;
@@ -48,8 +56,9 @@ struct Barriers {
     uint64_t q_full;
     uint64_t kv_full[NSTAGE];
     uint64_t kv_empty[NSTAGE];
-    uint64_t s_full[2];
-    uint64_t p_full[2];
+    uint64_t s_full[2][2];      // [tile][buffer]
+    uint64_t p_full[2][2];
+    uint64_t pv_done[2];        // one phase per PV of the tile
     uint64_t o_done;
     uint64_t o_free[2];
     uint32_t tmem_base;
@@ -58,10 +67,12 @@ struct Barriers {
 
 // ---- the work list: identical arithmetic in every role and in the merge kernel --------------------------
 struct Sched {
-    int nhb, n_pairs, h_q, t;
-    __device__ int nb_pair(int pair) const {                 // KV blocks of an item = blocks of its last active tile
-        return nhb + 2 * pair + (((2 * pair + 1) * BLK < t) ? 2 : 1);
+    int nhb, n_pairs, h_q, t;                                // nhb: 64-key blocks of history
+    __device__ int nb_tile(int pair, int tt) const {         // KV blocks tile tt of a pair attends to
+        const int row0 = (2 * pair + tt) * BQ;
+        return row0 < t ? nhb + row0 / BK + 2 : 0;           // chunk blocks 0 .. row0/64 + 1 reach the diagonal
     }
+    __device__ int nb_pair(int pair) const { return max(nb_tile(pair, 0), nb_tile(pair, 1)); }
     __device__ long long total() const {
         long long w = 0;
         for (int pr = 0; pr < n_pairs; ++pr) w += (long long)h_q * nb_pair(pr);
@@ -107,15 +118,16 @@ struct PartIter {
         const long long room = w_end - w;
         p.j1 = (int)min((long long)p.nb_item, (long long)p.j0 + room);
         w += p.j1 - p.j0;
-        const int nb_t0 = (2 * p.pair) * BLK < s.t ? s.nhb + 2 * p.pair + 1 : 0;
-        const int nb_t1 = (2 * p.pair + 1) * BLK < s.t ? s.nhb + 2 * p.pair + 2 : 0;
-        p.cnt0 = max(0, min(p.j1, nb_t0) - p.j0);
-        p.cnt1 = max(0, min(p.j1, nb_t1) - p.j0);
+        p.cnt0 = max(0, min(p.j1, s.nb_tile(p.pair, 0)) - p.j0);
+        p.cnt1 = max(0, min(p.j1, s.nb_tile(p.pair, 1)) - p.j0);
         p.final_ = p.j0 == 0 && p.j1 == p.nb_item;
         p.slot = p.j0 > 0 ? 0 : 1;
         return true;
     }
 };
+
+// Position, in the part's load order  K0 K1 V0 K2 V1 K3 ... V_{n-2} V_{n-1},  of the V tile of local block jj.
+__device__ __forceinline__ int pos_v(int jj, int n) { return n == 1 ? 1 : (jj == n - 1 ? 2 * n - 1 : 2 + 2 * jj); }
 
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kh,
@@ -124,20 +136,21 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - tc::smem_u32(smem_raw));
-    const uint32_t q_smem = smem_base;                       // 2 tiles
-    const uint32_t kv_smem = smem_base + 2 * TILE_BYTES;     // NSTAGE tiles
-    Barriers* bars = reinterpret_cast<Barriers*>(smem_gen + 2 * TILE_BYTES + NSTAGE * TILE_BYTES);
+    const uint32_t q_smem = smem_base;                          // 2 Q tiles
+    const uint32_t kv_smem = smem_base + 2 * Q_TILE_BYTES;      // NSTAGE K/V tiles
+    Barriers* bars = reinterpret_cast<Barriers*>(smem_gen + 2 * Q_TILE_BYTES + NSTAGE * KV_TILE_BYTES);
     volatile int* abort_flag = &bars->abort_flag;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0);      // provably warp-uniform
+    const int lane = threadIdx.x & 31;
 
     int n_hist = p.n_hist_dev ? *p.n_hist_dev : p.n_hist_max;
     if (n_hist < 0 || n_hist > p.n_hist_max) {
         if (threadIdx.x == 0 && blockIdx.x == 0) atomicOr(p.status, OMNI_DEV_BAD_COUNT);
         n_hist = max(0, min(n_hist, p.n_hist_max));
     }
-    const int nhb = (n_hist + BLK - 1) / BLK;
-    const int hist_tail = n_hist - (nhb - 1) * BLK;          // valid keys in the last history block (if nhb > 0)
-    const bool tail_partial = nhb > 0 && hist_tail < BLK;
+    const int nhb = (n_hist + BK - 1) / BK;
+    const int hist_tail = n_hist - (nhb - 1) * BK;           // valid keys in the last history block (if nhb > 0)
+    const bool tail_partial = nhb > 0 && hist_tail < BK;
 
     PartIter it;
     it.s.nhb = nhb; it.s.n_pairs = p.n_pairs; it.s.h_q = p.h_q; it.s.t = p.t;
@@ -152,14 +165,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         tc::mbar_init(tc::smem_u32(&bars->q_full), 1);
         for (int s = 0; s < NSTAGE; ++s) {
             tc::mbar_init(tc::smem_u32(&bars->kv_full[s]), 1);
-            tc::mbar_init(tc::smem_u32(&bars->kv_empty[s]), 1);
+            tc::mbar_init(tc::smem_u32(&bars->kv_empty[s]), 2);          // released by both MMA warps
         }
         for (int tt = 0; tt < 2; ++tt) {
-            tc::mbar_init(tc::smem_u32(&bars->s_full[tt]), 1);
-            tc::mbar_init(tc::smem_u32(&bars->p_full[tt]), 128);
+            for (int b = 0; b < 2; ++b) {
+                tc::mbar_init(tc::smem_u32(&bars->s_full[tt][b]), 1);
+                tc::mbar_init(tc::smem_u32(&bars->p_full[tt][b]), 128);
+            }
+            tc::mbar_init(tc::smem_u32(&bars->pv_done[tt]), 1);
             tc::mbar_init(tc::smem_u32(&bars->o_free[tt]), 128);
         }
-        tc::mbar_init(tc::smem_u32(&bars->o_done), 1);
+        tc::mbar_init(tc::smem_u32(&bars->o_done), 2);                   // both MMA warps
         bars->abort_flag = 0;
         tc::fence_barrier_init();
     }
@@ -167,13 +183,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     tc::tcgen05_fence_before();
     __syncthreads();
     tc::tcgen05_fence_after();
-    const uint32_t tmem = bars->tmem_base;
+    const uint32_t tmem = __shfl_sync(0xffffffffu, bars->tmem_base, 0);
 
     Part part;
     int part_idx = 0;
     int kv_base = 0;                                         // K/V tiles loaded by earlier parts of this CTA
 
-    if (warp == 9) {
+    if (warp == 10) {
         // ================================ TMA producer ================================
         if (lane == 0) {
             tc::tma_prefetch_desc(&tm_q);
@@ -183,38 +199,43 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             tc::tma_prefetch_desc(&tm_vc);
             int issued = 0;
             bool ok = true;
+            int kvh = 0;
+            auto load_tile = [&](int j, bool is_v) {         // block j of the item, next ring slot
+                const int idx = issued;
+                const int stage = idx % NSTAGE, use = idx / NSTAGE;
+                ok = tc::mbar_wait(tc::smem_u32(&bars->kv_empty[stage]), (use & 1) ^ 1, abort_flag);
+                if (!ok) return;
+                const uint32_t full = tc::smem_u32(&bars->kv_full[stage]);
+                tc::mbar_expect_tx(full, KV_TILE_BYTES);
+                const bool hist = j < nhb;
+                const CUtensorMap* map = hist ? (is_v ? &tm_vh : &tm_kh) : (is_v ? &tm_vc : &tm_kc);
+                const int row = (hist ? j : j - nhb) * BK;
+                const uint32_t dst = kv_smem + stage * KV_TILE_BYTES;
+                tc::tma_load_2d(dst, map, kvh * HD, row, full);
+                tc::tma_load_2d(dst + KV_HALF_BYTES, map, kvh * HD + 64, row, full);
+                issued = idx + 1;
+            };
             while (ok && it.next(part)) {
                 // the Q tiles are free once every MMA of the previous part has completed
                 if (part_idx > 0) ok = tc::mbar_wait(tc::smem_u32(&bars->o_done), (part_idx - 1) & 1, abort_flag);
                 if (!ok) break;
-                const int kvh = part.head / (p.h_q / p.h_kv);
+                kvh = part.head / (p.h_q / p.h_kv);
                 const int n_active = (part.cnt0 > 0) + (part.cnt1 > 0);
-                tc::mbar_expect_tx(tc::smem_u32(&bars->q_full), n_active * TILE_BYTES);
+                tc::mbar_expect_tx(tc::smem_u32(&bars->q_full), n_active * Q_TILE_BYTES);
                 for (int tt = 0; tt < 2; ++tt) {
                     if ((tt ? part.cnt1 : part.cnt0) == 0) continue;
-                    const int row0 = (2 * part.pair + tt) * BLK;
-                    tc::tma_load_2d(q_smem + tt * TILE_BYTES, &tm_q, part.head * HD, row0, tc::smem_u32(&bars->q_full));
-                    tc::tma_load_2d(q_smem + tt * TILE_BYTES + HALF_BYTES, &tm_q, part.head * HD + 64, row0,
+                    const int row0 = (2 * part.pair + tt) * BQ;
+                    tc::tma_load_2d(q_smem + tt * Q_TILE_BYTES, &tm_q, part.head * HD, row0, tc::smem_u32(&bars->q_full));
+                    tc::tma_load_2d(q_smem + tt * Q_TILE_BYTES + Q_HALF_BYTES, &tm_q, part.head * HD + 64, row0,
                                     tc::smem_u32(&bars->q_full));
                 }
-                const int n_loads = 2 * (part.j1 - part.j0);
-                for (int i = 0; i < n_loads && ok; ++i) {
-                    const int idx = kv_base + i;
-                    const int j = part.j0 + (i >> 1), is_v = i & 1;
-                    const int stage = idx % NSTAGE, use = idx / NSTAGE;
-                    ok = tc::mbar_wait(tc::smem_u32(&bars->kv_empty[stage]), (use & 1) ^ 1, abort_flag);
-                    if (!ok) break;
-                    const uint32_t full = tc::smem_u32(&bars->kv_full[stage]);
-                    tc::mbar_expect_tx(full, TILE_BYTES);
-                    const bool hist = j < nhb;
-                    const CUtensorMap* map = hist ? (is_v ? &tm_vh : &tm_kh) : (is_v ? &tm_vc : &tm_kc);
-                    const int row = (hist ? j : j - nhb) * BLK;
-                    const uint32_t dst = kv_smem + stage * TILE_BYTES;
-                    tc::tma_load_2d(dst, map, kvh * HD, row, full);
-                    tc::tma_load_2d(dst + HALF_BYTES, map, kvh * HD + 64, row, full);
-                    issued = idx + 1;
+                const int n = part.j1 - part.j0;
+                load_tile(part.j0, false);
+                if (ok && n > 1) load_tile(part.j0 + 1, false);
+                for (int jj = 0; jj < n && ok; ++jj) {
+                    load_tile(part.j0 + jj, true);
+                    if (ok && jj + 2 < n) load_tile(part.j0 + jj + 2, false);
                 }
-                kv_base += n_loads;
                 ++part_idx;
             }
             if (*abort_flag) {
@@ -226,149 +247,150 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
             }
         }
-    } else if (warp == 8) {
-        // ================================ MMA issuer ================================
-        if (lane == 0) {
-            auto issue_qk = [&](int tt, int stage) {
-                const uint32_t a0 = q_smem + tt * TILE_BYTES, b0 = kv_smem + stage * TILE_BYTES;
+    } else if (warp >= 8) {
+        // ================================ MMA issuer of tile tt ================================
+        // All 32 lanes run this code convergently; `elect` is set in lane 0 only and predicates the
+        // tcgen05 instructions, so descriptors and addresses are computed once, warp-uniformly.
+        const int tt = warp - 8;
+        const uint32_t elect = lane == 0;
+        const uint32_t a0 = q_smem + tt * Q_TILE_BYTES;
+        const uint32_t s_col = tmem + tt * 128, o_col = tmem + 256 + tt * 128;
+        auto wait = [&](uint64_t* bar, int parity) {
+            const bool r = tc::mbar_wait(tc::smem_u32(bar), parity, abort_flag);
+            return __all_sync(0xffffffffu, r);
+        };
+        // S_t[buf] = Q_t K^T over the 64 keys of ring stage `stage`
+        auto issue_qk = [&](int buf, int stage) {
+            const uint32_t b0 = kv_smem + stage * KV_TILE_BYTES;
 #pragma unroll
-                for (int kk = 0; kk < HD / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
-                    tc::umma_ss(tmem + tt * 128, tc::umma_smem_desc(a0 + off, 16, 1024),
-                                tc::umma_smem_desc(b0 + off, 16, 1024), IDESC_QK, kk > 0);
-                }
-            };
-            auto issue_pv = [&](int tt, int stage, bool accumulate) {
-                const uint32_t b0 = kv_smem + stage * TILE_BYTES;
+            for (int kk = 0; kk < HD / 16; ++kk) {
+                tc::umma_ss(s_col + buf * 64, tc::umma_smem_desc(a0 + (kk >> 2) * Q_HALF_BYTES + (kk & 3) * 32, 16, 1024),
+                            tc::umma_smem_desc(b0 + (kk >> 2) * KV_HALF_BYTES + (kk & 3) * 32, 16, 1024), IDESC_QK, kk > 0, elect);
+            }
+        };
+        // O_t += P_t[buf] V over the 64 keys of ring stage `stage`
+        auto issue_pv = [&](int buf, int stage, bool accumulate) {
+            const uint32_t b0 = kv_smem + stage * KV_TILE_BYTES;
 #pragma unroll
-                for (int kk = 0; kk < BLK / 16; ++kk) {
-                    tc::umma_ts(tmem + 256 + tt * 128, tmem + tt * 128 + kk * 8,
-                                tc::umma_smem_desc(b0 + kk * 2048, HALF_BYTES, 1024), IDESC_PV, accumulate || kk > 0);
-                }
-            };
-            auto kv_wait = [&](int idx) {
-                return tc::mbar_wait(tc::smem_u32(&bars->kv_full[idx % NSTAGE]), (idx / NSTAGE) & 1, abort_flag);
-            };
-            int sp0 = 0, sp1 = 0;                            // blocks handed to each tile's softmax so far
-            bool ok = true;
-            // one tile's share of a block step: O_t += P_t V_j, then S_t = Q_t K_{j+1}
-            auto tile_step = [&](int tt, int cnt, int& sp, int jj, int v_stage, int k_stage) {
-                if (jj < cnt) {
-                    ok = tc::mbar_wait(tc::smem_u32(&bars->p_full[tt]), sp & 1, abort_flag);
-                    ++sp;
-                    // the first PV of a part overwrites O_t: the previous part's epilogue must have read it
-                    if (ok && jj == 0 && part_idx > 0)
-                        ok = tc::mbar_wait(tc::smem_u32(&bars->o_free[tt]), (part_idx - 1) & 1, abort_flag);
-                    if (!ok) return;
-                    tc::tcgen05_fence_after();
-                    issue_pv(tt, v_stage, jj > 0);
-                }
-                if (jj + 1 < cnt) {
-                    issue_qk(tt, k_stage);
-                    tc::umma_commit(tc::smem_u32(&bars->s_full[tt]));
-                }
-            };
-            while (ok && it.next(part)) {
-                const int n = part.j1 - part.j0;
-                ok = tc::mbar_wait(tc::smem_u32(&bars->q_full), part_idx & 1, abort_flag);
-                if (ok) ok = kv_wait(kv_base);
+            for (int kk = 0; kk < BK / 16; ++kk) {
+                tc::umma_ts(o_col, s_col + buf * 64 + kk * 8, tc::umma_smem_desc(b0 + kk * 2048, KV_HALF_BYTES, 1024), IDESC_PV,
+                            accumulate || kk > 0, elect);
+            }
+        };
+        int cons = 0;                                    // K/V tiles consumed so far (same order as produced)
+        int g = 0;                                       // blocks of this tile started so far (buffer = g & 1)
+        bool ok = true;
+        while (ok && it.next(part)) {
+            const int n = part.j1 - part.j0;
+            const int cnt = tt ? part.cnt1 : part.cnt0;
+            ok = wait(&bars->q_full, part_idx & 1);
+            // S of the first two blocks
+            for (int jj = 0; jj < 2 && jj < n && ok; ++jj) {
+                ok = wait(&bars->kv_full[cons % NSTAGE], (cons / NSTAGE) & 1);
                 if (!ok) break;
                 tc::tcgen05_fence_after();
-                if (part.cnt0 > 0) {
-                    issue_qk(0, kv_base % NSTAGE);
-                    tc::umma_commit(tc::smem_u32(&bars->s_full[0]));
+                if (jj < cnt) {
+                    issue_qk((g + jj) & 1, cons % NSTAGE);
+                    tc::umma_commit(tc::smem_u32(&bars->s_full[tt][(g + jj) & 1]), elect);
                 }
-                if (part.cnt1 > 0) {
-                    issue_qk(1, kv_base % NSTAGE);
-                    tc::umma_commit(tc::smem_u32(&bars->s_full[1]));
-                }
-                tc::umma_commit(tc::smem_u32(&bars->kv_empty[kv_base % NSTAGE]));
-                for (int jj = 0; jj < n && ok; ++jj) {
-                    const int v_idx = kv_base + 2 * jj + 1, k_idx = v_idx + 1;
-                    const bool has_next = jj + 1 < n;
-                    ok = kv_wait(v_idx);
-                    if (ok && has_next) ok = kv_wait(k_idx);
-                    if (ok) tile_step(0, part.cnt0, sp0, jj, v_idx % NSTAGE, k_idx % NSTAGE);
-                    if (ok) tile_step(1, part.cnt1, sp1, jj, v_idx % NSTAGE, k_idx % NSTAGE);
-                    if (!ok) break;
-                    tc::umma_commit(tc::smem_u32(&bars->kv_empty[v_idx % NSTAGE]));
-                    if (has_next) tc::umma_commit(tc::smem_u32(&bars->kv_empty[k_idx % NSTAGE]));
-                }
-                // every softmax warpgroup must have seen the previous part's o_done before this part's is
-                // committed (a waiter may lag one mbarrier phase, never two)
-                if (ok && part_idx > 0) ok = tc::mbar_wait(tc::smem_u32(&bars->o_free[0]), (part_idx - 1) & 1, abort_flag);
-                if (ok && part_idx > 0) ok = tc::mbar_wait(tc::smem_u32(&bars->o_free[1]), (part_idx - 1) & 1, abort_flag);
-                if (ok) tc::umma_commit(tc::smem_u32(&bars->o_done));
-                kv_base += 2 * n;
-                ++part_idx;
+                tc::umma_commit(tc::smem_u32(&bars->kv_empty[cons % NSTAGE]), elect);
+                ++cons;
             }
+            for (int jj = 0; jj < n && ok; ++jj) {
+                const int v_idx = cons, k_idx = cons + 1;
+                const bool has_k = jj + 2 < n;
+                const int gb = g + jj;                   // running block index of this tile
+                // both warps walk every stage, in step with the producer, also past their own tile's last block
+                ok = wait(&bars->kv_full[v_idx % NSTAGE], (v_idx / NSTAGE) & 1);
+                if (ok && has_k) ok = wait(&bars->kv_full[k_idx % NSTAGE], (k_idx / NSTAGE) & 1);
+                if (ok && jj < cnt) {
+                    ok = wait(&bars->p_full[tt][gb & 1], (gb >> 1) & 1);
+                    // the first PV of a part overwrites O_t: the previous part's epilogue must have read it
+                    if (ok && jj == 0 && part_idx > 0) ok = wait(&bars->o_free[tt], (part_idx - 1) & 1);
+                    if (ok) {
+                        tc::tcgen05_fence_after();
+                        issue_pv(gb & 1, v_idx % NSTAGE, jj > 0);
+                        tc::umma_commit(tc::smem_u32(&bars->pv_done[tt]), elect);
+                    }
+                }
+                if (ok && jj + 2 < cnt) {
+                    issue_qk(gb & 1, k_idx % NSTAGE);
+                    tc::umma_commit(tc::smem_u32(&bars->s_full[tt][gb & 1]), elect);
+                }
+                if (!ok) break;
+                tc::umma_commit(tc::smem_u32(&bars->kv_empty[v_idx % NSTAGE]), elect);
+                if (has_k) tc::umma_commit(tc::smem_u32(&bars->kv_empty[k_idx % NSTAGE]), elect);
+                cons += has_k ? 2 : 1;
+            }
+            // this tile's softmax warpgroup must have seen the previous part's o_done before this part's is
+            // committed (a waiter may lag one mbarrier phase, never two)
+            if (ok && part_idx > 0) ok = wait(&bars->o_free[tt], (part_idx - 1) & 1);
+            if (ok) tc::umma_commit(tc::smem_u32(&bars->o_done), elect);
+            g += cnt;
+            ++part_idx;
         }
     } else {
         // ================================ softmax + epilogue ================================
         const int tt = warp >> 2;                          // tile of this warpgroup
         const int r = (warp & 3) * 32 + lane;              // row inside the tile == TMEM lane
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t s_tmem = tmem + tt * 128 + lane_addr;
         const uint32_t o_tmem = tmem + 256 + tt * 128 + lane_addr;
-        int sp = 0;
+        int g = 0;                                         // blocks of this tile processed so far
         bool ok = true;
         while (it.next(part)) {
-            const int row0 = (2 * part.pair + tt) * BLK;
+            const int row0 = (2 * part.pair + tt) * BQ;
             const int my_n = tt ? part.cnt1 : part.cnt0;
-            const int diag_block = nhb + 2 * part.pair + tt;   // KV block index of the causal diagonal
-            float m_ref = 0.f, l_sum = 0.f;
+            const int n_part = part.j1 - part.j0;
+            const int diag0 = nhb + row0 / BK;             // the two KV blocks that cross the causal diagonal
+            float m_ref = -INFINITY, l_sum = 0.f;
 
-            for (int jj = 0; jj < my_n && ok; ++jj) {
+            for (int jj = 0; jj < my_n && ok; ++jj, ++g) {
                 const int j = part.j0 + jj;
-                ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&bars->s_full[tt]), sp & 1, abort_flag));
-                ++sp;
+                const int buf = g & 1;
+                const uint32_t s_tmem = tmem + tt * 128 + buf * 64 + lane_addr;
+                ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&bars->s_full[tt][buf]), (g >> 1) & 1, abort_flag));
                 tc::tcgen05_fence_after();
-                uint32_t sv[4][32];
-#pragma unroll
-                for (int c = 0; c < 4; ++c) tc::tmem_ld32(s_tmem + c * 32, sv[c]);
+                uint32_t sa[32], sb[32];
+                tc::tmem_ld32(s_tmem, sa);
+                tc::tmem_ld32(s_tmem + 32, sb);
                 tc::tmem_wait_ld();
 
-                // masking: ragged history tail, causal diagonal
-                int n_valid = BLK;
+                // masking: ragged history tail, the two blocks on the causal diagonal
+                int n_valid = BK;
                 if (j == nhb - 1 && tail_partial) n_valid = hist_tail;
-                if (j == diag_block) n_valid = r + 1;
-                if (n_valid < BLK) {
+                if (j == diag0) n_valid = min(BK, r + 1);
+                if (j == diag0 + 1) n_valid = r - (BK - 1);               // <= 0: the row sees nothing of this block
+                if (n_valid < BK) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c)
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (c * 32 + i >= n_valid) sv[c][i] = 0xff800000u;   // -inf
-                }
-                // eight independent running maxima (a single chain of 128 dependent max ops would stall)
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-                float mx4 = -INFINITY, mx5 = -INFINITY, mx6 = -INFINITY, mx7 = -INFINITY;
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-#pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        mx0 = fmaxf(mx0, __uint_as_float(sv[c][i]));
-                        mx1 = fmaxf(mx1, __uint_as_float(sv[c][i + 1]));
-                        mx2 = fmaxf(mx2, __uint_as_float(sv[c][i + 2]));
-                        mx3 = fmaxf(mx3, __uint_as_float(sv[c][i + 3]));
-                        mx4 = fmaxf(mx4, __uint_as_float(sv[c][i + 4]));
-                        mx5 = fmaxf(mx5, __uint_as_float(sv[c][i + 5]));
-                        mx6 = fmaxf(mx6, __uint_as_float(sv[c][i + 6]));
-                        mx7 = fmaxf(mx7, __uint_as_float(sv[c][i + 7]));
+                    for (int i = 0; i < 32; ++i) {
+                        if (i >= n_valid) sa[i] = 0xff800000u;           // -inf
+                        if (32 + i >= n_valid) sb[i] = 0xff800000u;
                     }
-                float bm = fmaxf(fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)), fmaxf(fmaxf(mx4, mx5), fmaxf(mx6, mx7)));
-                if (bm == -INFINITY) bm = 0.f;
+                }
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+                for (int i = 0; i < 32; i += 4) {
+                    mx0 = fmaxf(mx0, fmaxf(__uint_as_float(sa[i]), __uint_as_float(sb[i])));
+                    mx1 = fmaxf(mx1, fmaxf(__uint_as_float(sa[i + 1]), __uint_as_float(sb[i + 1])));
+                    mx2 = fmaxf(mx2, fmaxf(__uint_as_float(sa[i + 2]), __uint_as_float(sb[i + 2])));
+                    mx3 = fmaxf(mx3, fmaxf(__uint_as_float(sa[i + 3]), __uint_as_float(sb[i + 3])));
+                }
+                const float bm = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
 
+                // O_t is touched only after the PV of the previous block has completed
+                if (jj > 0)
+                    ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&bars->pv_done[tt]), (g - 1) & 1, abort_flag));
                 float alpha = 1.f;
                 bool need = false;
-                if (jj == 0) {
-                    m_ref = bm;
+                if (m_ref == -INFINITY) {
+                    m_ref = bm;                              // first block with a visible key (may stay -inf)
                 } else if ((bm - m_ref) * p.scale_log2 > RESCALE_THRESHOLD) {
                     alpha = tc::ex2_approx((m_ref - bm) * p.scale_log2);
                     m_ref = bm;
                     need = true;
                 }
                 if (__any_sync(0xffffffffu, need)) {
-                    // O_t of the previous blocks is complete: S_t(j) was committed after PV_t(j-1)
+                    tc::tcgen05_fence_after();
                     l_sum *= alpha;
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
@@ -380,32 +402,35 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         tc::tmem_st32(o_tmem + c * 32, ov);
                     }
                 }
-                const float neg_m = -m_ref * p.scale_log2;
+                // a row that has seen no key yet keeps m_ref = -inf; exponentiate against 0 so that P = 0, not NaN
+                const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref * p.scale_log2;
                 float rs0 = 0.f, rs1 = 0.f;
+                uint32_t pk[32];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const float p0 = tc::ex2_approx(fmaf(__uint_as_float(sv[c][2 * i]), p.scale_log2, neg_m));
-                        const float p1 = tc::ex2_approx(fmaf(__uint_as_float(sv[c][2 * i + 1]), p.scale_log2, neg_m));
-                        pk[i] = tc::pack_bf16x2(p0, p1);
-                        // the normaliser sums the ROUNDED weights the tensor core will use, so that the
-                        // weights of a row sum to one exactly and the rounding of a dominant weight cancels
-                        rs0 += __uint_as_float(pk[i] << 16);
-                        rs1 += __uint_as_float(pk[i] & 0xffff0000u);
-                    }
-                    tc::tmem_st16(s_tmem + c * 16, pk);
+                for (int i = 0; i < 16; ++i) {
+                    const float a0 = tc::ex2_approx(fmaf(__uint_as_float(sa[2 * i]), p.scale_log2, neg_m));
+                    const float a1 = tc::ex2_approx(fmaf(__uint_as_float(sa[2 * i + 1]), p.scale_log2, neg_m));
+                    const float b0 = tc::ex2_approx(fmaf(__uint_as_float(sb[2 * i]), p.scale_log2, neg_m));
+                    const float b1 = tc::ex2_approx(fmaf(__uint_as_float(sb[2 * i + 1]), p.scale_log2, neg_m));
+                    pk[i] = tc::pack_bf16x2(a0, a1);
+                    pk[16 + i] = tc::pack_bf16x2(b0, b1);
+                    // the normaliser sums the ROUNDED weights the tensor core will use, so that the
+                    // weights of a row sum to one exactly and the rounding of a dominant weight cancels
+                    rs0 += __uint_as_float(pk[i] << 16) + __uint_as_float(pk[i] & 0xffff0000u);
+                    rs1 += __uint_as_float(pk[16 + i] << 16) + __uint_as_float(pk[16 + i] & 0xffff0000u);
                 }
+                tc::tmem_st32(s_tmem, pk);                   // P over the first 32 columns of the S buffer
                 l_sum += rs0 + rs1;
 
-                if (tt == 0 && tail_partial && j == nhb - 1) {
-                    // rows of the V tile past the end of the history may hold anything: zero them
-                    const int v_idx = kv_base + 2 * jj + 1, v_stage = v_idx % NSTAGE;
+                if (tail_partial && j == nhb - 1) {
+                    // rows of the V tile past the end of the history may hold anything: zero them (each tile's
+                    // warpgroup does it before it releases its own PV; the two MMA warps do not wait on each other)
+                    const int v_idx = kv_base + pos_v(jj, n_part), v_stage = v_idx % NSTAGE;
                     ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&bars->kv_full[v_stage]), (v_idx / NSTAGE) & 1, abort_flag));
-                    if (r >= hist_tail) {
-                        uint4* row_a = reinterpret_cast<uint4*>(smem_gen + 2 * TILE_BYTES + v_stage * TILE_BYTES + r * 128);
-                        uint4* row_b = reinterpret_cast<uint4*>(smem_gen + 2 * TILE_BYTES + v_stage * TILE_BYTES + HALF_BYTES + r * 128);
+                    if (r >= hist_tail && r < BK) {
+                        uint8_t* vt = smem_gen + 2 * Q_TILE_BYTES + v_stage * KV_TILE_BYTES + r * 128;
+                        uint4* row_a = reinterpret_cast<uint4*>(vt);
+                        uint4* row_b = reinterpret_cast<uint4*>(vt + KV_HALF_BYTES);
 #pragma unroll
                         for (int i = 0; i < 8; ++i) { row_a[i] = make_uint4(0, 0, 0, 0); row_b[i] = make_uint4(0, 0, 0, 0); }
                     }
@@ -413,13 +438,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
                 tc::tmem_wait_st();
                 tc::tcgen05_fence_before();
-                tc::mbar_arrive(tc::smem_u32(&bars->p_full[tt]));
+                tc::mbar_arrive(tc::smem_u32(&bars->p_full[tt][buf]));
             }
 
             const int row = row0 + r;
             const size_t pslot = ((size_t)blockIdx.x * 2 + part.slot) * 2 + tt;
+            ok = __all_sync(0xffffffffu, ok && tc::mbar_wait(tc::smem_u32(&bars->o_done), part_idx & 1, abort_flag));
             if (my_n > 0) {
-                ok = __all_sync(0xffffffffu, ok && tc::mbar_wait(tc::smem_u32(&bars->o_done), part_idx & 1, abort_flag));
                 tc::tcgen05_fence_after();
                 const float inv = part.final_ ? 1.f / l_sum : 1.f;
 #pragma unroll
@@ -429,7 +454,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     tc::tmem_wait_ld();
                     if (!ok) continue;
                     if (!part.final_) {
-                        float4* dst = reinterpret_cast<float4*>(p.part_o + (pslot * BLK + r) * HD + c * 32);
+                        float4* dst = reinterpret_cast<float4*>(p.part_o + (pslot * BQ + r) * HD + c * 32);
 #pragma unroll
                         for (int i = 0; i < 8; ++i)
                             dst[i] = make_float4(__uint_as_float(ov[4 * i]), __uint_as_float(ov[4 * i + 1]),
@@ -456,18 +481,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         }
                     }
                 }
-                if (ok && !part.final_) p.part_ml[pslot * BLK + r] = make_float2(m_ref, l_sum);
+                if (ok && !part.final_) p.part_ml[pslot * BQ + r] = make_float2(m_ref, l_sum);
                 if (ok && part.final_ && p.lse_out && row < p.t)
                     p.lse_out[(size_t)row * p.h_q + part.head] = m_ref * p.scale + logf(l_sum);
-            } else {
-                // no block of this tile in the part: still consume the part's o_done phase, in step with the others
-                ok = __all_sync(0xffffffffu, ok && tc::mbar_wait(tc::smem_u32(&bars->o_done), part_idx & 1, abort_flag));
-                if (!part.final_) p.part_ml[pslot * BLK + r] = make_float2(-INFINITY, 0.f);
+            } else if (!part.final_) {
+                p.part_ml[pslot * BQ + r] = make_float2(-INFINITY, 0.f);        // no block of this tile in the part
             }
             // O_t (and the part's Q tile) may be reused
             tc::tcgen05_fence_before();
             tc::mbar_arrive(tc::smem_u32(&bars->o_free[tt]));
-            kv_base += 2 * (part.j1 - part.j0);
+            kv_base += 2 * n_part;
             ++part_idx;
         }
     }
@@ -482,65 +505,67 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 }
 
 // Merge the partial outputs of every item that was cut between CTAs.  Grid (items, 8 groups of 32 rows);
-// a warp owns 4 rows and a lane 4 of a row's 128 columns.
-constexpr int MERGE_MAX_PARTS = 8;
+// a warp owns 4 rows and a lane 4 of a row's 128 columns.  Shared memory: one int per CTA of the main kernel.
+constexpr int MERGE_BATCH = 4;
 __global__ void __launch_bounds__(256) attention_merge_kernel(const AttnParams p, int n_cta) {
+    extern __shared__ int s_slot[];                          // partial slot of every part of the item
+    __shared__ int s_n;
     const int pair = p.n_pairs - 1 - blockIdx.x / p.h_q;
     const int head = blockIdx.x % p.h_q;
-    int n_hist = p.n_hist_dev ? *p.n_hist_dev : p.n_hist_max;
-    n_hist = max(0, min(n_hist, p.n_hist_max));
-    Sched s;
-    s.nhb = (n_hist + BLK - 1) / BLK; s.n_pairs = p.n_pairs; s.h_q = p.h_q; s.t = p.t;
-    const long long total = s.total();
-    const long long w0 = s.item_begin(pair, head);
-    const int nb = s.nb_pair(pair);
-    auto cta_of = [&](long long w) {
-        int b = (int)(w * n_cta / total);
-        b = max(0, min(b, n_cta - 1));
-        while (b + 1 < n_cta && share_begin(total, b + 1, n_cta) <= w) ++b;
-        while (b > 0 && share_begin(total, b, n_cta) > w) --b;
-        return b;
-    };
-    const int b_first = cta_of(w0), b_last = cta_of(w0 + nb - 1);
-    if (b_first == b_last) return;                           // the item was computed by one CTA
+    if (threadIdx.x == 0) {
+        int n_hist = p.n_hist_dev ? *p.n_hist_dev : p.n_hist_max;
+        n_hist = max(0, min(n_hist, p.n_hist_max));
+        Sched s;
+        s.nhb = (n_hist + BK - 1) / BK; s.n_pairs = p.n_pairs; s.h_q = p.h_q; s.t = p.t;
+        const long long total = s.total();
+        const long long w0 = s.item_begin(pair, head);
+        const int nb = s.nb_pair(pair);
+        auto cta_of = [&](long long w) {
+            int b = (int)(w * n_cta / total);
+            b = max(0, min(b, n_cta - 1));
+            while (b + 1 < n_cta && share_begin(total, b + 1, n_cta) <= w) ++b;
+            while (b > 0 && share_begin(total, b, n_cta) > w) --b;
+            return b;
+        };
+        const int b_first = cta_of(w0), b_last = cta_of(w0 + nb - 1);
+        int n = 0;
+        if (b_first != b_last)
+            for (int b = b_first; b <= b_last; ++b)
+                if (share_begin(total, b, n_cta) != share_begin(total, b + 1, n_cta))
+                    s_slot[n++] = b * 2 + (b == b_first ? 1 : 0);
+        s_n = n;
+    }
+    __syncthreads();
+    const int n_parts = s_n;
+    if (n_parts == 0) return;                                // the item was computed by one CTA
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int q4 = 0; q4 < 4; ++q4) {
         const int rr = blockIdx.y * 32 + warp * 4 + q4;      // 0..255: tile * 128 + row
-        const int tt = rr / BLK, r = rr % BLK;
-        const int row = (2 * pair + tt) * BLK + r;
+        const int tt = rr / BQ, r = rr % BQ;
+        const int row = (2 * pair + tt) * BQ + r;
         if (row >= p.t) continue;
         float M = -INFINITY;
-        for (int b0 = b_first; b0 <= b_last; b0 += MERGE_MAX_PARTS) {      // (an item rarely has more than 3 parts)
-            float2 ml[MERGE_MAX_PARTS];
-#pragma unroll
-            for (int i = 0; i < MERGE_MAX_PARTS; ++i) {
-                const int b = b0 + i;
-                ml[i] = make_float2(-INFINITY, 0.f);
-                if (b <= b_last && share_begin(total, b, n_cta) != share_begin(total, b + 1, n_cta))
-                    ml[i] = p.part_ml[(((size_t)b * 2 + (b == b_first ? 1 : 0)) * 2 + tt) * BLK + r];
-            }
-#pragma unroll
-            for (int i = 0; i < MERGE_MAX_PARTS; ++i)
-                if (ml[i].y > 0.f) M = fmaxf(M, ml[i].x);
+        for (int i = 0; i < n_parts; ++i) {
+            const float2 ml = p.part_ml[((size_t)s_slot[i] * 2 + tt) * BQ + r];
+            if (ml.y > 0.f) M = fmaxf(M, ml.x);
         }
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         float L = 0.f;
-        for (int b0 = b_first; b0 <= b_last; b0 += MERGE_MAX_PARTS) {
-            float2 ml[MERGE_MAX_PARTS];
-            float4 o[MERGE_MAX_PARTS];
+        for (int i0 = 0; i0 < n_parts; i0 += MERGE_BATCH) {
+            float2 ml[MERGE_BATCH];
+            float4 o[MERGE_BATCH];
 #pragma unroll
-            for (int i = 0; i < MERGE_MAX_PARTS; ++i) {
-                const int b = b0 + i;
+            for (int i = 0; i < MERGE_BATCH; ++i) {
                 ml[i] = make_float2(-INFINITY, 0.f);
                 o[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (b <= b_last && share_begin(total, b, n_cta) != share_begin(total, b + 1, n_cta)) {
-                    const size_t pslot = ((size_t)b * 2 + (b == b_first ? 1 : 0)) * 2 + tt;
-                    ml[i] = p.part_ml[pslot * BLK + r];
-                    if (ml[i].y > 0.f) o[i] = *reinterpret_cast<const float4*>(p.part_o + (pslot * BLK + r) * HD + lane * 4);
+                if (i0 + i < n_parts) {
+                    const size_t pslot = (size_t)s_slot[i0 + i] * 2 + tt;
+                    ml[i] = p.part_ml[pslot * BQ + r];
+                    if (ml[i].y > 0.f) o[i] = *reinterpret_cast<const float4*>(p.part_o + (pslot * BQ + r) * HD + lane * 4);
                 }
             }
 #pragma unroll
-            for (int i = 0; i < MERGE_MAX_PARTS; ++i) {
+            for (int i = 0; i < MERGE_BATCH; ++i) {
                 if (!(ml[i].y > 0.f)) continue;
                 const float wgt = exp2f((ml[i].x - M) * p.scale_log2);
                 acc.x += wgt * o[i].x; acc.y += wgt * o[i].y; acc.z += wgt * o[i].z; acc.w += wgt * o[i].w;
@@ -570,19 +595,22 @@ omni_status omni_attention_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q,
     const omni_geometry& g = ctx->g;
     CUtensorMap tm_q, tm_kh, tm_vh, tm_kc, tm_vc;
     const uint64_t q_inner = (uint64_t)g.h_q * HD, kv_inner = (uint64_t)g.h_kv * HD;
-    bool ok = omni_make_map_bf16(ctx->encode_tiled, &tm_q, q, t, q_inner, BLK);
-    ok &= omni_make_map_bf16(ctx->encode_tiled, &tm_kc, k_chunk, t, kv_inner, BLK);
-    ok &= omni_make_map_bf16(ctx->encode_tiled, &tm_vc, v_chunk, t, kv_inner, BLK);
+    bool ok = omni_make_map_bf16(ctx->encode_tiled, &tm_q, q, t, q_inner, BQ);
+    ok &= omni_make_map_bf16(ctx->encode_tiled, &tm_kc, k_chunk, t, kv_inner, BK);
+    ok &= omni_make_map_bf16(ctx->encode_tiled, &tm_vc, v_chunk, t, kv_inner, BK);
     // with an empty history the history maps are never used; point them at the chunk to stay valid
-    ok &= omni_make_map_bf16(ctx->encode_tiled, &tm_kh, n_hist_max > 0 ? k_hist : k_chunk, n_hist_max > 0 ? n_hist_max : t, kv_inner, BLK);
-    ok &= omni_make_map_bf16(ctx->encode_tiled, &tm_vh, n_hist_max > 0 ? v_hist : v_chunk, n_hist_max > 0 ? n_hist_max : t, kv_inner, BLK);
+    ok &= omni_make_map_bf16(ctx->encode_tiled, &tm_kh, n_hist_max > 0 ? k_hist : k_chunk, n_hist_max > 0 ? n_hist_max : t, kv_inner, BK);
+    ok &= omni_make_map_bf16(ctx->encode_tiled, &tm_vh, n_hist_max > 0 ? v_hist : v_chunk, n_hist_max > 0 ? n_hist_max : t, kv_inner, BK);
     if (!ok) OMNI_FAIL(ctx, OMNI_ERR_CUDA, "attention: cuTensorMapEncodeTiled failed");
-    const int n_cta = ctx->sm_count;
     AttnParams p;
     p.t = t; p.h_q = g.h_q; p.h_kv = g.h_kv; p.n_hist_dev = n_hist_dev; p.n_hist_max = n_hist_max;
     p.scale = scale; p.scale_log2 = scale * 1.4426950408889634f;
     p.o_out = o_out; p.out_dtype = out_dtype; p.lse_out = lse_out; p.status = ctx->status_dev;
-    p.n_pairs = (t + 2 * BLK - 1) / (2 * BLK);
+    p.n_pairs = (t + 2 * BQ - 1) / (2 * BQ);
+    // one CTA per SM, fewer when the whole job is small (at least 8 block steps per CTA)
+    long long w_max = 0;
+    for (int pr = 0; pr < p.n_pairs; ++pr) w_max += (long long)g.h_q * ((n_hist_max + BK - 1) / BK + 4 * pr + 4);
+    const int n_cta = (int)std::max(1ll, std::min((long long)ctx->sm_count, w_max / 8));
     p.part_o = ctx->attn_part_o; p.part_ml = reinterpret_cast<float2*>(ctx->attn_part_ml);
     static bool attr_set = false;
     if (!attr_set) {
@@ -591,7 +619,7 @@ omni_status omni_attention_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q,
     }
     attention_tc_kernel<<<n_cta, ATT_THREADS, SMEM_BYTES, st>>>(tm_q, tm_kh, tm_vh, tm_kc, tm_vc, p);
     OMNI_CHECK_LAUNCH(ctx, "attention_tc_kernel");
-    attention_merge_kernel<<<dim3(p.n_pairs * g.h_q, 8), 256, 0, st>>>(p, n_cta);
+    attention_merge_kernel<<<dim3(p.n_pairs * g.h_q, 8), 256, (n_cta + 1) * sizeof(int), st>>>(p, n_cta);
     OMNI_CHECK_LAUNCH(ctx, "attention_merge_kernel");
     return OMNI_OK;
 }

@@ -155,7 +155,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     for (int kk = 0; kk < HD / 16; ++kk) {
                         const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
                         tc::umma_ss(tmem + tt * 256 + buf * 128, tc::umma_smem_desc(a0 + off, 16, 1024),
-                                    tc::umma_smem_desc(bb + off, 16, 1024), IDESC_QK, kk > 0);
+                                    tc::umma_smem_desc(bb + off, 16, 1024), IDESC_QK, kk > 0, 1u);
                     }
                     tc::umma_commit(tc::smem_u32(&bars->s_full[tt][buf]));
                 }
