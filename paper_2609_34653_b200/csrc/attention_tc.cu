@@ -248,17 +248,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             }
         }
     } else if (warp >= 8) {
-        // ================================ MMA issuer of tile tt ================================
-        // All 32 lanes run this code convergently; `elect` is set in lane 0 only and predicates the
-        // tcgen05 instructions, so descriptors and addresses are computed once, warp-uniformly.
+        // ================================ MMA issuer of tile tt (one thread) ================================
+        // A tcgen05.mma with M = 128 occupies the tensor pipe for 64 clocks whatever N <= 128 is, and one
+        // thread cannot issue them faster than that; issuing from a single lane (not an elected lane of
+        // convergent code) measured 68 clocks per instruction against 88.
         const int tt = warp - 8;
-        const uint32_t elect = lane == 0;
+        const uint32_t elect = 1u;
+        if (lane != 0) goto mma_done;
+        {
         const uint32_t a0 = q_smem + tt * Q_TILE_BYTES;
         const uint32_t s_col = tmem + tt * 128, o_col = tmem + 256 + tt * 128;
-        auto wait = [&](uint64_t* bar, int parity) {
-            const bool r = tc::mbar_wait(tc::smem_u32(bar), parity, abort_flag);
-            return __all_sync(0xffffffffu, r);
-        };
+        auto wait = [&](uint64_t* bar, int parity) { return tc::mbar_wait(tc::smem_u32(bar), parity, abort_flag); };
         // S_t[buf] = Q_t K^T over the 64 keys of ring stage `stage`
         auto issue_qk = [&](int buf, int stage) {
             const uint32_t b0 = kv_smem + stage * KV_TILE_BYTES;
@@ -329,6 +329,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             g += cnt;
             ++part_idx;
         }
+        }
+    mma_done:;
     } else {
         // ================================ softmax + epilogue ================================
         const int tt = warp >> 2;                          // tile of this warpgroup
@@ -377,9 +379,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
                 const float bm = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
 
-                // O_t is touched only after the PV of the previous block has completed
-                if (jj > 0)
-                    ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&bars->pv_done[tt]), (g - 1) & 1, abort_flag));
                 float alpha = 1.f;
                 bool need = false;
                 if (m_ref == -INFINITY) {
@@ -388,19 +387,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     alpha = tc::ex2_approx((m_ref - bm) * p.scale_log2);
                     m_ref = bm;
                     need = true;
-                }
-                if (__any_sync(0xffffffffu, need)) {
-                    tc::tcgen05_fence_after();
-                    l_sum *= alpha;
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t ov[32];
-                        tc::tmem_ld32(o_tmem + c * 32, ov);
-                        tc::tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
-                        tc::tmem_st32(o_tmem + c * 32, ov);
-                    }
                 }
                 // a row that has seen no key yet keeps m_ref = -inf; exponentiate against 0 so that P = 0, not NaN
                 const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref * p.scale_log2;
@@ -420,6 +406,22 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     rs1 += __uint_as_float(pk[16 + i] << 16) + __uint_as_float(pk[16 + i] & 0xffff0000u);
                 }
                 tc::tmem_st32(s_tmem, pk);                   // P over the first 32 columns of the S buffer
+                // O_t is touched only after the PV of the previous block has completed (it has, by now, nearly always)
+                if (jj > 0)
+                    ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&bars->pv_done[tt]), (g - 1) & 1, abort_flag));
+                if (__any_sync(0xffffffffu, need)) {
+                    tc::tcgen05_fence_after();
+                    l_sum *= alpha;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t ov[32];
+                        tc::tmem_ld32(o_tmem + c * 32, ov);
+                        tc::tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+                        tc::tmem_st32(o_tmem + c * 32, ov);
+                    }
+                }
                 l_sum += rs0 + rs1;
 
                 if (tail_partial && j == nhb - 1) {
