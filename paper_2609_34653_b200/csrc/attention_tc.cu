@@ -1,23 +1,26 @@
 // GQA chunk-prefill attention on tcgen05 tensor cores (bf16, head dim 128).
 //
-// Work unit: one 64-key KV block of one "item" = (pair of 128-row query tiles, head).  The KV sequence
-// of an item is the history blocks followed by the causal chunk blocks.  The kernel is persistent, one
-// CTA per SM: the units of all items are laid end to end and cut into equal contiguous shares, so every
-// SM gets the same amount of tensor work whatever the number of items.  A share is a list of "parts"
-// (item, block range).  A part that covers its whole item writes the output directly; an item cut
-// between CTAs leaves un-normalised partial outputs with their (max, sum) in scratch and a small
-// second kernel merges them.
+// Work unit: one 128-key KV block of one "item" = (128-row query tile, head).  The KV sequence of an item
+// is the history blocks followed by the causal chunk blocks.  The kernel is persistent, one CTA per SM:
+// the units of all items are laid end to end and cut into equal contiguous shares, so every SM gets the
+// same amount of tensor work whatever the number of items.  A share is a list of "parts" (item, block
+// range).  A part that covers its whole item writes the output directly; an item cut between CTAs leaves
+// un-normalised partial outputs with their (max, sum) in scratch and a small second kernel merges them.
 //
 // Inside a CTA:
-//   warp 10     TMA producer: the part's Q tiles, then K / V tiles (64 keys) through an 8-stage ring
-//   warps 8, 9  MMA issuer of tile 0 / tile 1 (one elected lane, warp-uniform code): S_t = Q_t K_j^T
-//               (operands in shared memory) and O_t += P_t V_j (P read from tensor memory, V as an
-//               MN-major shared-memory operand).  One issuer per tile: issuing is the scarce resource.
-//   warps 0-3   softmax of tile 0, one thread per query row: S from TMEM, running max with lazy
-//   warps 4-7   rescale of O, exp2, P written back to TMEM as bf16 over the S columns; same for tile 1
-// S is double-buffered per tile, and QK^T runs two blocks ahead of PV, so the softmax of block j never
-// waits for the tensor pipe: S_{j+1} is already in tensor memory when block j is done.
-// TMEM map (512 columns): tile t: S/P buffer 0 [128t, 128t+64)  buffer 1 [128t+64, 128t+128);  O_t [256+128t, +128).
+//   warp 9      TMA producer: the part's Q tile, then K / V tiles (128 keys) through a 5-stage ring
+//   warp 8      one thread issues tcgen05.mma.  S = Q K_j^T is one N = 128 instruction group (an M = 128
+//               instruction occupies the tensor pipe for 64 clocks whatever N <= 128 is, so narrower
+//               blocks would waste it); S is double-buffered and runs two blocks ahead of PV.
+//   warps 0-3   softmax warpgroup A: columns 0-63 of every S block (keys 0-63 of the block)
+//   warps 4-7   softmax warpgroup B: columns 64-127.  One thread per query row and half block: logits
+//               from tensor memory, running max with lazy rescale, exp2, P written back over the S columns
+//               as bf16.  Each warpgroup is its own online-softmax stream with its own accumulator:
+//               O_A += P_A V[keys 0-63], O_B += P_B V[keys 64-127]; the two are merged by their (max, sum)
+//               when the part ends.  Two warpgroups keep the exp unit busy; splitting columns instead of
+//               owning two query tiles leaves tensor memory for the second S buffer.
+// TMEM map (512 columns): S buffer 0 [0,128)  S buffer 1 [128,256)  O_A [256,384)  O_B [384,512);
+// P_A / P_B overwrite columns [0,32) / [64,96) of their S buffer.
 #include "common.cuh"
 #include "tc_ptx.cuh"
 
@@ -26,20 +29,30 @@
 namespace {
 
 constexpr int BQ = 128;                  // rows per query tile
-constexpr int BK = 64;                   // keys per KV block
+constexpr int BK = 128;                  // keys per KV block
+constexpr int HK = 64;                   // keys per softmax warpgroup and block
 constexpr int HD = 128;                  // head dim
-constexpr int Q_TILE_BYTES = BQ * HD * 2;    // 32 KiB, two 64-column halves of 16 KiB
-constexpr int Q_HALF_BYTES = Q_TILE_BYTES / 2;
-constexpr int KV_TILE_BYTES = BK * HD * 2;   // 16 KiB, two 64-column halves of 8 KiB
-constexpr int KV_HALF_BYTES = KV_TILE_BYTES / 2;
-constexpr int NSTAGE = 8;
-constexpr int ATT_THREADS = 352;
-constexpr int SMEM_BYTES = 2 * Q_TILE_BYTES + NSTAGE * KV_TILE_BYTES + 1024 /*alignment*/ + 512 /*barriers*/;
+constexpr int TILE_BYTES = 128 * HD * 2; // 32 KiB (Q, K and V tiles), two 64-column halves of 16 KiB
+constexpr int HALF_BYTES = TILE_BYTES / 2;
+constexpr int NSTAGE = 5;
+constexpr int ATT_THREADS = 320;
+constexpr int XCH_BYTES = BQ * 2 * 8;    // (max, sum) of both warpgroups, exchanged when a part ends
+constexpr int SMEM_BYTES = TILE_BYTES + NSTAGE * TILE_BYTES + 1024 /*alignment*/ + 512 /*barriers*/ + XCH_BYTES;
 // O is rescaled only when the row max grows by more than this many log2 units (P stays below 2^8).
 constexpr float RESCALE_THRESHOLD = 8.0f;
 
 constexpr uint32_t IDESC_QK = tc::umma_idesc_bf16(128, BK, false, false);
 constexpr uint32_t IDESC_PV = tc::umma_idesc_bf16(128, HD, false, true);
+
+// Debug aid (-DATT_TRACE): CTA 0 records clock64() stamps of a few blocks and prints them at exit.
+#ifdef ATT_TRACE
+#define TRACE_N 40
+#define TRACE(role, k) do { if (blockIdx.x == 0 && lane == 0 && trace_i < TRACE_N) trace_buf[((role) * TRACE_N + trace_i) * 6 + (k)] = clock64(); } while (0)
+#define TRACE_NEXT() (++trace_i)
+#else
+#define TRACE(role, k)
+#define TRACE_NEXT()
+#endif
 
 struct AttnParams {
     int t, h_q, h_kv;
@@ -47,50 +60,44 @@ struct AttnParams {
     float scale_log2, scale;
     void* o_out; int out_dtype; float* lse_out;
     int32_t* status;
-    int n_pairs;
-    float* part_o;        // [cta][2 slots][2 tiles][128 rows][128] un-normalised partial outputs
-    float2* part_ml;      // [cta][2 slots][2 tiles][128 rows] (running max, sum)
+    int n_tiles;          // query tiles of 128 rows
+    float* part_o;        // [cta][2 slots][128 rows][128] un-normalised partial outputs
+    float2* part_ml;      // [cta][2 slots][128 rows] (running max, sum)
 };
 
 struct Barriers {
     uint64_t q_full;
     uint64_t kv_full[NSTAGE];
     uint64_t kv_empty[NSTAGE];
-    uint64_t s_full[2][2];      // [tile][buffer]
-    uint64_t p_full[2][2];
-    uint64_t pv_done[2];        // one phase per PV of the tile
+    uint64_t s_full[2];         // [buffer]
+    uint64_t p_full[2][2];      // [warpgroup][buffer]
+    uint64_t pv_done;           // one phase per block: both PVs of the block have completed
     uint64_t o_done;
-    uint64_t o_free[2];
+    uint64_t o_free;            // both warpgroups have read O of the part
     uint32_t tmem_base;
     int abort_flag;
 };
 
 // ---- the work list: identical arithmetic in every role and in the merge kernel --------------------------
 struct Sched {
-    int nhb, n_pairs, h_q, t;                                // nhb: 64-key blocks of history
-    __device__ int nb_tile(int pair, int tt) const {         // KV blocks tile tt of a pair attends to
-        const int row0 = (2 * pair + tt) * BQ;
-        return row0 < t ? nhb + row0 / BK + 2 : 0;           // chunk blocks 0 .. row0/64 + 1 reach the diagonal
-    }
-    __device__ int nb_pair(int pair) const { return max(nb_tile(pair, 0), nb_tile(pair, 1)); }
+    int nhb, n_tiles, h_q;                                   // nhb: 128-key blocks of history
+    __device__ int nb_item(int qt) const { return nhb + qt + 1; }      // history + chunk blocks 0 .. qt (the diagonal)
     __device__ long long total() const {
-        long long w = 0;
-        for (int pr = 0; pr < n_pairs; ++pr) w += (long long)h_q * nb_pair(pr);
-        return w;
+        return (long long)h_q * ((long long)n_tiles * (nhb + 1) + (long long)n_tiles * (n_tiles - 1) / 2);
     }
-    // items are ordered by descending pair, then head
-    __device__ long long item_begin(int pair, int head) const {
+    // items are ordered by descending query tile, then head
+    __device__ long long item_begin(int qt, int head) const {
         long long w = 0;
-        for (int pr = n_pairs - 1; pr > pair; --pr) w += (long long)h_q * nb_pair(pr);
-        return w + (long long)head * nb_pair(pair);
+        for (int q = n_tiles - 1; q > qt; --q) w += (long long)h_q * nb_item(q);
+        return w + (long long)head * nb_item(qt);
     }
-    __device__ void locate(long long w, int& pair, int& head, int& j) const {
+    __device__ void locate(long long w, int& qt, int& head, int& j) const {
         long long base = 0;
-        for (int pr = n_pairs - 1; pr >= 0; --pr) {
-            const int nb = nb_pair(pr);
+        for (int q = n_tiles - 1; q >= 0; --q) {
+            const int nb = nb_item(q);
             const long long span = (long long)h_q * nb;
-            if (w < base + span || pr == 0) {
-                pair = pr;
+            if (w < base + span || q == 0) {
+                qt = q;
                 head = (int)((w - base) / nb);
                 j = (int)((w - base) - (long long)head * nb);
                 return;
@@ -102,8 +109,7 @@ struct Sched {
 __device__ __forceinline__ long long share_begin(long long total, int cta, int n_cta) { return total * cta / n_cta; }
 
 struct Part {
-    int pair, head, j0, j1, nb_item;
-    int cnt0, cnt1;       // blocks of this part tile 0 / tile 1 takes part in
+    int qt, head, j0, j1;
     bool final_;          // the part covers the whole item
     int slot;             // partial slot of this CTA (when not final)
 };
@@ -113,14 +119,11 @@ struct PartIter {
     long long w, w_end;
     __device__ bool next(Part& p) {
         if (w >= w_end) return false;
-        s.locate(w, p.pair, p.head, p.j0);
-        p.nb_item = s.nb_pair(p.pair);
-        const long long room = w_end - w;
-        p.j1 = (int)min((long long)p.nb_item, (long long)p.j0 + room);
+        s.locate(w, p.qt, p.head, p.j0);
+        const int nb = s.nb_item(p.qt);
+        p.j1 = (int)min((long long)nb, (long long)p.j0 + (w_end - w));
         w += p.j1 - p.j0;
-        p.cnt0 = max(0, min(p.j1, s.nb_tile(p.pair, 0)) - p.j0);
-        p.cnt1 = max(0, min(p.j1, s.nb_tile(p.pair, 1)) - p.j0);
-        p.final_ = p.j0 == 0 && p.j1 == p.nb_item;
+        p.final_ = p.j0 == 0 && p.j1 == nb;
         p.slot = p.j0 > 0 ? 0 : 1;
         return true;
     }
@@ -129,6 +132,8 @@ struct PartIter {
 // Position, in the part's load order  K0 K1 V0 K2 V1 K3 ... V_{n-2} V_{n-1},  of the V tile of local block jj.
 __device__ __forceinline__ int pos_v(int jj, int n) { return n == 1 ? 1 : (jj == n - 1 ? 2 * n - 1 : 2 + 2 * jj); }
 
+__device__ __forceinline__ void named_barrier_256(int id) { asm volatile("bar.sync %0, 256;" ::"r"(id) : "memory"); }
+
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kh,
                     const __grid_constant__ CUtensorMap tm_vh, const __grid_constant__ CUtensorMap tm_kc,
@@ -136,12 +141,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - tc::smem_u32(smem_raw));
-    const uint32_t q_smem = smem_base;                          // 2 Q tiles
-    const uint32_t kv_smem = smem_base + 2 * Q_TILE_BYTES;      // NSTAGE K/V tiles
-    Barriers* bars = reinterpret_cast<Barriers*>(smem_gen + 2 * Q_TILE_BYTES + NSTAGE * KV_TILE_BYTES);
+    const uint32_t q_smem = smem_base;                          // Q tile
+    const uint32_t kv_smem = smem_base + TILE_BYTES;            // NSTAGE K/V tiles
+    constexpr int KV_OFF = TILE_BYTES;
+    Barriers* bars = reinterpret_cast<Barriers*>(smem_gen + KV_OFF + NSTAGE * TILE_BYTES);
+    float2* xch = reinterpret_cast<float2*>(smem_gen + KV_OFF + NSTAGE * TILE_BYTES + 512);     // [2][128] (m, l)
     volatile int* abort_flag = &bars->abort_flag;
-    const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0);      // provably warp-uniform
-    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     int n_hist = p.n_hist_dev ? *p.n_hist_dev : p.n_hist_max;
     if (n_hist < 0 || n_hist > p.n_hist_max) {
@@ -153,7 +159,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const bool tail_partial = nhb > 0 && hist_tail < BK;
 
     PartIter it;
-    it.s.nhb = nhb; it.s.n_pairs = p.n_pairs; it.s.h_q = p.h_q; it.s.t = p.t;
+    it.s.nhb = nhb; it.s.n_tiles = p.n_tiles; it.s.h_q = p.h_q;
     {
         const long long total = it.s.total();
         it.w = share_begin(total, blockIdx.x, gridDim.x);
@@ -165,17 +171,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         tc::mbar_init(tc::smem_u32(&bars->q_full), 1);
         for (int s = 0; s < NSTAGE; ++s) {
             tc::mbar_init(tc::smem_u32(&bars->kv_full[s]), 1);
-            tc::mbar_init(tc::smem_u32(&bars->kv_empty[s]), 2);          // released by both MMA warps
+            tc::mbar_init(tc::smem_u32(&bars->kv_empty[s]), 1);
         }
-        for (int tt = 0; tt < 2; ++tt) {
-            for (int b = 0; b < 2; ++b) {
-                tc::mbar_init(tc::smem_u32(&bars->s_full[tt][b]), 1);
-                tc::mbar_init(tc::smem_u32(&bars->p_full[tt][b]), 128);
-            }
-            tc::mbar_init(tc::smem_u32(&bars->pv_done[tt]), 1);
-            tc::mbar_init(tc::smem_u32(&bars->o_free[tt]), 128);
+        for (int b = 0; b < 2; ++b) {
+            tc::mbar_init(tc::smem_u32(&bars->s_full[b]), 1);
+            tc::mbar_init(tc::smem_u32(&bars->p_full[0][b]), 128);
+            tc::mbar_init(tc::smem_u32(&bars->p_full[1][b]), 128);
         }
-        tc::mbar_init(tc::smem_u32(&bars->o_done), 2);                   // both MMA warps
+        tc::mbar_init(tc::smem_u32(&bars->pv_done), 1);
+        tc::mbar_init(tc::smem_u32(&bars->o_done), 1);
+        tc::mbar_init(tc::smem_u32(&bars->o_free), 256);
         bars->abort_flag = 0;
         tc::fence_barrier_init();
     }
@@ -183,13 +188,18 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     tc::tcgen05_fence_before();
     __syncthreads();
     tc::tcgen05_fence_after();
-    const uint32_t tmem = __shfl_sync(0xffffffffu, bars->tmem_base, 0);
+    const uint32_t tmem = bars->tmem_base;
 
+#ifdef ATT_TRACE
+    // the tail-part slot of the last CTA is never used by the kernel proper
+    long long* trace_buf = reinterpret_cast<long long*>(p.part_o + ((size_t)(gridDim.x - 1) * 2 + 1) * BQ * HD);
+    int trace_i = 0;
+#endif
     Part part;
     int part_idx = 0;
     int kv_base = 0;                                         // K/V tiles loaded by earlier parts of this CTA
 
-    if (warp == 10) {
+    if (warp == 9) {
         // ================================ TMA producer ================================
         if (lane == 0) {
             tc::tma_prefetch_desc(&tm_q);
@@ -206,29 +216,23 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 ok = tc::mbar_wait(tc::smem_u32(&bars->kv_empty[stage]), (use & 1) ^ 1, abort_flag);
                 if (!ok) return;
                 const uint32_t full = tc::smem_u32(&bars->kv_full[stage]);
-                tc::mbar_expect_tx(full, KV_TILE_BYTES);
+                tc::mbar_expect_tx(full, TILE_BYTES);
                 const bool hist = j < nhb;
                 const CUtensorMap* map = hist ? (is_v ? &tm_vh : &tm_kh) : (is_v ? &tm_vc : &tm_kc);
                 const int row = (hist ? j : j - nhb) * BK;
-                const uint32_t dst = kv_smem + stage * KV_TILE_BYTES;
+                const uint32_t dst = kv_smem + stage * TILE_BYTES;
                 tc::tma_load_2d(dst, map, kvh * HD, row, full);
-                tc::tma_load_2d(dst + KV_HALF_BYTES, map, kvh * HD + 64, row, full);
+                tc::tma_load_2d(dst + HALF_BYTES, map, kvh * HD + 64, row, full);
                 issued = idx + 1;
             };
             while (ok && it.next(part)) {
-                // the Q tiles are free once every MMA of the previous part has completed
+                // the Q tile is free once every MMA of the previous part has completed
                 if (part_idx > 0) ok = tc::mbar_wait(tc::smem_u32(&bars->o_done), (part_idx - 1) & 1, abort_flag);
                 if (!ok) break;
                 kvh = part.head / (p.h_q / p.h_kv);
-                const int n_active = (part.cnt0 > 0) + (part.cnt1 > 0);
-                tc::mbar_expect_tx(tc::smem_u32(&bars->q_full), n_active * Q_TILE_BYTES);
-                for (int tt = 0; tt < 2; ++tt) {
-                    if ((tt ? part.cnt1 : part.cnt0) == 0) continue;
-                    const int row0 = (2 * part.pair + tt) * BQ;
-                    tc::tma_load_2d(q_smem + tt * Q_TILE_BYTES, &tm_q, part.head * HD, row0, tc::smem_u32(&bars->q_full));
-                    tc::tma_load_2d(q_smem + tt * Q_TILE_BYTES + Q_HALF_BYTES, &tm_q, part.head * HD + 64, row0,
-                                    tc::smem_u32(&bars->q_full));
-                }
+                tc::mbar_expect_tx(tc::smem_u32(&bars->q_full), TILE_BYTES);
+                tc::tma_load_2d(q_smem, &tm_q, part.head * HD, part.qt * BQ, tc::smem_u32(&bars->q_full));
+                tc::tma_load_2d(q_smem + HALF_BYTES, &tm_q, part.head * HD + 64, part.qt * BQ, tc::smem_u32(&bars->q_full));
                 const int n = part.j1 - part.j0;
                 load_tile(part.j0, false);
                 if (ok && n > 1) load_tile(part.j0 + 1, false);
@@ -247,122 +251,115 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
             }
         }
-    } else if (warp >= 8) {
-        // ================================ MMA issuer of tile tt (one thread) ================================
-        // A tcgen05.mma with M = 128 occupies the tensor pipe for 64 clocks whatever N <= 128 is, and one
-        // thread cannot issue them faster than that; issuing from a single lane (not an elected lane of
-        // convergent code) measured 68 clocks per instruction against 88.
-        const int tt = warp - 8;
-        const uint32_t elect = 1u;
-        if (lane != 0) goto mma_done;
-        {
-        const uint32_t a0 = q_smem + tt * Q_TILE_BYTES;
-        const uint32_t s_col = tmem + tt * 128, o_col = tmem + 256 + tt * 128;
-        auto wait = [&](uint64_t* bar, int parity) { return tc::mbar_wait(tc::smem_u32(bar), parity, abort_flag); };
-        // S_t[buf] = Q_t K^T over the 64 keys of ring stage `stage`
-        auto issue_qk = [&](int buf, int stage) {
-            const uint32_t b0 = kv_smem + stage * KV_TILE_BYTES;
+    } else if (warp == 8) {
+        // ================================ MMA issuer (one thread) ================================
+        if (lane == 0) {
+            auto wait = [&](uint64_t* bar, int parity) { return tc::mbar_wait(tc::smem_u32(bar), parity, abort_flag); };
+            // S[buf] = Q K^T over the 128 keys of ring stage `stage`
+            auto issue_qk = [&](int buf, int stage) {
+                const uint32_t b0 = kv_smem + stage * TILE_BYTES;
 #pragma unroll
-            for (int kk = 0; kk < HD / 16; ++kk) {
-                tc::umma_ss(s_col + buf * 64, tc::umma_smem_desc(a0 + (kk >> 2) * Q_HALF_BYTES + (kk & 3) * 32, 16, 1024),
-                            tc::umma_smem_desc(b0 + (kk >> 2) * KV_HALF_BYTES + (kk & 3) * 32, 16, 1024), IDESC_QK, kk > 0, elect);
-            }
-        };
-        // O_t += P_t[buf] V over the 64 keys of ring stage `stage`
-        auto issue_pv = [&](int buf, int stage, bool accumulate) {
-            const uint32_t b0 = kv_smem + stage * KV_TILE_BYTES;
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
+                    tc::umma_ss(tmem + buf * 128, tc::umma_smem_desc(q_smem + off, 16, 1024), tc::umma_smem_desc(b0 + off, 16, 1024),
+                                IDESC_QK, kk > 0, 1u);
+                }
+            };
+            // O_w += P_w[buf] V[keys 64w .. 64w+63] of ring stage `stage`
+            auto issue_pv = [&](int w, int buf, int stage, bool accumulate) {
+                const uint32_t b0 = kv_smem + stage * TILE_BYTES + w * (HK * 128);
 #pragma unroll
-            for (int kk = 0; kk < BK / 16; ++kk) {
-                tc::umma_ts(o_col, s_col + buf * 64 + kk * 8, tc::umma_smem_desc(b0 + kk * 2048, KV_HALF_BYTES, 1024), IDESC_PV,
-                            accumulate || kk > 0, elect);
-            }
-        };
-        int cons = 0;                                    // K/V tiles consumed so far (same order as produced)
-        int g = 0;                                       // blocks of this tile started so far (buffer = g & 1)
-        bool ok = true;
-        while (ok && it.next(part)) {
-            const int n = part.j1 - part.j0;
-            const int cnt = tt ? part.cnt1 : part.cnt0;
-            ok = wait(&bars->q_full, part_idx & 1);
-            // S of the first two blocks
-            for (int jj = 0; jj < 2 && jj < n && ok; ++jj) {
-                ok = wait(&bars->kv_full[cons % NSTAGE], (cons / NSTAGE) & 1);
-                if (!ok) break;
-                tc::tcgen05_fence_after();
-                if (jj < cnt) {
+                for (int kk = 0; kk < HK / 16; ++kk) {
+                    tc::umma_ts(tmem + 256 + w * 128, tmem + buf * 128 + w * HK + kk * 8,
+                                tc::umma_smem_desc(b0 + kk * 2048, HALF_BYTES, 1024), IDESC_PV, accumulate || kk > 0, 1u);
+                }
+            };
+            int cons = 0;                                    // K/V tiles consumed so far (same order as produced)
+            int g = 0;                                       // blocks started so far (buffer = g & 1)
+            bool ok = true;
+            while (ok && it.next(part)) {
+                const int n = part.j1 - part.j0;
+                ok = wait(&bars->q_full, part_idx & 1);
+                // S of the first two blocks
+                for (int jj = 0; jj < 2 && jj < n && ok; ++jj) {
+                    ok = wait(&bars->kv_full[cons % NSTAGE], (cons / NSTAGE) & 1);
+                    if (!ok) break;
+                    tc::tcgen05_fence_after();
                     issue_qk((g + jj) & 1, cons % NSTAGE);
-                    tc::umma_commit(tc::smem_u32(&bars->s_full[tt][(g + jj) & 1]), elect);
+                    tc::umma_commit(tc::smem_u32(&bars->s_full[(g + jj) & 1]));
+                    tc::umma_commit(tc::smem_u32(&bars->kv_empty[cons % NSTAGE]));
+                    ++cons;
                 }
-                tc::umma_commit(tc::smem_u32(&bars->kv_empty[cons % NSTAGE]), elect);
-                ++cons;
-            }
-            for (int jj = 0; jj < n && ok; ++jj) {
-                const int v_idx = cons, k_idx = cons + 1;
-                const bool has_k = jj + 2 < n;
-                const int gb = g + jj;                   // running block index of this tile
-                // both warps walk every stage, in step with the producer, also past their own tile's last block
-                ok = wait(&bars->kv_full[v_idx % NSTAGE], (v_idx / NSTAGE) & 1);
-                if (ok && has_k) ok = wait(&bars->kv_full[k_idx % NSTAGE], (k_idx / NSTAGE) & 1);
-                if (ok && jj < cnt) {
-                    ok = wait(&bars->p_full[tt][gb & 1], (gb >> 1) & 1);
-                    // the first PV of a part overwrites O_t: the previous part's epilogue must have read it
-                    if (ok && jj == 0 && part_idx > 0) ok = wait(&bars->o_free[tt], (part_idx - 1) & 1);
-                    if (ok) {
-                        tc::tcgen05_fence_after();
-                        issue_pv(gb & 1, v_idx % NSTAGE, jj > 0);
-                        tc::umma_commit(tc::smem_u32(&bars->pv_done[tt]), elect);
+                for (int jj = 0; jj < n && ok; ++jj) {
+                    const int v_idx = cons, k_idx = cons + 1;
+                    const bool has_k = jj + 2 < n;
+                    const int gb = g + jj, buf = gb & 1;
+                    TRACE(2, 0);
+                    ok = wait(&bars->kv_full[v_idx % NSTAGE], (v_idx / NSTAGE) & 1);
+                    if (ok) ok = wait(&bars->p_full[0][buf], (gb >> 1) & 1);
+                    // the first PV of a part overwrites O: the previous part's epilogue must have read it
+                    if (ok && jj == 0 && part_idx > 0) ok = wait(&bars->o_free, (part_idx - 1) & 1);
+                    if (!ok) break;
+                    TRACE(2, 1);
+                    tc::tcgen05_fence_after();
+                    issue_pv(0, buf, v_idx % NSTAGE, jj > 0);
+                    TRACE(2, 2);
+                    ok = wait(&bars->p_full[1][buf], (gb >> 1) & 1);
+                    if (!ok) break;
+                    TRACE(2, 3);
+                    tc::tcgen05_fence_after();
+                    issue_pv(1, buf, v_idx % NSTAGE, jj > 0);
+                    tc::umma_commit(tc::smem_u32(&bars->pv_done));
+                    tc::umma_commit(tc::smem_u32(&bars->kv_empty[v_idx % NSTAGE]));
+                    if (has_k) {
+                        ok = wait(&bars->kv_full[k_idx % NSTAGE], (k_idx / NSTAGE) & 1);
+                        if (!ok) break;
+                        issue_qk(buf, k_idx % NSTAGE);       // S of block j+2 into the buffer the PVs just read
+                        tc::umma_commit(tc::smem_u32(&bars->s_full[buf]));
+                        tc::umma_commit(tc::smem_u32(&bars->kv_empty[k_idx % NSTAGE]));
                     }
+                    TRACE(2, 4);
+                    TRACE_NEXT();
+                    cons += has_k ? 2 : 1;
                 }
-                if (ok && jj + 2 < cnt) {
-                    issue_qk(gb & 1, k_idx % NSTAGE);
-                    tc::umma_commit(tc::smem_u32(&bars->s_full[tt][gb & 1]), elect);
-                }
-                if (!ok) break;
-                tc::umma_commit(tc::smem_u32(&bars->kv_empty[v_idx % NSTAGE]), elect);
-                if (has_k) tc::umma_commit(tc::smem_u32(&bars->kv_empty[k_idx % NSTAGE]), elect);
-                cons += has_k ? 2 : 1;
+                // the softmax warpgroups must have seen the previous part's o_done before this part's is
+                // committed (a waiter may lag one mbarrier phase, never two)
+                if (ok && part_idx > 0) ok = wait(&bars->o_free, (part_idx - 1) & 1);
+                if (ok) tc::umma_commit(tc::smem_u32(&bars->o_done));
+                g += n;
+                ++part_idx;
             }
-            // this tile's softmax warpgroup must have seen the previous part's o_done before this part's is
-            // committed (a waiter may lag one mbarrier phase, never two)
-            if (ok && part_idx > 0) ok = wait(&bars->o_free[tt], (part_idx - 1) & 1);
-            if (ok) tc::umma_commit(tc::smem_u32(&bars->o_done), elect);
-            g += cnt;
-            ++part_idx;
         }
-        }
-    mma_done:;
     } else {
         // ================================ softmax + epilogue ================================
-        const int tt = warp >> 2;                          // tile of this warpgroup
-        const int r = (warp & 3) * 32 + lane;              // row inside the tile == TMEM lane
+        const int w = warp >> 2;                           // warpgroup: key half of every block
+        const int r = (warp & 3) * 32 + lane;              // query row inside the tile == TMEM lane
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t o_tmem = tmem + 256 + tt * 128 + lane_addr;
-        int g = 0;                                         // blocks of this tile processed so far
+        const uint32_t o_own = tmem + 256 + w * 128 + lane_addr;
+        int g = 0;                                         // blocks processed so far
         bool ok = true;
         while (it.next(part)) {
-            const int row0 = (2 * part.pair + tt) * BQ;
-            const int my_n = tt ? part.cnt1 : part.cnt0;
             const int n_part = part.j1 - part.j0;
-            const int diag0 = nhb + row0 / BK;             // the two KV blocks that cross the causal diagonal
+            const int diag_block = nhb + part.qt;          // KV block index of the causal diagonal
             float m_ref = -INFINITY, l_sum = 0.f;
 
-            for (int jj = 0; jj < my_n && ok; ++jj, ++g) {
+            for (int jj = 0; jj < n_part && ok; ++jj, ++g) {
                 const int j = part.j0 + jj;
                 const int buf = g & 1;
-                const uint32_t s_tmem = tmem + tt * 128 + buf * 64 + lane_addr;
-                ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&bars->s_full[tt][buf]), (g >> 1) & 1, abort_flag));
+                const uint32_t s_tmem = tmem + buf * 128 + w * HK + lane_addr;
+                ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&bars->s_full[buf]), (g >> 1) & 1, abort_flag));
                 tc::tcgen05_fence_after();
+                if ((warp & 3) == 0) TRACE(w, 0);
                 uint32_t sa[32], sb[32];
                 tc::tmem_ld32(s_tmem, sa);
                 tc::tmem_ld32(s_tmem + 32, sb);
                 tc::tmem_wait_ld();
 
-                // masking: ragged history tail, the two blocks on the causal diagonal
-                int n_valid = BK;
-                if (j == nhb - 1 && tail_partial) n_valid = hist_tail;
-                if (j == diag0) n_valid = min(BK, r + 1);
-                if (j == diag0 + 1) n_valid = r - (BK - 1);               // <= 0: the row sees nothing of this block
-                if (n_valid < BK) {
+                // masking of this warpgroup's 64 keys: ragged history tail, causal diagonal
+                int n_valid = HK;
+                if (j == nhb - 1 && tail_partial) n_valid = hist_tail - w * HK;
+                if (j == diag_block) n_valid = r + 1 - w * HK;             // <= 0: the row sees nothing of this half
+                if (n_valid < HK) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
                         if (i >= n_valid) sa[i] = 0xff800000u;           // -inf
@@ -378,6 +375,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     mx3 = fmaxf(mx3, fmaxf(__uint_as_float(sa[i + 3]), __uint_as_float(sb[i + 3])));
                 }
                 const float bm = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                if ((warp & 3) == 0) TRACE(w, 1);
 
                 float alpha = 1.f;
                 bool need = false;
@@ -405,93 +403,104 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     rs0 += __uint_as_float(pk[i] << 16) + __uint_as_float(pk[i] & 0xffff0000u);
                     rs1 += __uint_as_float(pk[16 + i] << 16) + __uint_as_float(pk[16 + i] & 0xffff0000u);
                 }
-                tc::tmem_st32(s_tmem, pk);                   // P over the first 32 columns of the S buffer
-                // O_t is touched only after the PV of the previous block has completed (it has, by now, nearly always)
+                tc::tmem_st32(s_tmem, pk);                   // P over the first 32 columns of this half of the S buffer
+                if ((warp & 3) == 0) TRACE(w, 2);
+                // O is touched only after the PVs of the previous block have completed (they have, by now, nearly always)
                 if (jj > 0)
-                    ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&bars->pv_done[tt]), (g - 1) & 1, abort_flag));
+                    ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&bars->pv_done), (g - 1) & 1, abort_flag));
                 if (__any_sync(0xffffffffu, need)) {
                     tc::tcgen05_fence_after();
                     l_sum *= alpha;
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         uint32_t ov[32];
-                        tc::tmem_ld32(o_tmem + c * 32, ov);
+                        tc::tmem_ld32(o_own + c * 32, ov);
                         tc::tmem_wait_ld();
 #pragma unroll
                         for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
-                        tc::tmem_st32(o_tmem + c * 32, ov);
+                        tc::tmem_st32(o_own + c * 32, ov);
                     }
                 }
                 l_sum += rs0 + rs1;
+                if ((warp & 3) == 0) TRACE(w, 3);
 
                 if (tail_partial && j == nhb - 1) {
-                    // rows of the V tile past the end of the history may hold anything: zero them (each tile's
-                    // warpgroup does it before it releases its own PV; the two MMA warps do not wait on each other)
+                    // rows of the V tile past the end of the history may hold anything: this warpgroup zeroes
+                    // the ones among its own 64 keys before it releases its PV
                     const int v_idx = kv_base + pos_v(jj, n_part), v_stage = v_idx % NSTAGE;
                     ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&bars->kv_full[v_stage]), (v_idx / NSTAGE) & 1, abort_flag));
-                    if (r >= hist_tail && r < BK) {
-                        uint8_t* vt = smem_gen + 2 * Q_TILE_BYTES + v_stage * KV_TILE_BYTES + r * 128;
-                        uint4* row_a = reinterpret_cast<uint4*>(vt);
-                        uint4* row_b = reinterpret_cast<uint4*>(vt + KV_HALF_BYTES);
+                    const int key = w * HK + (r & (HK - 1));             // two threads per key row: each takes one 64-dim half
+                    if (key >= hist_tail) {
+                        uint4* row_v = reinterpret_cast<uint4*>(smem_gen + KV_OFF + v_stage * TILE_BYTES + (r >> 6) * HALF_BYTES + key * 128);
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) { row_a[i] = make_uint4(0, 0, 0, 0); row_b[i] = make_uint4(0, 0, 0, 0); }
+                        for (int i = 0; i < 8; ++i) row_v[i] = make_uint4(0, 0, 0, 0);
                     }
                     tc::fence_proxy_async_smem();
                 }
                 tc::tmem_wait_st();
                 tc::tcgen05_fence_before();
-                tc::mbar_arrive(tc::smem_u32(&bars->p_full[tt][buf]));
+                tc::mbar_arrive(tc::smem_u32(&bars->p_full[w][buf]));
+                if ((warp & 3) == 0) { TRACE(w, 4); TRACE_NEXT(); }
             }
 
-            const int row = row0 + r;
-            const size_t pslot = ((size_t)blockIdx.x * 2 + part.slot) * 2 + tt;
+            // ---- end of the part: merge the two warpgroups' streams, write the output or the partial -------
             ok = __all_sync(0xffffffffu, ok && tc::mbar_wait(tc::smem_u32(&bars->o_done), part_idx & 1, abort_flag));
-            if (my_n > 0) {
-                tc::tcgen05_fence_after();
-                const float inv = part.final_ ? 1.f / l_sum : 1.f;
+            tc::tcgen05_fence_after();
+            xch[w * BQ + r] = make_float2(m_ref, l_sum);
+            named_barrier_256(1);
+            const float2 other = xch[(w ^ 1) * BQ + r];
+            const float M = fmaxf(m_ref, other.x);
+            const float w_own = l_sum > 0.f ? tc::ex2_approx((m_ref - M) * p.scale_log2) : 0.f;
+            const float w_oth = other.y > 0.f ? tc::ex2_approx((other.x - M) * p.scale_log2) : 0.f;
+            const float L = w_own * l_sum + w_oth * other.y;
+            const float inv = part.final_ ? 1.f / L : 1.f;
+            const uint32_t o_oth = tmem + 256 + (w ^ 1) * 128 + lane_addr;
+            const int row = part.qt * BQ + r;
+            const size_t pslot = (size_t)blockIdx.x * 2 + part.slot;
+            // this warpgroup writes output columns [64 w, 64 w + 64)
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t ov[32];
-                    tc::tmem_ld32(o_tmem + c * 32, ov);
-                    tc::tmem_wait_ld();
-                    if (!ok) continue;
-                    if (!part.final_) {
-                        float4* dst = reinterpret_cast<float4*>(p.part_o + (pslot * BQ + r) * HD + c * 32);
+            for (int c = 0; c < 2; ++c) {
+                uint32_t oa[32], ob[32];
+                tc::tmem_ld32(o_own + w * 64 + c * 32, oa);
+                tc::tmem_ld32(o_oth + w * 64 + c * 32, ob);
+                tc::tmem_wait_ld();
+                if (!ok) continue;
+                float v[32];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            dst[i] = make_float4(__uint_as_float(ov[4 * i]), __uint_as_float(ov[4 * i + 1]),
-                                                 __uint_as_float(ov[4 * i + 2]), __uint_as_float(ov[4 * i + 3]));
-                    } else if (row < p.t) {
-                        const size_t off = ((size_t)row * p.h_q + part.head) * HD + c * 32;
-                        if (p.out_dtype == OMNI_DTYPE_FP32) {
-                            float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o_out) + off);
+                for (int i = 0; i < 32; ++i) {
+                    // a stream that saw no key contributes nothing (its accumulator may hold anything)
+                    const float va = w_own > 0.f ? w_own * __uint_as_float(oa[i]) : 0.f;
+                    const float vb = w_oth > 0.f ? w_oth * __uint_as_float(ob[i]) : 0.f;
+                    v[i] = (va + vb) * inv;
+                }
+                const int col = w * 64 + c * 32;
+                if (!part.final_) {
+                    float4* dst = reinterpret_cast<float4*>(p.part_o + (pslot * BQ + r) * HD + col);
 #pragma unroll
-                            for (int i = 0; i < 8; ++i)
-                                dst[i] = make_float4(__uint_as_float(ov[4 * i]) * inv, __uint_as_float(ov[4 * i + 1]) * inv,
-                                                     __uint_as_float(ov[4 * i + 2]) * inv, __uint_as_float(ov[4 * i + 3]) * inv);
-                        } else {
-                            uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.o_out) + off);
+                    for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                } else if (row < p.t) {
+                    const size_t off = ((size_t)row * p.h_q + part.head) * HD + col;
+                    if (p.out_dtype == OMNI_DTYPE_FP32) {
+                        float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o_out) + off);
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                uint4 v;
-                                v.x = tc::pack_bf16x2(__uint_as_float(ov[8 * i]) * inv, __uint_as_float(ov[8 * i + 1]) * inv);
-                                v.y = tc::pack_bf16x2(__uint_as_float(ov[8 * i + 2]) * inv, __uint_as_float(ov[8 * i + 3]) * inv);
-                                v.z = tc::pack_bf16x2(__uint_as_float(ov[8 * i + 4]) * inv, __uint_as_float(ov[8 * i + 5]) * inv);
-                                v.w = tc::pack_bf16x2(__uint_as_float(ov[8 * i + 6]) * inv, __uint_as_float(ov[8 * i + 7]) * inv);
-                                dst[i] = v;
-                            }
-                        }
+                        for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                    } else {
+                        uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.o_out) + off);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            dst[i] = make_uint4(tc::pack_bf16x2(v[8 * i], v[8 * i + 1]), tc::pack_bf16x2(v[8 * i + 2], v[8 * i + 3]),
+                                                tc::pack_bf16x2(v[8 * i + 4], v[8 * i + 5]), tc::pack_bf16x2(v[8 * i + 6], v[8 * i + 7]));
                     }
                 }
-                if (ok && !part.final_) p.part_ml[pslot * BQ + r] = make_float2(m_ref, l_sum);
-                if (ok && part.final_ && p.lse_out && row < p.t)
-                    p.lse_out[(size_t)row * p.h_q + part.head] = m_ref * p.scale + logf(l_sum);
-            } else if (!part.final_) {
-                p.part_ml[pslot * BQ + r] = make_float2(-INFINITY, 0.f);        // no block of this tile in the part
             }
-            // O_t (and the part's Q tile) may be reused
+            if (ok && w == 0) {
+                if (!part.final_) p.part_ml[pslot * BQ + r] = make_float2(M, L);
+                else if (p.lse_out && row < p.t) p.lse_out[(size_t)row * p.h_q + part.head] = M * p.scale + logf(L);
+            }
+            // O (and the part's Q tile) may be reused; the exchange buffer too, once both warpgroups are here
             tc::tcgen05_fence_before();
-            tc::mbar_arrive(tc::smem_u32(&bars->o_free[tt]));
+            tc::mbar_arrive(tc::smem_u32(&bars->o_free));
+            named_barrier_256(2);
             kv_base += 2 * n_part;
             ++part_idx;
         }
@@ -499,6 +508,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
     tc::tcgen05_fence_before();
     __syncthreads();
+#ifdef ATT_TRACE
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        const long long t0 = trace_buf[(2 * TRACE_N + 8) * 6];
+        for (int role = 0; role < 3; ++role)
+            for (int i = 8; i < TRACE_N; ++i) {
+                const long long* e = trace_buf + (role * TRACE_N + i) * 6;
+                printf("role %d blk %d : %lld %lld %lld %lld %lld\n", role, i, e[0] - t0, e[1] - t0, e[2] - t0, e[3] - t0, e[4] - t0);
+            }
+    }
+#endif
     if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, OMNI_DEV_TIMEOUT);
     if (warp == 8) {
         tc::tcgen05_fence_after();
@@ -506,22 +525,22 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
 }
 
-// Merge the partial outputs of every item that was cut between CTAs.  Grid (items, 8 groups of 32 rows);
+// Merge the partial outputs of every item that was cut between CTAs.  Grid (items, 4 groups of 32 rows);
 // a warp owns 4 rows and a lane 4 of a row's 128 columns.  Shared memory: one int per CTA of the main kernel.
 constexpr int MERGE_BATCH = 4;
 __global__ void __launch_bounds__(256) attention_merge_kernel(const AttnParams p, int n_cta) {
     extern __shared__ int s_slot[];                          // partial slot of every part of the item
     __shared__ int s_n;
-    const int pair = p.n_pairs - 1 - blockIdx.x / p.h_q;
+    const int qt = p.n_tiles - 1 - blockIdx.x / p.h_q;
     const int head = blockIdx.x % p.h_q;
     if (threadIdx.x == 0) {
         int n_hist = p.n_hist_dev ? *p.n_hist_dev : p.n_hist_max;
         n_hist = max(0, min(n_hist, p.n_hist_max));
         Sched s;
-        s.nhb = (n_hist + BK - 1) / BK; s.n_pairs = p.n_pairs; s.h_q = p.h_q; s.t = p.t;
+        s.nhb = (n_hist + BK - 1) / BK; s.n_tiles = p.n_tiles; s.h_q = p.h_q;
         const long long total = s.total();
-        const long long w0 = s.item_begin(pair, head);
-        const int nb = s.nb_pair(pair);
+        const long long w0 = s.item_begin(qt, head);
+        const int nb = s.nb_item(qt);
         auto cta_of = [&](long long w) {
             int b = (int)(w * n_cta / total);
             b = max(0, min(b, n_cta - 1));
@@ -542,13 +561,12 @@ __global__ void __launch_bounds__(256) attention_merge_kernel(const AttnParams p
     if (n_parts == 0) return;                                // the item was computed by one CTA
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int q4 = 0; q4 < 4; ++q4) {
-        const int rr = blockIdx.y * 32 + warp * 4 + q4;      // 0..255: tile * 128 + row
-        const int tt = rr / BQ, r = rr % BQ;
-        const int row = (2 * pair + tt) * BQ + r;
+        const int r = blockIdx.y * 32 + warp * 4 + q4;       // row of the tile
+        const int row = qt * BQ + r;
         if (row >= p.t) continue;
         float M = -INFINITY;
         for (int i = 0; i < n_parts; ++i) {
-            const float2 ml = p.part_ml[((size_t)s_slot[i] * 2 + tt) * BQ + r];
+            const float2 ml = p.part_ml[(size_t)s_slot[i] * BQ + r];
             if (ml.y > 0.f) M = fmaxf(M, ml.x);
         }
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -561,7 +579,7 @@ __global__ void __launch_bounds__(256) attention_merge_kernel(const AttnParams p
                 ml[i] = make_float2(-INFINITY, 0.f);
                 o[i] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (i0 + i < n_parts) {
-                    const size_t pslot = (size_t)s_slot[i0 + i] * 2 + tt;
+                    const size_t pslot = (size_t)s_slot[i0 + i];
                     ml[i] = p.part_ml[pslot * BQ + r];
                     if (ml[i].y > 0.f) o[i] = *reinterpret_cast<const float4*>(p.part_o + (pslot * BQ + r) * HD + lane * 4);
                 }
@@ -608,11 +626,11 @@ omni_status omni_attention_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q,
     p.t = t; p.h_q = g.h_q; p.h_kv = g.h_kv; p.n_hist_dev = n_hist_dev; p.n_hist_max = n_hist_max;
     p.scale = scale; p.scale_log2 = scale * 1.4426950408889634f;
     p.o_out = o_out; p.out_dtype = out_dtype; p.lse_out = lse_out; p.status = ctx->status_dev;
-    p.n_pairs = (t + 2 * BQ - 1) / (2 * BQ);
-    // one CTA per SM, fewer when the whole job is small (at least 8 block steps per CTA)
-    long long w_max = 0;
-    for (int pr = 0; pr < p.n_pairs; ++pr) w_max += (long long)g.h_q * ((n_hist_max + BK - 1) / BK + 4 * pr + 4);
-    const int n_cta = (int)std::max(1ll, std::min((long long)ctx->sm_count, w_max / 8));
+    p.n_tiles = (t + BQ - 1) / BQ;
+    // one CTA per SM, fewer when the whole job is small (at least 4 block steps per CTA)
+    const long long nhb_max = (n_hist_max + BK - 1) / BK;
+    const long long w_max = (long long)g.h_q * ((long long)p.n_tiles * (nhb_max + 1) + (long long)p.n_tiles * (p.n_tiles - 1) / 2);
+    const int n_cta = (int)std::max(1ll, std::min((long long)ctx->sm_count, w_max / 4));
     p.part_o = ctx->attn_part_o; p.part_ml = reinterpret_cast<float2*>(ctx->attn_part_ml);
     static bool attr_set = false;
     if (!attr_set) {
@@ -621,7 +639,7 @@ omni_status omni_attention_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q,
     }
     attention_tc_kernel<<<n_cta, ATT_THREADS, SMEM_BYTES, st>>>(tm_q, tm_kh, tm_vh, tm_kc, tm_vc, p);
     OMNI_CHECK_LAUNCH(ctx, "attention_tc_kernel");
-    attention_merge_kernel<<<dim3(p.n_pairs * g.h_q, 8), 256, (n_cta + 1) * sizeof(int), st>>>(p, n_cta);
+    attention_merge_kernel<<<dim3(p.n_tiles * g.h_q, 4), 256, (n_cta + 1) * sizeof(int), st>>>(p, n_cta);
     OMNI_CHECK_LAUNCH(ctx, "attention_merge_kernel");
     return OMNI_OK;
 }
