@@ -8,10 +8,12 @@
 // un-normalised partial outputs with their (max, sum) in scratch and a small second kernel merges them.
 //
 // Inside a CTA:
-//   warp 9      TMA producer: the part's Q tile, then K / V tiles (128 keys) through a 5-stage ring
-//   warp 8      one thread issues tcgen05.mma.  S = Q K_j^T is one N = 128 instruction group (an M = 128
-//               instruction occupies the tensor pipe for 64 clocks whatever N <= 128 is, so narrower
-//               blocks would waste it); S is double-buffered and runs two blocks ahead of PV.
+//   warp 10     TMA producer: the part's Q tile, then K / V tiles (128 keys) through a 5-stage ring
+//   warp 8      one thread issues S = Q K_j^T as one N = 128 instruction group (an M = 128 tcgen05.mma
+//               occupies the tensor pipe for 64 clocks whatever N <= 128 is, so narrower blocks would waste
+//               it); S is double-buffered and runs two blocks ahead of PV.
+//   warp 9      one thread issues the PVs.  One thread cannot issue faster than one instruction per ~70-100
+//               clocks, so QK and PV have an issuer each; they are ordered by the pv_done barriers.
 //   warps 0-3   softmax warpgroup A: columns 0-63 of every S block (keys 0-63 of the block)
 //   warps 4-7   softmax warpgroup B: columns 64-127.  One thread per query row and half block: logits
 //               from tensor memory, running max with lazy rescale, exp2, P written back over the S columns
@@ -35,7 +37,7 @@ constexpr int HD = 128;                  // head dim
 constexpr int TILE_BYTES = 128 * HD * 2; // 32 KiB (Q, K and V tiles), two 64-column halves of 16 KiB
 constexpr int HALF_BYTES = TILE_BYTES / 2;
 constexpr int NSTAGE = 5;
-constexpr int ATT_THREADS = 320;
+constexpr int ATT_THREADS = 352;
 constexpr int XCH_BYTES = BQ * 2 * 8;    // (max, sum) of both warpgroups, exchanged when a part ends
 constexpr int SMEM_BYTES = TILE_BYTES + NSTAGE * TILE_BYTES + 1024 /*alignment*/ + 512 /*barriers*/ + XCH_BYTES;
 // O is rescaled only when the row max grows by more than this many log2 units (P stays below 2^8).
@@ -71,7 +73,7 @@ struct Barriers {
     uint64_t kv_empty[NSTAGE];
     uint64_t s_full[2];         // [buffer]
     uint64_t p_full[2][2];      // [warpgroup][buffer]
-    uint64_t pv_done;           // one phase per block: both PVs of the block have completed
+    uint64_t pv_done[2];        // [buffer] both PVs of the block in that buffer have completed
     uint64_t o_done;
     uint64_t o_free;            // both warpgroups have read O of the part
     uint32_t tmem_base;
@@ -178,8 +180,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             tc::mbar_init(tc::smem_u32(&bars->p_full[0][b]), 128);
             tc::mbar_init(tc::smem_u32(&bars->p_full[1][b]), 128);
         }
-        tc::mbar_init(tc::smem_u32(&bars->pv_done), 1);
-        tc::mbar_init(tc::smem_u32(&bars->o_done), 1);
+        tc::mbar_init(tc::smem_u32(&bars->pv_done[0]), 1);
+        tc::mbar_init(tc::smem_u32(&bars->pv_done[1]), 1);
+        tc::mbar_init(tc::smem_u32(&bars->o_done), 2);                   // QK issuer and PV issuer
         tc::mbar_init(tc::smem_u32(&bars->o_free), 256);
         bars->abort_flag = 0;
         tc::fence_barrier_init();
@@ -199,7 +202,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     int part_idx = 0;
     int kv_base = 0;                                         // K/V tiles loaded by earlier parts of this CTA
 
-    if (warp == 9) {
+    if (warp == 10) {
         // ================================ TMA producer ================================
         if (lane == 0) {
             tc::tma_prefetch_desc(&tm_q);
@@ -252,19 +255,64 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             }
         }
     } else if (warp == 8) {
-        // ================================ MMA issuer (one thread) ================================
+        // ================================ QK issuer (one thread) ================================
         if (lane == 0) {
             auto wait = [&](uint64_t* bar, int parity) { return tc::mbar_wait(tc::smem_u32(bar), parity, abort_flag); };
-            // S[buf] = Q K^T over the 128 keys of ring stage `stage`
-            auto issue_qk = [&](int buf, int stage) {
-                const uint32_t b0 = kv_smem + stage * TILE_BYTES;
+            // S[buf] = Q K^T over the 128 keys of ring slot idx
+            auto issue_qk = [&](int buf, int idx) {
+                const uint32_t b0 = kv_smem + (idx % NSTAGE) * TILE_BYTES;
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk) {
                     const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
                     tc::umma_ss(tmem + buf * 128, tc::umma_smem_desc(q_smem + off, 16, 1024), tc::umma_smem_desc(b0 + off, 16, 1024),
                                 IDESC_QK, kk > 0, 1u);
                 }
+                tc::umma_commit(tc::smem_u32(&bars->s_full[buf]));
+                tc::umma_commit(tc::smem_u32(&bars->kv_empty[idx % NSTAGE]));
             };
+            int g = 0;                                       // blocks started so far (buffer = g & 1)
+            bool ok = true;
+            while (ok && it.next(part)) {
+                const int n = part.j1 - part.j0;
+                ok = wait(&bars->q_full, part_idx & 1);
+                // S of the first two blocks: K tiles at ring positions 0 and 1 of the part.  Both buffers are
+                // free: every pv_done of the previous part was waited for below.
+                for (int jj = 0; jj < 2 && jj < n && ok; ++jj) {
+                    const int idx = kv_base + jj;
+                    ok = wait(&bars->kv_full[idx % NSTAGE], (idx / NSTAGE) & 1);
+                    if (!ok) break;
+                    tc::tcgen05_fence_after();
+                    issue_qk((g + jj) & 1, idx);
+                }
+                for (int jj = 0; jj < n && ok; ++jj) {
+                    const int gb = g + jj, buf = gb & 1;
+                    TRACE(2, 0);
+                    // the PVs of block j have read P out of the buffer: S of block j+2 may overwrite it
+                    ok = wait(&bars->pv_done[buf], (gb >> 1) & 1);
+                    TRACE(2, 1);
+                    if (ok && jj + 2 < n) {
+                        const int idx = kv_base + 2 * (jj + 2) - 1;          // K_{j+2} in the part's load order
+                        ok = wait(&bars->kv_full[idx % NSTAGE], (idx / NSTAGE) & 1);
+                        if (!ok) break;
+                        tc::tcgen05_fence_after();
+                        issue_qk(buf, idx);
+                    }
+                    TRACE(2, 2); TRACE(2, 3); TRACE(2, 4);
+                    TRACE_NEXT();
+                }
+                // the softmax warpgroups must have seen the previous part's o_done before this part's is
+                // committed (a waiter may lag one mbarrier phase, never two)
+                if (ok && part_idx > 0) ok = wait(&bars->o_free, (part_idx - 1) & 1);
+                if (ok) tc::umma_commit(tc::smem_u32(&bars->o_done));
+                g += n;
+                kv_base += 2 * n;
+                ++part_idx;
+            }
+        }
+    } else if (warp == 9) {
+        // ================================ PV issuer (one thread) ================================
+        if (lane == 0) {
+            auto wait = [&](uint64_t* bar, int parity) { return tc::mbar_wait(tc::smem_u32(bar), parity, abort_flag); };
             // O_w += P_w[buf] V[keys 64w .. 64w+63] of ring stage `stage`
             auto issue_pv = [&](int w, int buf, int stage, bool accumulate) {
                 const uint32_t b0 = kv_smem + stage * TILE_BYTES + w * (HK * 128);
@@ -274,59 +322,31 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                                 tc::umma_smem_desc(b0 + kk * 2048, HALF_BYTES, 1024), IDESC_PV, accumulate || kk > 0, 1u);
                 }
             };
-            int cons = 0;                                    // K/V tiles consumed so far (same order as produced)
-            int g = 0;                                       // blocks started so far (buffer = g & 1)
+            int g = 0;
             bool ok = true;
             while (ok && it.next(part)) {
                 const int n = part.j1 - part.j0;
-                ok = wait(&bars->q_full, part_idx & 1);
-                // S of the first two blocks
-                for (int jj = 0; jj < 2 && jj < n && ok; ++jj) {
-                    ok = wait(&bars->kv_full[cons % NSTAGE], (cons / NSTAGE) & 1);
-                    if (!ok) break;
-                    tc::tcgen05_fence_after();
-                    issue_qk((g + jj) & 1, cons % NSTAGE);
-                    tc::umma_commit(tc::smem_u32(&bars->s_full[(g + jj) & 1]));
-                    tc::umma_commit(tc::smem_u32(&bars->kv_empty[cons % NSTAGE]));
-                    ++cons;
-                }
                 for (int jj = 0; jj < n && ok; ++jj) {
-                    const int v_idx = cons, k_idx = cons + 1;
-                    const bool has_k = jj + 2 < n;
+                    const int v_idx = kv_base + pos_v(jj, n);
                     const int gb = g + jj, buf = gb & 1;
-                    TRACE(2, 0);
                     ok = wait(&bars->kv_full[v_idx % NSTAGE], (v_idx / NSTAGE) & 1);
                     if (ok) ok = wait(&bars->p_full[0][buf], (gb >> 1) & 1);
                     // the first PV of a part overwrites O: the previous part's epilogue must have read it
                     if (ok && jj == 0 && part_idx > 0) ok = wait(&bars->o_free, (part_idx - 1) & 1);
                     if (!ok) break;
-                    TRACE(2, 1);
                     tc::tcgen05_fence_after();
                     issue_pv(0, buf, v_idx % NSTAGE, jj > 0);
-                    TRACE(2, 2);
                     ok = wait(&bars->p_full[1][buf], (gb >> 1) & 1);
                     if (!ok) break;
-                    TRACE(2, 3);
                     tc::tcgen05_fence_after();
                     issue_pv(1, buf, v_idx % NSTAGE, jj > 0);
-                    tc::umma_commit(tc::smem_u32(&bars->pv_done));
+                    tc::umma_commit(tc::smem_u32(&bars->pv_done[buf]));
                     tc::umma_commit(tc::smem_u32(&bars->kv_empty[v_idx % NSTAGE]));
-                    if (has_k) {
-                        ok = wait(&bars->kv_full[k_idx % NSTAGE], (k_idx / NSTAGE) & 1);
-                        if (!ok) break;
-                        issue_qk(buf, k_idx % NSTAGE);       // S of block j+2 into the buffer the PVs just read
-                        tc::umma_commit(tc::smem_u32(&bars->s_full[buf]));
-                        tc::umma_commit(tc::smem_u32(&bars->kv_empty[k_idx % NSTAGE]));
-                    }
-                    TRACE(2, 4);
-                    TRACE_NEXT();
-                    cons += has_k ? 2 : 1;
                 }
-                // the softmax warpgroups must have seen the previous part's o_done before this part's is
-                // committed (a waiter may lag one mbarrier phase, never two)
                 if (ok && part_idx > 0) ok = wait(&bars->o_free, (part_idx - 1) & 1);
                 if (ok) tc::umma_commit(tc::smem_u32(&bars->o_done));
                 g += n;
+                kv_base += 2 * n;
                 ++part_idx;
             }
         }
@@ -407,7 +427,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if ((warp & 3) == 0) TRACE(w, 2);
                 // O is touched only after the PVs of the previous block have completed (they have, by now, nearly always)
                 if (jj > 0)
-                    ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&bars->pv_done), (g - 1) & 1, abort_flag));
+                    ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&bars->pv_done[(g - 1) & 1]), ((g - 1) >> 1) & 1, abort_flag));
                 if (__any_sync(0xffffffffu, need)) {
                     tc::tcgen05_fence_after();
                     l_sum *= alpha;
