@@ -159,6 +159,9 @@ omni_status omnitide_select_units(omnitide_ctx* ctx, void* stream,
  * it holds page_size retained rows (promoted to selected-history), else 2 if partly filled (stays
  * recent-context), else OMNI_PAGE_EMPTY.
  *   slot_map_out [dev] s_span_max int32 (nullable), info_out [dev], page_class_out [dev] nullable.
+ *   keep_mask [dev] is read in aligned 16-byte vectors: the buffer must extend to s_span_max rounded up to a
+ *   multiple of 16 bytes; bytes at and beyond *s_span_dev are ignored.  Calls on one context must not overlap
+ *   (the CTAs of the kernel exchange their counts through context scratch).
  * mode must be OMNI_COMPACT_PACK.
  */
 omni_status omnipage_compact(omnitide_ctx* ctx, void* stream,

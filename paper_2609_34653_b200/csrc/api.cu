@@ -18,7 +18,7 @@ cudaError_t alloc(T** p, size_t n) {
 void free_all(omnitide_ctx* c) {
     void* ptrs[] = {c->status_dev, c->score_part, c->score_tile_mass, c->score_mass64, c->inplace_k, c->inplace_v,
                     c->ws_scores, c->ws_unit_keep, c->ws_keep_mask, c->ws_slot_map, c->ws_counts, c->ws_info, c->st_q,
-                    c->st_k, c->st_v, c->st_o, c->st_units, c->attn_part_o, c->attn_part_ml};
+                    c->st_k, c->st_v, c->st_o, c->st_units, c->attn_part_o, c->attn_part_ml, c->cp_words};
     for (void* p : ptrs)
         if (p) cudaFree(p);
 }
@@ -52,6 +52,8 @@ extern "C" omni_status omnitide_create(omnitide_ctx** ctx_out, const omni_geomet
     ok &= alloc(&c->score_part, row_tiles * ((size_t)g->u_cap + 64) * 128) == cudaSuccess;   // + split boundaries
     ok &= alloc(&c->score_tile_mass, row_tiles * g->u_cap) == cudaSuccess;
     ok &= alloc(&c->score_mass64, (size_t)g->u_cap) == cudaSuccess;
+    ok &= alloc(&c->cp_words, (size_t)c->sm_count + 1) == cudaSuccess;
+    ok = ok && cudaMemset(c->cp_words, 0, ((size_t)c->sm_count + 1) * sizeof(unsigned long long)) == cudaSuccess;
     ok &= alloc(&c->ws_scores, (size_t)g->u_cap) == cudaSuccess;
     ok &= alloc(&c->ws_unit_keep, (size_t)g->u_cap + 16) == cudaSuccess;
     ok &= alloc(&c->ws_keep_mask, (size_t)g->s_cap + 16) == cudaSuccess;

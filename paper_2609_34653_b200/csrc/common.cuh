@@ -25,6 +25,8 @@ struct omnitide_ctx {
     void* inplace_k;              // staging for in-place compaction, allocated on first use
     void* inplace_v;
     size_t inplace_rows;
+    unsigned long long* cp_words; // [SMs] per-CTA count words of the compaction kernel, tagged with cp_epoch
+    uint32_t cp_epoch;            // launches of the compaction kernel on this context so far
     // work buffers of omnitide_chunk_step
     float* ws_scores;             // [u_cap]
     uint8_t* ws_unit_keep;        // [u_cap]

@@ -1,19 +1,24 @@
 // OmniPage eager compaction (mode PACK) and the append step.
 //
-// One persistent kernel does the whole compaction: every CTA scans the keep mask (a few tens of
-// KB, served from L2) into per-chunk prefix counts held in shared memory, so no CTA waits on
-// another; the retained rows are then split evenly by DESTINATION slot across the CTAs, each
-// of which rebuilds the source slots of its share from the mask and moves the rows with 16-byte
-// vector loads/stores, eight in flight per thread.  The slot map, page classes and the integer
-// summary come out of the same scan.  HBM traffic is one read and one write per retained row.
+// One kernel, one CTA per SM, does the whole compaction.  The keep mask is cut into one part per
+// CTA; a CTA counts its own part (one 16-byte vector per lane, kept in registers), publishes the
+// count in global memory and waits (bounded) until all CTAs have arrived: the launch is cooperative,
+// so all CTAs are resident.  Each CTA then gathers the per-part counts, scans them, takes an equal
+// share of the DESTINATION rows, rebuilds the source slots of that share from the mask parts that
+// hold them and streams the rows HBM -> shared memory -> HBM with bulk asynchronous copies issued
+// by one lane per warp (no per-vector instructions).  The slot map, the page classes and the integer
+// summary come out of the same pass.  HBM traffic is one read and one write per retained row; the
+// mask is read about once in total (every CTA reading all of it cost 4 us of L2 time).
 #include "common.cuh"
+#include "tc_ptx.cuh"
+
+#include <algorithm>
 
 namespace {
 
+
 constexpr int CP_THREADS = 512;
 constexpr int CP_WARPS = CP_THREADS / 32;
-constexpr int CP_UNROLL = 8;
-constexpr int CP_MAX_CHUNKS = 2048;
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
     uint4 v;
@@ -86,140 +91,309 @@ __device__ int block_excl_scan(int* data, int n, int* warp_tot /*[CP_WARPS+1]*/)
 struct CompactArgs {
     const char* k_src; const char* v_src; char* k_dst; char* v_dst;
     const uint8_t* mask; const int32_t* s_span_dev; int s_span_max;
-    int page_size; int row_bytes; int vpr; int vpr_shift; int chunk_shift;
+    int page_size; int row_bytes; int vpr; int vpr_shift;
     const omni_unit* units_kept; const int32_t* n_units_kept_dev; int n_units_max;
     int32_t* slot_map; omni_compact_info* info; uint8_t* page_class; int32_t* status;
     int rows_cap;      // capacity of the per-CTA source list
+    int max_chunks;    // capacity of the chunk-prefix array
+    int n_slots;       // row buffers per warp for the bulk-copy path (0: move rows with vector loads/stores)
+    int part_groups;   // 512-byte mask groups per CTA
+    unsigned long long* words;   // [0]: arrival counter (low half, never reset); [1 + i]: (epoch << 32) | retained count of part i
+    uint32_t epoch;
 };
 
-__global__ void __launch_bounds__(CP_THREADS, 1) compact_pack_kernel(const CompactArgs a) {
-    extern __shared__ int smem_i[];
-    int* prefix = smem_i;                                   // [n_chunks + 1]
-    __shared__ int warp_tot[CP_WARPS + 1];
-    __shared__ int s_misc[4];
-    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+constexpr int CP_BATCH = 16;        // 16-byte vectors in flight per thread (vector path)
+constexpr int CP_MAX_SLOTS = 4;     // more rows in flight per warp than this measured slower
 
-    int s = a.s_span_dev ? *a.s_span_dev : a.s_span_max;
+// zeroes the bytes of v at and beyond `valid` (any int: <= 0 clears all, >= 16 keeps all)
+__device__ __forceinline__ uint32_t clip_word(uint32_t w, int nv) {
+    return nv >= 4 ? w : (nv <= 0 ? 0u : (w & ((1u << (8 * nv)) - 1u)));
+}
+__device__ __forceinline__ uint4 clip_vec(uint4 v, int valid) {
+    v.x = clip_word(v.x, valid); v.y = clip_word(v.y, valid - 4);
+    v.z = clip_word(v.z, valid - 8); v.w = clip_word(v.w, valid - 12);
+    return v;
+}
+__device__ __forceinline__ uint32_t byte_at(const uint4& v, int b) {      // b is a compile-time constant after unrolling
+    const uint32_t w = b < 4 ? v.x : (b < 8 ? v.y : (b < 12 ? v.z : v.w));
+    return (w >> ((b & 3) * 8)) & 0xffu;
+}
+__device__ __forceinline__ int count_kept(const uint4& v) {
+    return nonzero_bytes(v.x) + nonzero_bytes(v.y) + nonzero_bytes(v.z) + nonzero_bytes(v.w);
+}
+// index of the first zero byte of v, 16 if there is none
+__device__ __forceinline__ int first_zero_byte(const uint4& v) {
+    const uint32_t zx = __vcmpeq4(v.x, 0u), zy = __vcmpeq4(v.y, 0u), zz = __vcmpeq4(v.z, 0u), zw = __vcmpeq4(v.w, 0u);
+    int z = 16;
+    if (zw) z = 12 + ((__ffs(zw) - 1) >> 3);
+    if (zz) z = 8 + ((__ffs(zz) - 1) >> 3);
+    if (zy) z = 4 + ((__ffs(zy) - 1) >> 3);
+    if (zx) z = (__ffs(zx) - 1) >> 3;
+    return z;
+}
+__device__ __forceinline__ uint4 ld_mask(const uint8_t* mask, int vec) {
+    return __ldg(reinterpret_cast<const uint4*>(mask) + vec);
+}
+
+// A warp holds the 512 mask bytes that start at `base` (16 per lane, v); `run` = retained slots before them.
+// Writes the source slots of the destinations in [d0, d0 + n_rows) that fall in this group.
+__device__ __forceinline__ void emit_sources(const uint4& v, int base, int run, int lane, int d0, int n_rows,
+                                             int* src_list) {
+    const int cnt = count_kept(v);
+    int tot;
+    int r = run + warp_excl_scan(cnt, lane, tot) - d0;
+    if (cnt && r < n_rows && r + cnt > 0) {
+        const int pos = base + lane * 16;
+#pragma unroll
+        for (int b = 0; b < 16; ++b)
+            if (byte_at(v, b)) {
+                if (r >= 0 && r < n_rows) src_list[r] = pos + b;
+                ++r;
+            }
+    }
+}
+// Same group: writes slot_map for the slots below s.
+__device__ __forceinline__ void emit_slot_map(const uint4& v, int base, int run, int lane, int s, int32_t* slot_map) {
+    const int cnt = count_kept(v);
+    int tot;
+    int r = run + warp_excl_scan(cnt, lane, tot);
+    const int pos = base + lane * 16;
+    int o[16];
+#pragma unroll
+    for (int b = 0; b < 16; ++b) {
+        const bool kept = byte_at(v, b) != 0;
+        o[b] = kept ? r : -1;
+        r += kept;
+    }
+    if (pos + 16 <= s) {
+        int4* o4 = reinterpret_cast<int4*>(slot_map + pos);
+        o4[0] = make_int4(o[0], o[1], o[2], o[3]);
+        o4[1] = make_int4(o[4], o[5], o[6], o[7]);
+        o4[2] = make_int4(o[8], o[9], o[10], o[11]);
+        o4[3] = make_int4(o[12], o[13], o[14], o[15]);
+    } else {
+#pragma unroll
+        for (int b = 0; b < 16; ++b)
+            if (pos + b < s) slot_map[pos + b] = o[b];
+    }
+}
+
+__device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void* gsrc, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_dst), "l"(gsrc), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* gdst, uint32_t smem_src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_src), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+
+
+__device__ __forceinline__ void st_relaxed_gpu(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long ld_relaxed_gpu(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// 16 mask bytes at slot `pos` (a multiple of 16) with the bytes at and beyond s zeroed
+__device__ __forceinline__ uint4 mask_at(const uint8_t* mask, int pos, int s) {
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (pos < s) v = clip_vec(ld_mask(mask, pos >> 4), s - pos);
+    return v;
+}
+
+// The mask is cut into gridDim.x parts of `part_groups` groups of 512 bytes; CTA i counts part i alone and
+// publishes the count in words[i] tagged with the epoch of this launch; every CTA then gathers all the
+// counts (the only cross-CTA step: all CTAs are resident, one per SM, and the wait is bounded).
+__global__ void __launch_bounds__(CP_THREADS, 1) compact_pack_kernel(const CompactArgs a) {
+    extern __shared__ __align__(128) int smem_i[];
+    int* prefix = smem_i;                                   // [max_chunks]: part counts, then their exclusive scan
+    int* src_list = smem_i + a.max_chunks;                  // [rows_cap]
+    char* rowbuf = reinterpret_cast<char*>(smem_i + a.max_chunks + a.rows_cap);   // row buffers of the bulk-copy path
+    __shared__ int warp_tot[CP_WARPS + 1];
+    __shared__ int wcnt[CP_WARPS];
+    __shared__ int s_misc[4];
+    __shared__ uint64_t cbar[CP_WARPS][CP_MAX_SLOTS];
+    __shared__ int abort_flag;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int G = gridDim.x;
+
+    // ---- prologue: every load whose address needs no device-side count is issued before anything waits ----
+    const int part_bytes = a.part_groups * 512;
+    const int my_base = blockIdx.x * part_bytes;
+    const int gpw = (a.part_groups + CP_WARPS - 1) / CP_WARPS;        // groups per warp (contiguous)
+    const int wg0 = wid * gpw, wg1 = min(a.part_groups, wg0 + gpw);   // this warp's groups of the part
+    uint4 mv = make_uint4(0, 0, 0, 0);                                // its first group stays in registers
+    if (wg0 < wg1 && my_base + wg0 * 512 + lane * 16 < a.s_span_max) mv = ld_mask(a.mask, (my_base + wg0 * 512) / 16 + lane);
+    int s = a.s_span_dev ? __ldg(a.s_span_dev) : a.s_span_max;
+    int nu = 0, u_len = 0, u_group = -1;
+    if (a.units_kept) {
+        nu = a.n_units_kept_dev ? __ldg(a.n_units_kept_dev) : a.n_units_max;
+        if (tid < a.n_units_max) { u_len = __ldg(&a.units_kept[tid].len); u_group = __ldg(&a.units_kept[tid].group); }
+    }
+    for (int c = tid; c < a.max_chunks; c += CP_THREADS) prefix[c] = 0;
+    if (tid == 0) { s_misc[0] = 0; s_misc[1] = 0; s_misc[2] = G; abort_flag = 0; }
+    if (lane == 0 && a.n_slots > 0) {
+        for (int q = 0; q < a.n_slots; ++q) tc::mbar_init(tc::smem_u32(&cbar[wid][q]), 1);
+        tc::fence_barrier_init();
+    }
     if (s > a.s_span_max || s < 0) {
         if (tid == 0 && blockIdx.x == 0) atomicOr(a.status, OMNI_DEV_BAD_COUNT);
         s = max(0, min(s, a.s_span_max));
     }
-    const int chunk_bytes = 1 << a.chunk_shift;
-    const int n_chunks = (s + chunk_bytes - 1) >> a.chunk_shift;
-    int* src_list = smem_i + (((a.s_span_max + chunk_bytes - 1) >> a.chunk_shift) + 2);
-    const int vec_per_lane = chunk_bytes >> 9;              // 16-byte vectors per lane per chunk
+    nu = max(0, min(nu, a.n_units_max));
 
-    // ---- phase A: every CTA counts every chunk -------------------------------------------
-    for (int c = wid; c < n_chunks; c += CP_WARPS) {
-        int cnt = 0;
-        const int base = c << a.chunk_shift;
-        for (int k = 0; k < vec_per_lane; ++k) {
-            uint4 v = load_mask16(a.mask, base + k * 512 + lane * 16, s);
-            cnt += nonzero_bytes(v.x) + nonzero_bytes(v.y) + nonzero_bytes(v.z) + nonzero_bytes(v.w);
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-        if (lane == 0) prefix[c] = cnt;
+    // ---- phase A: count the own part, publish, gather all parts ------------------------------------------
+    mv = clip_vec(mv, s - (my_base + wg0 * 512 + lane * 16));
+    {
+        int cnt = count_kept(mv);
+        for (int g = wg0 + 1; g < wg1; ++g) cnt += count_kept(mask_at(a.mask, my_base + g * 512 + lane * 16, s));
+        cnt = __reduce_add_sync(0xffffffffu, cnt);
+        if (lane == 0) wcnt[wid] = cnt;
+    }
+    // partitions from the compacted unit table
+    int p0 = 0, p1 = 0;
+    for (int u = tid; u < nu; u += CP_THREADS) {
+        if (u >= CP_THREADS) { u_len = a.units_kept[u].len; u_group = a.units_kept[u].group; }
+        if (u_group == OMNI_GROUP_MUST_KEEP) p0 += u_len;
+        else if (u_group == OMNI_GROUP_SELECTED) p1 += u_len;
     }
     __syncthreads();
-    const int n_kept = block_excl_scan(prefix, n_chunks, warp_tot);
-
-    // ---- partitions from the compacted unit table -----------------------------------------
-    int n0 = 0, n1 = 0;
     if (a.units_kept) {
-        int nu = a.n_units_kept_dev ? *a.n_units_kept_dev : a.n_units_max;
-        nu = max(0, min(nu, a.n_units_max));
-        int p0 = 0, p1 = 0;
-        for (int u = tid; u < nu; u += CP_THREADS) {
-            const omni_unit un = a.units_kept[u];
-            if (un.group == OMNI_GROUP_MUST_KEEP) p0 += un.len;
-            else if (un.group == OMNI_GROUP_SELECTED) p1 += un.len;
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            p0 += __shfl_xor_sync(0xffffffffu, p0, o);
-            p1 += __shfl_xor_sync(0xffffffffu, p1, o);
-        }
-        if (tid == 0) { s_misc[0] = 0; s_misc[1] = 0; }
-        __syncthreads();
-        if (lane == 0) { atomicAdd(&s_misc[0], p0); atomicAdd(&s_misc[1], p1); }
-        __syncthreads();
-        n0 = s_misc[0];
-        n1 = s_misc[1];
+        p0 = __reduce_add_sync(0xffffffffu, p0);
+        p1 = __reduce_add_sync(0xffffffffu, p1);
+        if (lane == 0 && (p0 | p1)) { atomicAdd(&s_misc[0], p0); atomicAdd(&s_misc[1], p1); }
     }
+    if (tid == 0) {
+        int tot = 0;
+#pragma unroll
+        for (int w = 0; w < CP_WARPS; ++w) tot += wcnt[w];
+        // publish the count tagged with the epoch, then arrive with release; the pollers acquire (measured
+        // faster than relaxed accesses, which linger in the SM).  Readers check the tags as well.
+        st_relaxed_gpu(a.words + 1 + blockIdx.x, ((unsigned long long)a.epoch << 32) | (unsigned)tot);
+        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(a.words) : "memory");
+        const unsigned target = a.epoch * (unsigned)G;       // the counter never resets: epoch e ends at e * G
+        const long long t0 = clock64();
+        for (;;) {
+            unsigned seen;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(a.words) : "memory");
+            if ((int)(seen - target) >= 0) break;
+            if (clock64() - t0 > (1ll << 31)) { abort_flag = 1; break; }
+        }
+    }
+    __syncthreads();
+    const bool want_lead = blockIdx.x == 0 && a.info != nullptr;   // only CTA 0 needs rows_moved
+    int n_kept;
+    if (G < CP_THREADS) {
+        // thread t gathers the count of part t; the scan runs on the registers
+        int cnt_t = 0;
+        if (tid < G && !abort_flag) {
+            const long long t0 = clock64();
+            for (;;) {
+                const unsigned long long w = ld_relaxed_gpu(a.words + 1 + tid);
+                if ((uint32_t)(w >> 32) == a.epoch) { cnt_t = (int)(uint32_t)w; break; }
+                if (clock64() - t0 > (1ll << 31)) { abort_flag = 1; break; }
+            }
+            // first part that is not retained completely
+            if (want_lead && cnt_t < max(0, min(part_bytes, s - tid * part_bytes))) atomicMin(&s_misc[2], tid);
+        }
+        int tot;
+        const int ex = warp_excl_scan(cnt_t, lane, tot);
+        if (lane == 0) warp_tot[wid] = tot;
+        __syncthreads();
+        int base = 0;
+        for (int w = 0; w < wid; ++w) base += warp_tot[w];
+        if (tid <= G) prefix[tid] = base + ex;
+        __syncthreads();
+        n_kept = prefix[G];
+    } else {
+        if (!abort_flag) {
+            for (int t = tid; t < G; t += CP_THREADS) {
+                const long long t0 = clock64();
+                for (;;) {
+                    const unsigned long long w = ld_relaxed_gpu(a.words + 1 + t);
+                    if ((uint32_t)(w >> 32) == a.epoch) { prefix[t] = (int)(uint32_t)w; break; }
+                    if (clock64() - t0 > (1ll << 31)) { abort_flag = 1; break; }
+                }
+                if (want_lead && prefix[t] < max(0, min(part_bytes, s - t * part_bytes))) atomicMin(&s_misc[2], t);
+            }
+        }
+        __syncthreads();
+        n_kept = block_excl_scan(prefix, G, warp_tot);
+    }
+    if (abort_flag) {
+        if (tid == 0) atomicOr(a.status, OMNI_DEV_TIMEOUT);
+        return;
+    }
+    const int n0 = s_misc[0], n1 = s_misc[1];
 
-    // ---- phase B: destination share of this CTA, slot map of its source chunks ---------------
-    const int G = gridDim.x;
+    // ---- phase B: destination share of this CTA, slot map of its own part -------------------------------
     const int rows_per = (n_kept + G - 1) / G;
     const int d0 = min(n_kept, (int)blockIdx.x * rows_per);
     const int d1 = min(n_kept, d0 + rows_per);
     const int n_rows = min(d1 - d0, a.rows_cap);
-
-    // first chunk that holds destination d0: largest c with prefix[c] <= d0
-    int c_first = 0;
-    {
-        int lo = 0, hi = n_chunks;       // prefix[lo] <= d0 invariant (prefix[0] = 0)
-        while (hi - lo > 1) {
-            int mid = (lo + hi) >> 1;
-            if (prefix[mid] <= d0) lo = mid; else hi = mid;
-        }
-        c_first = lo;
-    }
-    int moved_local = 0;
-    // chunks needed for the gather list [c_first, ...) and chunks owned for the slot map (c % G == b)
-    for (int pass = 0; pass < 2; ++pass) {
-        int c_begin, c_step;
-        if (pass == 0) { c_begin = c_first + wid; c_step = CP_WARPS; }
-        else { c_begin = blockIdx.x + wid * G; c_step = CP_WARPS * G; }
-        for (int c = c_begin; c < n_chunks; c += c_step) {
-            if (pass == 0 && (n_rows <= 0 || prefix[c] >= d1)) break;
-            if (pass == 1 && !a.slot_map && !a.info) break;
-            int run = prefix[c];
-            const int base = c << a.chunk_shift;
-            for (int k = 0; k < vec_per_lane; ++k) {
-                const int pos = base + k * 512 + lane * 16;
-                uint4 v = load_mask16(a.mask, pos, s);
-                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-                int cnt = nonzero_bytes(w[0]) + nonzero_bytes(w[1]) + nonzero_bytes(w[2]) + nonzero_bytes(w[3]);
-                int tot;
-                int r = run + warp_excl_scan(cnt, lane, tot);
-                run += tot;
-                int32_t out[16];
+    if (n_rows > 0) {
+        // largest part c with prefix[c] <= d0: prefix is non-decreasing, so count the entries <= d0
+        int n_le = 0;
+        for (int c0 = 0; c0 < G; c0 += 32)
+            n_le += __popc(__ballot_sync(0xffffffffu, c0 + lane < G && prefix[c0 + lane] <= d0));
+        const int c_first = n_le - 1;
+        // one warp per part that holds destinations of this CTA, taken from the last warp down (the first
+        // warps write the slot map meanwhile); a part is walked four groups at a time, loads first
+        for (int c = c_first + (CP_WARPS - 1 - wid); c < G; c += CP_WARPS) {
+            const int pc = prefix[c];
+            if (pc >= d1) break;
+            if (prefix[c + 1] == pc) continue;
+            int run = pc;
+            for (int g0 = 0; g0 < a.part_groups && run < d1; g0 += 4) {
+                uint4 v[4];
 #pragma unroll
-                for (int b = 0; b < 16; ++b) {
-                    const bool kept = (w[b >> 2] >> ((b & 3) * 8)) & 0xffu;
-                    out[b] = kept ? r : -1;
-                    if (kept) {
-                        if (pass == 0) {
-                            if (r >= d0 && r - d0 < n_rows) src_list[r - d0] = pos + b;
-                        } else if (r != pos + b) {
-                            ++moved_local;
-                        }
-                        ++r;
-                    }
-                }
-                if (pass == 1 && a.slot_map) {
-                    if (pos + 16 <= s) {
-                        int4* o4 = reinterpret_cast<int4*>(a.slot_map + pos);
-                        o4[0] = make_int4(out[0], out[1], out[2], out[3]);
-                        o4[1] = make_int4(out[4], out[5], out[6], out[7]);
-                        o4[2] = make_int4(out[8], out[9], out[10], out[11]);
-                        o4[3] = make_int4(out[12], out[13], out[14], out[15]);
-                    } else {
-                        for (int b = 0; b < 16 && pos + b < s; ++b) a.slot_map[pos + b] = out[b];
+                for (int j = 0; j < 4; ++j)
+                    v[j] = g0 + j < a.part_groups ? mask_at(a.mask, c * part_bytes + (g0 + j) * 512 + lane * 16, s)
+                                                  : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (g0 + j < a.part_groups && run < d1) {
+                        emit_sources(v[j], c * part_bytes + (g0 + j) * 512, run, lane, d0, n_rows, src_list);
+                        run += __reduce_add_sync(0xffffffffu, count_kept(v[j]));
                     }
                 }
             }
         }
     }
-    // ---- integer summary and page classes ------------------------------------------------------
-    if (a.info) {
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) moved_local += __shfl_xor_sync(0xffffffffu, moved_local, o);
-        if (lane == 0 && moved_local) atomicAdd(&a.info->rows_moved, moved_local);
-        if (blockIdx.x == 0 && tid == 0) {
+    if (a.slot_map && wg0 < wg1) {
+        int run = prefix[blockIdx.x];
+        for (int w = 0; w < wid; ++w) run += wcnt[w];
+        for (int g = wg0; g < wg1; ++g) {
+            const int base = my_base + g * 512;
+            if (base >= s) break;
+            const uint4 v = g == wg0 ? mv : mask_at(a.mask, base + lane * 16, s);
+            emit_slot_map(v, base, run, lane, s, a.slot_map);
+            run += __reduce_add_sync(0xffffffffu, count_kept(v));
+        }
+    }
+    // ---- integer summary and page classes ------------------------------------------------------------
+    if (want_lead && wid == CP_WARPS - 1) {
+        // a retained row keeps its slot exactly when every slot before it is retained: rows_moved counts the
+        // retained rows behind the first slot that is dropped
+        const int c_open = s_misc[2];
+        int lead = s;
+        if (c_open < G) {
+            for (int g = 0; g < a.part_groups; ++g) {
+                const int base = c_open * part_bytes + g * 512;
+                if (base >= s) break;
+                const uint4 v = mask_at(a.mask, base + lane * 16, s);
+                const int z = first_zero_byte(v);
+                const int cand = __reduce_min_sync(0xffffffffu, z < 16 ? base + lane * 16 + z : 0x7fffffff);
+                if (cand != 0x7fffffff) { lead = min(cand, s); break; }
+            }
+        }
+        if (lane == 0) {
             a.info->n_kept = n_kept;
             a.info->span_pages = (n_kept + a.page_size - 1) / a.page_size;
+            a.info->rows_moved = n_kept - min(lead, n_kept);
             a.info->part_begin[0] = 0;
             a.info->part_begin[1] = a.units_kept ? n0 : 0;
             a.info->part_begin[2] = a.units_kept ? n0 + n1 : 0;
@@ -241,33 +415,75 @@ __global__ void __launch_bounds__(CP_THREADS, 1) compact_pack_kernel(const Compa
             a.page_class[p] = cls;
         }
     }
-    __syncthreads();
-
-    // ---- phase C: move the rows ----------------------------------------------------------------
     if (a.k_dst == nullptr) return;
-    const long long total = (long long)n_rows * 2 * a.vpr;
-    for (long long base = tid; base < total; base += (long long)CP_THREADS * CP_UNROLL) {
-        uint4 buf[CP_UNROLL];
-        uint4* dst[CP_UNROLL];
+    __syncthreads();                                        // the source list is complete
+
+    // ---- phase C: move the rows ---------------------------------------------------------------------
+    if (a.n_slots > 0) {
+        // bulk-copy path: lane 0 of every warp streams its rows HBM -> shared memory -> HBM with
+        // cp.async.bulk, `n_slots` rows in flight per warp; no per-vector instructions at all.
+        if (lane == 0) {
+            const int n_copies = 2 * n_rows;                         // copy i: row i >> 1, K (even) or V (odd)
+            const int mcp = n_copies > wid ? (n_copies - wid + CP_WARPS - 1) / CP_WARPS : 0;
+            const uint32_t buf0 = tc::smem_u32(rowbuf) + (uint32_t)(wid * a.n_slots) * a.row_bytes;
+            auto src_of = [&](int q) {
+                const int i = wid + q * CP_WARPS;
+                return ((i & 1) ? a.v_src : a.k_src) + (size_t)src_list[i >> 1] * a.row_bytes;
+            };
+            auto dst_of = [&](int q) {
+                const int i = wid + q * CP_WARPS;
+                return ((i & 1) ? a.v_dst : a.k_dst) + (size_t)(d0 + (i >> 1)) * a.row_bytes;
+            };
+            auto issue_load = [&](int q) {
+                const int slot = q % a.n_slots;
+                const uint32_t bar = tc::smem_u32(&cbar[wid][slot]);
+                tc::mbar_expect_tx(bar, a.row_bytes);
+                bulk_load(buf0 + slot * a.row_bytes, src_of(q), a.row_bytes, bar);
+            };
+            for (int q = 0; q < mcp && q < a.n_slots; ++q) issue_load(q);
+            bool ok = true;
+            for (int q = 0; q < mcp && ok; ++q) {
+                const int slot = q % a.n_slots;
+                ok = tc::mbar_wait(tc::smem_u32(&cbar[wid][slot]), (q / a.n_slots) & 1, &abort_flag);
+                if (!ok) break;
+                bulk_store(dst_of(q), buf0 + slot * a.row_bytes, a.row_bytes);
+                // the buffer of copy q-1 is free once its store has read it: refill it
+                if (q >= 1 && q - 1 + a.n_slots < mcp) {
+                    asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    issue_load(q - 1 + a.n_slots);
+                }
+            }
+            asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+            if (!ok) atomicOr(a.status, OMNI_DEV_TIMEOUT);
+        }
+        return;
+    }
+    // vector path (rows too large for the buffers, or too small to be worth a bulk copy)
+    const int total = n_rows * 2 * a.vpr;                    // (row, K or V, vector)
+    for (int base = tid; base < total; base += CP_THREADS * CP_BATCH) {
+        uint4 buf[CP_BATCH];
 #pragma unroll
-        for (int u = 0; u < CP_UNROLL; ++u) {
-            const long long idx = base + (long long)u * CP_THREADS;
-            dst[u] = nullptr;
+        for (int u = 0; u < CP_BATCH; ++u) {
+            const int idx = base + u * CP_THREADS;
             if (idx < total) {
                 int rw, v;
-                if (a.vpr_shift >= 0) { rw = (int)(idx >> a.vpr_shift); v = (int)(idx & (a.vpr - 1)); }
-                else { rw = (int)(idx / a.vpr); v = (int)(idx - (long long)rw * a.vpr); }
-                const int r = rw >> 1;
-                const bool is_v = rw & 1;
-                const size_t so = (size_t)src_list[r] * a.row_bytes + (size_t)v * 16;
-                const size_t dof = (size_t)(d0 + r) * a.row_bytes + (size_t)v * 16;
-                buf[u] = ld_stream(reinterpret_cast<const uint4*>((is_v ? a.v_src : a.k_src) + so));
-                dst[u] = reinterpret_cast<uint4*>((is_v ? a.v_dst : a.k_dst) + dof);
+                if (a.vpr_shift >= 0) { rw = idx >> a.vpr_shift; v = idx & (a.vpr - 1); }
+                else { rw = idx / a.vpr; v = idx - rw * a.vpr; }
+                const size_t so = (size_t)src_list[rw >> 1] * a.row_bytes + (size_t)v * 16;
+                buf[u] = ld_stream(reinterpret_cast<const uint4*>(((rw & 1) ? a.v_src : a.k_src) + so));
             }
         }
 #pragma unroll
-        for (int u = 0; u < CP_UNROLL; ++u)
-            if (dst[u]) st_stream(dst[u], buf[u]);
+        for (int u = 0; u < CP_BATCH; ++u) {
+            const int idx = base + u * CP_THREADS;
+            if (idx < total) {
+                int rw, v;
+                if (a.vpr_shift >= 0) { rw = idx >> a.vpr_shift; v = idx & (a.vpr - 1); }
+                else { rw = idx / a.vpr; v = idx - rw * a.vpr; }
+                const size_t dof = (size_t)(d0 + (rw >> 1)) * a.row_bytes + (size_t)v * 16;
+                st_stream(reinterpret_cast<uint4*>(((rw & 1) ? a.v_dst : a.k_dst) + dof), buf[u]);
+            }
+        }
     }
 }
 
@@ -373,20 +589,40 @@ extern "C" omni_status omnipage_compact(omnitide_ctx* ctx, void* stream, const v
     a.page_size = page_size; a.row_bytes = (int)ctx->row_bytes; a.vpr = (int)(ctx->row_bytes >> 4);
     a.vpr_shift = -1;
     for (int sft = 0; sft < 20; ++sft) if ((1 << sft) == a.vpr) a.vpr_shift = sft;
-    a.chunk_shift = 9;
-    while (((s_span_max + (1 << a.chunk_shift) - 1) >> a.chunk_shift) > CP_MAX_CHUNKS) ++a.chunk_shift;
     a.units_kept = units_kept; a.n_units_kept_dev = n_units_kept_dev; a.n_units_max = n_units_max;
     a.slot_map = slot_map_out; a.info = info_out; a.page_class = page_class_out; a.status = ctx->status_dev;
     const int grid = ctx->sm_count;
     a.rows_cap = (s_span_max + grid - 1) / grid + 1;
-    const int max_chunks = ((s_span_max + (1 << a.chunk_shift) - 1) >> a.chunk_shift) + 2;
-    const size_t smem = (size_t)(max_chunks + a.rows_cap) * sizeof(int);
+    a.max_chunks = std::max(256, (grid + 2 + 3) & ~3);       // the one-warp scan touches 256 entries
+    a.rows_cap = (a.rows_cap + 3) & ~3;                      // keep what follows 16-byte aligned
+    const int n_grp = (s_span_max + 511) / 512;
+    a.part_groups = std::max(1, (n_grp + grid - 1) / grid);
+    ++ctx->cp_epoch;                                         // wraps together with the 32-bit arrival counter
+    a.words = ctx->cp_words;
+    a.epoch = ctx->cp_epoch;
+    const size_t smem_lists = (size_t)(a.max_chunks + a.rows_cap) * sizeof(int);
+    const size_t budget = 200 * 1024;
+    a.n_slots = 0;
+    if (k_src && ctx->row_bytes >= 512 && smem_lists < budget) {
+        const size_t per_warp = (budget - smem_lists) / CP_WARPS;
+        a.n_slots = (int)std::min<size_t>(CP_MAX_SLOTS, per_warp / ctx->row_bytes);
+        if (a.n_slots < 2) a.n_slots = 0;
+    }
+    const size_t smem = smem_lists + (size_t)a.n_slots * CP_WARPS * ctx->row_bytes;
     if (smem > 200 * 1024) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "compact: span too large for one launch");
-    if (info_out) OMNI_CUDA(ctx, cudaMemsetAsync(&info_out->rows_moved, 0, sizeof(int32_t), st));
     if (smem > 48 * 1024)
         OMNI_CUDA(ctx, cudaFuncSetAttribute(compact_pack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    compact_pack_kernel<<<grid, CP_THREADS, smem, st>>>(a);
-    OMNI_CHECK_LAUNCH(ctx, "compact_pack_kernel");
+    {
+        // cooperative: the CTAs wait for one another's counts, so all of them must be resident
+        void* kargs[] = {&a};
+        const cudaError_t le = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(compact_pack_kernel), dim3(grid),
+                                                           dim3(CP_THREADS), kargs, smem, st);
+        if (le != cudaSuccess) {
+            --ctx->cp_epoch;                                 // nothing arrived: keep the counter in step
+            OMNI_FAIL(ctx, OMNI_ERR_CUDA, "launch compact_pack_kernel: %s", cudaGetErrorString(le));
+        }
+        ctx->launches++;
+    }
     if (in_place) {
         if (!info_out) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "compact: in-place mode needs info_out");
         copy_rows_kernel<<<ctx->sm_count * 4, 256, 0, st>>>(
