@@ -46,6 +46,17 @@ def make_workload(name):
     raise SystemExit(f"unknown workload {name}")
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from one ncu capture per kernel on this workload
+# (the summaries under profiles/ give the commands); None for workloads that were not captured.
+NCU_TRAFFIC_BYTES = {
+    "long_stream": {"attention": 66.909e6 + 24.608e6, "compact": 33.702e6 + 0.810e6, "score": 186.894e6 + 57.194e6},
+}
+# special-function pipe: 16 exponentials per clock per SM (the bound of the scoring kernel)
+XU_PER_CLK_PER_SM = 16
+N_SM = 148
+SM_MAX_MHZ = 1965.0
+
+
 def algorithmic_work(w, n_kept):
     """FLOPs and bytes of one step, as defined for the roofline (masked work not counted)."""
     N, T = w.n_hist, w.t
@@ -53,6 +64,7 @@ def algorithmic_work(w, n_kept):
     row = w.h_kv * w.d * es
     return {
         "score_flop": 2.0 * w.d * w.h_q * T * N,
+        "score_exp": 1.0 * w.h_q * T * N,
         "attn_flop": 4.0 * w.d * w.h_q * (T * n_kept + T * (T + 1) / 2.0),
         "compact_bytes": 2.0 * n_kept * 2 * row + N + 4.0 * N,        # rows (R+W, K and V) + mask + slot map
         "select_bytes": 24.0 * len(w.units) + 5.0 * N,
@@ -296,15 +308,19 @@ def main():
     att_tf = work["attn_flop"] / (att_ms * 1e-3) / 1e12
     sc_tf = work["score_flop"] / (sc_ms * 1e-3) / 1e12
     cp_gbs = work["compact_bytes"] / (cp_ms * 1e-3) / 1e9
+    traffic = NCU_TRAFFIC_BYTES.get(args.workload, {})
+    xu_peak = XU_PER_CLK_PER_SM * N_SM * SM_MAX_MHZ * 1e6 / 1e12   # Texp/s
+    sc_texp = work["score_exp"] / (sc_ms * 1e-3) / 1e12
     kernels = {
         "attention": {"bound": "tensor", "achieved": att_tf, "peak": tensor_peak, "unit": "TFLOP/s",
                       "frac": att_tf / tensor_peak, "frac_of_burst_peak": att_tf / peaks["bf16_tflops"],
-                      "frac_of_nominal": att_tf / NOMINAL["bf16_tflops"], "ms": att_ms, "traffic": None},
-        "score": {"bound": "tensor", "achieved": sc_tf, "peak": tensor_peak, "unit": "TFLOP/s",
-                  "frac": sc_tf / tensor_peak, "ms": sc_ms, "traffic": None},
+                      "frac_of_nominal": att_tf / NOMINAL["bf16_tflops"], "ms": att_ms, "traffic": traffic.get("attention")},
+        "score": {"bound": "alu", "achieved": sc_texp, "peak": xu_peak, "unit": "Texp/s", "frac": sc_texp / xu_peak,
+                  "tensor_tflops": sc_tf, "tensor_frac": sc_tf / tensor_peak, "ms": sc_ms, "traffic": traffic.get("score"),
+                  "note": "bound by the exponential rate of the special-function pipe (16 per clock per SM at the max SM clock)"},
         "compact": {"bound": "hbm", "achieved": cp_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": cp_gbs / peaks["hbm_gbs"], "frac_of_nominal": cp_gbs / NOMINAL["hbm_gbs"], "ms": cp_ms,
-                    "traffic": None},
+                    "traffic": traffic.get("compact")},
         "select": {"bound": "latency", "ms": sel_ms, "achieved": work["select_bytes"] / (sel_ms * 1e-3) / 1e9, "unit": "GB/s"},
         "append": {"bound": "hbm", "ms": app_ms, "achieved": work["append_bytes"] / (app_ms * 1e-3) / 1e9,
                    "peak": peaks["hbm_gbs"], "unit": "GB/s"},
