@@ -1,18 +1,22 @@
 // Unit scoring on tcgen05 tensor cores (bf16, head dim 128).
 //
 // score_u needs, for every query row, the softmax mass that falls on each history unit.  One pass
-// over QK^T is enough: a CTA owns a pair of 128-row query tiles of one head and one contiguous range
+// over QK^T is enough: a CTA owns four 128-row query tiles of one head and one contiguous range
 // of 128-key blocks ("split"); for every row a thread keeps a running max m and the sum of
 // exp2(c*(s - m)) over the keys of the CURRENT unit, and when the unit (or the split) ends it
 // writes the pair (m, sum) -- a flash-style partial -- to scratch.  A second kernel merges a row's
 // partials into its normaliser and per-unit masses and reduces them over the 128 rows of a tile; a
 // third sums the tiles in a fixed order.  Everything is deterministic (no floating-point atomics).
 //
-//   warp 9      TMA producer: Q tiles once, then K blocks through a 4-stage shared-memory ring
-//   warp 8      one thread issues tcgen05.mma S_t = Q_t K_j^T into TMEM, two S buffers per tile
-//   warps 0-3   row sums of tile 0 (one thread per row, S read from TMEM in 32-column chunks)
-//   warps 4-7   row sums of tile 1
-// TMEM map (512 columns): S0 buffers [0,128) [128,256), S1 buffers [256,384) [384,512).
+// The kernel is bound by the exponentials (16 per clock per SM on the special-function pipe), not by
+// the contraction: a loop of this instruction mix reaches 52 / 72 / 84 / 86 % of that rate with
+// 1 / 2 / 3 / 4 warps per scheduler, hence sixteen softmax warps (four per scheduler) and one S
+// buffer per tile: while a warpgroup waits for its next S the other three keep the pipe busy.
+//
+//   warp 17     TMA producer: Q tiles once, then K blocks through a 2-stage shared-memory ring
+//   warp 16     one thread issues tcgen05.mma S_t = Q_t K_j^T into TMEM, tile after tile
+//   warps 4t..4t+3   row sums of tile t (one thread per row, S read from TMEM in 32-column chunks)
+// TMEM map (512 columns): S of tile t at [128 t, 128 t + 128).
 #include "common.cuh"
 #include "tc_ptx.cuh"
 
@@ -22,8 +26,9 @@ constexpr int BLK = 128;
 constexpr int HD = 128;
 constexpr int TILE_BYTES = BLK * HD * 2;
 constexpr int HALF_BYTES = TILE_BYTES / 2;
-constexpr int NSTAGE = 4;
-constexpr int SC_THREADS = 320;
+constexpr int NSTAGE = 2;
+constexpr int NT = 4;                          // query tiles per CTA
+constexpr int SC_THREADS = 32 * (4 * NT + 2);
 constexpr int MAX_SPLITS = 64;
 constexpr uint32_t IDESC_QK = tc::umma_idesc_bf16(128, 128, false, false);
 
@@ -42,13 +47,19 @@ struct Barriers {
     uint64_t q_full;
     uint64_t k_full[NSTAGE];
     uint64_t k_empty[NSTAGE];
-    uint64_t s_full[2][2];
-    uint64_t s_empty[2][2];
+    uint64_t s_full[NT];
+    uint64_t s_empty[NT];
     uint32_t tmem_base;
     int abort_flag;
 };
 
-constexpr int SMEM_FIXED = 2 * TILE_BYTES + NSTAGE * TILE_BYTES + 1024 + 256;
+constexpr int SMEM_FIXED = NT * TILE_BYTES + NSTAGE * TILE_BYTES + 1024 + 256;
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 
 __device__ __forceinline__ int blocks_per_split(int nkb, int n_splits) { return (nkb + n_splits - 1) / n_splits; }
 
@@ -58,9 +69,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t smem_base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - tc::smem_u32(smem_raw));
     const uint32_t q_smem = smem_base;
-    const uint32_t k_smem = smem_base + 2 * TILE_BYTES;
-    Barriers* bars = reinterpret_cast<Barriers*>(smem_gen + 2 * TILE_BYTES + NSTAGE * TILE_BYTES);
-    int* unit_end = reinterpret_cast<int*>(smem_gen + 2 * TILE_BYTES + NSTAGE * TILE_BYTES + 256);   // [n_units_max]
+    const uint32_t k_smem = smem_base + NT * TILE_BYTES;
+    Barriers* bars = reinterpret_cast<Barriers*>(smem_gen + NT * TILE_BYTES + NSTAGE * TILE_BYTES);
+    int* unit_end = reinterpret_cast<int*>(smem_gen + NT * TILE_BYTES + NSTAGE * TILE_BYTES + 256);   // [n_units_max]
     volatile int* abort_flag = &bars->abort_flag;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -84,9 +95,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int b0 = split * bps, b1 = min(nkb, b0 + bps);
     const int nb = b1 - b0;
     if (nb <= 0) return;
-    bool active[2];
+    bool active[NT];
 #pragma unroll
-    for (int tt = 0; tt < 2; ++tt) active[tt] = (2 * pair + tt) * BLK < p.t;
+    for (int tt = 0; tt < NT; ++tt) active[tt] = (NT * pair + tt) * BLK < p.t;
 
     for (int u = threadIdx.x; u < n_units; u += SC_THREADS) unit_end[u] = p.units[u].start + p.units[u].len;
     if (threadIdx.x == 0) {
@@ -95,29 +106,29 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             tc::mbar_init(tc::smem_u32(&bars->k_full[s]), 1);
             tc::mbar_init(tc::smem_u32(&bars->k_empty[s]), 1);
         }
-        for (int tt = 0; tt < 2; ++tt)
-            for (int b = 0; b < 2; ++b) {
-                tc::mbar_init(tc::smem_u32(&bars->s_full[tt][b]), 1);
-                tc::mbar_init(tc::smem_u32(&bars->s_empty[tt][b]), 128);
-            }
+        for (int tt = 0; tt < NT; ++tt) {
+            tc::mbar_init(tc::smem_u32(&bars->s_full[tt]), 1);
+            tc::mbar_init(tc::smem_u32(&bars->s_empty[tt]), 128);
+        }
         bars->abort_flag = 0;
         tc::fence_barrier_init();
     }
-    if (warp == 8) tc::tmem_alloc<512>(tc::smem_u32(&bars->tmem_base));
+    if (warp == 4 * NT) tc::tmem_alloc<512>(tc::smem_u32(&bars->tmem_base));
     tc::tcgen05_fence_before();
     __syncthreads();
     tc::tcgen05_fence_after();
     const uint32_t tmem = bars->tmem_base;
 
-    if (warp == 9) {
+    if (warp == 4 * NT + 1) {
         if (lane == 0) {
             tc::tma_prefetch_desc(&tm_q);
             tc::tma_prefetch_desc(&tm_k);
-            const int n_active = (int)active[0] + (int)active[1];
+            int n_active = 0;
+            for (int tt = 0; tt < NT; ++tt) n_active += (int)active[tt];
             tc::mbar_expect_tx(tc::smem_u32(&bars->q_full), n_active * TILE_BYTES);
-            for (int tt = 0; tt < 2; ++tt) {
+            for (int tt = 0; tt < NT; ++tt) {
                 if (!active[tt]) continue;
-                const int row0 = (2 * pair + tt) * BLK;
+                const int row0 = (NT * pair + tt) * BLK;
                 tc::tma_load_2d(q_smem + tt * TILE_BYTES, &tm_q, head * HD, row0, tc::smem_u32(&bars->q_full));
                 tc::tma_load_2d(q_smem + tt * TILE_BYTES + HALF_BYTES, &tm_q, head * HD + 64, row0, tc::smem_u32(&bars->q_full));
             }
@@ -140,24 +151,24 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
             }
         }
-    } else if (warp == 8) {
+    } else if (warp == 4 * NT) {
         if (lane == 0) {
             bool ok = tc::mbar_wait(tc::smem_u32(&bars->q_full), 0, abort_flag);
             for (int j = 0; j < nb && ok; ++j) {
-                const int stage = j % NSTAGE, buf = j & 1, use = j >> 1;
+                const int stage = j % NSTAGE;
                 ok = tc::mbar_wait(tc::smem_u32(&bars->k_full[stage]), (j / NSTAGE) & 1, abort_flag);
-                for (int tt = 0; tt < 2 && ok; ++tt) {
+                for (int tt = 0; tt < NT && ok; ++tt) {
                     if (!active[tt]) continue;
-                    ok = tc::mbar_wait(tc::smem_u32(&bars->s_empty[tt][buf]), (use & 1) ^ 1, abort_flag);
+                    ok = tc::mbar_wait(tc::smem_u32(&bars->s_empty[tt]), (j & 1) ^ 1, abort_flag);
                     tc::tcgen05_fence_after();
                     const uint32_t a0 = q_smem + tt * TILE_BYTES, bb = k_smem + stage * TILE_BYTES;
 #pragma unroll
                     for (int kk = 0; kk < HD / 16; ++kk) {
                         const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
-                        tc::umma_ss(tmem + tt * 256 + buf * 128, tc::umma_smem_desc(a0 + off, 16, 1024),
+                        tc::umma_ss(tmem + tt * 128, tc::umma_smem_desc(a0 + off, 16, 1024),
                                     tc::umma_smem_desc(bb + off, 16, 1024), IDESC_QK, kk > 0, 1u);
                     }
-                    tc::umma_commit(tc::smem_u32(&bars->s_full[tt][buf]));
+                    tc::umma_commit(tc::smem_u32(&bars->s_full[tt]));
                 }
                 tc::umma_commit(tc::smem_u32(&bars->k_empty[stage]));
             }
@@ -167,7 +178,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (active[tt]) {
             const int r = (warp & 3) * 32 + lane;
             const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-            const int tile = head * p.n_row_tiles + 2 * pair + tt;
+            const int tile = head * p.n_row_tiles + NT * pair + tt;
             float2* part = p.part + (size_t)tile * p.seg_cap * BLK + r;
             const float c = p.scale_log2;
             // unit that holds the first key of this split
@@ -185,39 +196,43 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             float m = -INFINITY, acc = 0.f;
             bool ok = true;
             for (int j = 0; j < nb && ok; ++j) {
-                const int buf = j & 1;
-                ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&bars->s_full[tt][buf]), (j >> 1) & 1, abort_flag));
+                ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&bars->s_full[tt]), j & 1, abort_flag));
                 tc::tcgen05_fence_after();
-                const uint32_t s_tmem = tmem + tt * 256 + buf * 128 + lane_addr;
-#pragma unroll 1
-                for (int ch = 0; ch < 4; ++ch) {
-                    uint32_t sv[32];
-                    tc::tmem_ld32(s_tmem + ch * 32, sv);
-                    tc::tmem_wait_ld();
+                const uint32_t s_tmem = tmem + tt * 128 + lane_addr;
+                // two register buffers: the TMEM load of chunk ch+1 is in flight while chunk ch is summed
+                uint32_t sva[32], svb[32];
+                auto process = [&](uint32_t (&sv)[32], const int ch) {
                     const int k0 = key + ch * 32;
                     const int n_valid = min(32, n_hist - k0);           // <= 0 past the end of the history
-                    if (n_valid <= 0) break;
+                    if (n_valid <= 0) return;
                     if (n_valid < 32) {
 #pragma unroll
                         for (int i = 0; i < 32; ++i)
                             if (i >= n_valid) sv[i] = 0xff800000u;
                     }
-                    float cm = __uint_as_float(sv[0]);
+                    // row maximum of the chunk: a tree of three-input maxima (depth 4 instead of a chain of 31)
+                    float t[11];
 #pragma unroll
-                    for (int i = 1; i < 32; ++i) cm = fmaxf(cm, __uint_as_float(sv[i]));
+                    for (int i = 0; i < 10; ++i)
+                        t[i] = max3(__uint_as_float(sv[3 * i]), __uint_as_float(sv[3 * i + 1]), __uint_as_float(sv[3 * i + 2]));
+                    t[10] = fmaxf(__uint_as_float(sv[30]), __uint_as_float(sv[31]));
+                    const float t0 = max3(t[0], t[1], t[2]), t1 = max3(t[3], t[4], t[5]), t2 = max3(t[6], t[7], t[8]);
+                    const float cm = max3(max3(t0, t1, t2), t[9], t[10]);
                     const float m_new = fmaxf(m, cm);
                     acc *= tc::ex2_approx((m - m_new) * c);             // exp2(-inf) = 0 on the first chunk
                     m = m_new;
                     const float neg_m = -m * c;
                     if (k0 + 32 <= u_end) {
                         // the whole chunk lies inside the current unit
-                        float s0 = 0.f, s1 = 0.f;
+                        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-                        for (int i = 0; i < 32; i += 2) {
+                        for (int i = 0; i < 32; i += 4) {
                             s0 += tc::ex2_approx(fmaf(__uint_as_float(sv[i]), c, neg_m));
                             s1 += tc::ex2_approx(fmaf(__uint_as_float(sv[i + 1]), c, neg_m));
+                            s2 += tc::ex2_approx(fmaf(__uint_as_float(sv[i + 2]), c, neg_m));
+                            s3 += tc::ex2_approx(fmaf(__uint_as_float(sv[i + 3]), c, neg_m));
                         }
-                        acc += s0 + s1;
+                        acc += (s0 + s1) + (s2 + s3);
                         if (k0 + 32 == u_end && k0 + 32 < n_hist) {
                             part[(size_t)(u + split) * BLK] = make_float2(m, acc);
                             acc = 0.f;
@@ -237,9 +252,21 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                             acc += tc::ex2_approx(fmaf(__uint_as_float(sv[i]), c, neg_m));
                         }
                     }
-                }
+                };
+                tc::tmem_ld32(s_tmem, sva);
+                tc::tmem_wait_ld();
+                tc::tmem_ld32(s_tmem + 32, svb);
+                process(sva, 0);
+                tc::tmem_wait_ld();
+                tc::tmem_ld32(s_tmem + 64, sva);
+                process(svb, 1);
+                tc::tmem_wait_ld();
+                tc::tmem_ld32(s_tmem + 96, svb);
+                process(sva, 2);
+                tc::tmem_wait_ld();
+                process(svb, 3);
                 tc::tcgen05_fence_before();
-                tc::mbar_arrive(tc::smem_u32(&bars->s_empty[tt][buf]));
+                tc::mbar_arrive(tc::smem_u32(&bars->s_empty[tt]));
                 key += BLK;
             }
             // the split (or the history) ends inside unit u
@@ -250,7 +277,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     tc::tcgen05_fence_before();
     __syncthreads();
     if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, OMNI_DEV_TIMEOUT);
-    if (warp == 8) {
+    if (warp == 4 * NT) {
         tc::tcgen05_fence_after();
         tc::tmem_dealloc<512>(tmem);
     }
@@ -350,7 +377,7 @@ omni_status omni_score_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q, int
     p.units = units; p.n_units_dev = n_units_dev; p.n_units_max = n_units_max;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.part = ctx->score_part; p.seg_cap = g.u_cap + MAX_SPLITS;
-    p.n_pairs = (t + 2 * BLK - 1) / (2 * BLK);
+    p.n_pairs = (t + NT * BLK - 1) / (NT * BLK);
     p.n_row_tiles = (t + BLK - 1) / BLK;
     p.status = ctx->status_dev;
     // split the key range so that the grid fills whole waves of SMs and a split keeps >= 8 key blocks
