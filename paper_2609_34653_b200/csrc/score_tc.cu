@@ -61,6 +61,72 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     return d;
 }
 
+// 2^x for x <= 0 on the FMA and integer pipes (no special-function unit): x is split into the nearest
+// integer n and f in [-0.5, 0.5], 2^f comes from a degree-4 minimax polynomial (relative error 2.7e-6),
+// and n is added to the exponent field.  Inputs below -125 (masked columns hold -inf) give about 2^-125.
+__device__ __forceinline__ float exp2_poly(float x) {
+    x = fmaxf(x, -125.f);
+    const float t = x + 12582912.f;                          // 1.5 * 2^23: the low mantissa bits now hold n
+    const float f = x - (t - 12582912.f);
+    float p = 0.009570031426846981f;
+    p = fmaf(p, f, 0.055917657911777496f);
+    p = fmaf(p, f, 0.240247443318367f);
+    p = fmaf(p, f, 0.6931218504905701f);
+    p = fmaf(p, f, 0.9999992847442627f);
+    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+// packed fp32 pairs (one instruction for two lanes of arithmetic)
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// the same for a packed pair
+__device__ __forceinline__ uint64_t exp2_poly2(uint64_t x2) {
+    float x0, x1;
+    unpack2(x2, x0, x1);
+    x2 = pack2(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
+    const uint64_t t2 = add2(x2, pack2(12582912.f, 12582912.f));
+    const uint64_t n2 = add2(t2, pack2(-12582912.f, -12582912.f));
+    const uint64_t f2 = fma2(n2, pack2(-1.f, -1.f), x2);
+    uint64_t p2 = pack2(0.009570031426846981f, 0.009570031426846981f);
+    p2 = fma2(p2, f2, pack2(0.055917657911777496f, 0.055917657911777496f));
+    p2 = fma2(p2, f2, pack2(0.240247443318367f, 0.240247443318367f));
+    p2 = fma2(p2, f2, pack2(0.6931218504905701f, 0.6931218504905701f));
+    p2 = fma2(p2, f2, pack2(0.9999992847442627f, 0.9999992847442627f));
+    float p0, p1, t0, t1;
+    unpack2(p2, p0, p1);
+    unpack2(t2, t0, t1);
+    return pack2(__int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23)),
+                 __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23)));
+}
+#ifndef SC_ROLL
+#define SC_ROLL 0
+#endif
+#ifndef SC_POLY_EVERY
+#define SC_POLY_EVERY 4        // every n-th pair of exponentials of a full chunk takes the polynomial path (0: none)
+#endif
+template <int PAIR>
+__device__ __forceinline__ uint64_t exp2_pair(uint64_t x2) {
+    if (SC_POLY_EVERY > 0 && (PAIR % SC_POLY_EVERY) == SC_POLY_EVERY - 1) return exp2_poly2(x2);
+    float x0, x1;
+    unpack2(x2, x0, x1);
+    return pack2(tc::ex2_approx(x0), tc::ex2_approx(x1));
+}
+
 __device__ __forceinline__ int blocks_per_split(int nkb, int n_splits) { return (nkb + n_splits - 1) / n_splits; }
 
 __global__ void __launch_bounds__(SC_THREADS, 1)
@@ -201,7 +267,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const uint32_t s_tmem = tmem + tt * 128 + lane_addr;
                 // two register buffers: the TMEM load of chunk ch+1 is in flight while chunk ch is summed
                 uint32_t sva[32], svb[32];
-                auto process = [&](uint32_t (&sv)[32], const int ch) {
+                auto process = [&](uint32_t (&sv)[32], const int ch) __attribute__((always_inline)) {
                     const int k0 = key + ch * 32;
                     const int n_valid = min(32, n_hist - k0);           // <= 0 past the end of the history
                     if (n_valid <= 0) return;
@@ -224,15 +290,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     const float neg_m = -m * c;
                     if (k0 + 32 <= u_end) {
                         // the whole chunk lies inside the current unit
-                        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-                        for (int i = 0; i < 32; i += 4) {
-                            s0 += tc::ex2_approx(fmaf(__uint_as_float(sv[i]), c, neg_m));
-                            s1 += tc::ex2_approx(fmaf(__uint_as_float(sv[i + 1]), c, neg_m));
-                            s2 += tc::ex2_approx(fmaf(__uint_as_float(sv[i + 2]), c, neg_m));
-                            s3 += tc::ex2_approx(fmaf(__uint_as_float(sv[i + 3]), c, neg_m));
-                        }
-                        acc += (s0 + s1) + (s2 + s3);
+                        float s0, s1;
+                        // pairs of columns: one packed FMA scales two logits, one packed add sums two weights
+                        const uint64_t c2 = pack2(c, c), nm2 = pack2(neg_m, neg_m);
+                        uint64_t a0 = 0ull, a1 = 0ull;
+#define SC_PAIR(i, acc) \
+    acc = add2(acc, exp2_pair<(i) / 2>(fma2(pack2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), c2, nm2)));
+                        SC_PAIR(0, a0)  SC_PAIR(2, a1)  SC_PAIR(4, a0)  SC_PAIR(6, a1)
+                        SC_PAIR(8, a0)  SC_PAIR(10, a1) SC_PAIR(12, a0) SC_PAIR(14, a1)
+                        SC_PAIR(16, a0) SC_PAIR(18, a1) SC_PAIR(20, a0) SC_PAIR(22, a1)
+                        SC_PAIR(24, a0) SC_PAIR(26, a1) SC_PAIR(28, a0) SC_PAIR(30, a1)
+#undef SC_PAIR
+                        unpack2(add2(a0, a1), s0, s1);
+                        acc += s0 + s1;
                         if (k0 + 32 == u_end && k0 + 32 < n_hist) {
                             part[(size_t)(u + split) * BLK] = make_float2(m, acc);
                             acc = 0.f;
@@ -254,19 +324,25 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     }
                 };
                 tc::tmem_ld32(s_tmem, sva);
-                tc::tmem_wait_ld();
-                tc::tmem_ld32(s_tmem + 32, svb);
-                process(sva, 0);
-                tc::tmem_wait_ld();
-                tc::tmem_ld32(s_tmem + 64, sva);
-                process(svb, 1);
-                tc::tmem_wait_ld();
-                tc::tmem_ld32(s_tmem + 96, svb);
-                process(sva, 2);
-                tc::tmem_wait_ld();
-                process(svb, 3);
-                tc::tcgen05_fence_before();
-                tc::mbar_arrive(tc::smem_u32(&bars->s_empty[tt]));
+#if SC_ROLL
+#pragma unroll 1
+#else
+#pragma unroll
+#endif
+                for (int h = 0; h < 2; ++h) {
+                    tc::tmem_wait_ld();
+                    tc::tmem_ld32(s_tmem + h * 64 + 32, svb);
+                    process(sva, 2 * h);
+                    tc::tmem_wait_ld();
+                    if (h == 0) {
+                        tc::tmem_ld32(s_tmem + 64, sva);
+                    } else {
+                        // S is in registers: the next block's MMA may overwrite it while the last chunk is summed
+                        tc::tcgen05_fence_before();
+                        tc::mbar_arrive(tc::smem_u32(&bars->s_empty[tt]));
+                    }
+                    process(svb, 2 * h + 1);
+                }
                 key += BLK;
             }
             // the split (or the history) ends inside unit u
