@@ -360,8 +360,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 }
 
 // Merge the partials of each row, reduce over the 128 rows of a tile: tile_mass[tile][u].
+// blockIdx.y cuts the units into COMBINE_Y ranges (every range recomputes the row normaliser, which is cheap).
+constexpr int COMBINE_Y = 4;
 __global__ void __launch_bounds__(128) score_combine_kernel(const ScoreParams p, float* tile_mass) {
-    __shared__ float red[4];
+    extern __shared__ int cmb_smem[];
     const int tile = blockIdx.x;
     const int row_tile = tile % p.n_row_tiles;
     const int r = threadIdx.x, lane = r & 31, wid = r >> 5;
@@ -372,41 +374,56 @@ __global__ void __launch_bounds__(128) score_combine_kernel(const ScoreParams p,
     if (n_hist > p.n_hist_max) return;
     const int nkb = (n_hist + BLK - 1) / BLK;
     const int bps = blocks_per_split(nkb, p.n_splits);
+    // first and last split of every unit, once per CTA
+    int* s_first = cmb_smem;                                  // [n_units]
+    int* s_last = cmb_smem + p.n_units_max;                   // [n_units]
+    float* red = reinterpret_cast<float*>(cmb_smem + 2 * p.n_units_max);   // [n_units][4]
+    for (int u = r; u < n_units; u += 128) {
+        const omni_unit un = p.units[u];
+        s_first[u] = (un.start / BLK) / bps;
+        s_last[u] = ((un.start + un.len - 1) / BLK) / bps;
+    }
+    __syncthreads();
     const bool valid = row_tile * BLK + r < p.t;
     const float2* part = p.part + (size_t)tile * p.seg_cap * BLK + r;
     const float c = p.scale_log2;
+    // the row's partials are the consecutive slots [0, n_units + s_last[n_units-1]]: slot u + s holds (unit u, split s)
+    const int n_slots = n_units + s_last[n_units - 1];
     float M = -INFINITY, Z = 0.f;
     if (valid) {
-        for (int u = 0; u < n_units; ++u) {
-            const omni_unit un = p.units[u];
-            const int s_first = (un.start / BLK) / bps, s_last = ((un.start + un.len - 1) / BLK) / bps;
-            for (int s = s_first; s <= s_last; ++s) {
-                const float2 ml = part[(size_t)(u + s) * BLK];
-                const float m_new = fmaxf(M, ml.x);
-                Z = Z * exp2f((M - m_new) * c) + ml.y * exp2f((ml.x - m_new) * c);
-                M = m_new;
-            }
+        for (int i0 = 0; i0 < n_slots; i0 += 8) {
+            float2 ml[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) ml[k] = i0 + k < n_slots ? part[(size_t)(i0 + k) * BLK] : make_float2(-INFINITY, 0.f);
+            float mx = M;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) mx = fmaxf(mx, ml[k].x);
+            float z = Z * tc::ex2_approx((M - mx) * c);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) z += ml[k].y * tc::ex2_approx((ml[k].x - mx) * c);
+            M = mx;
+            Z = z;
         }
     }
     const float inv_z = valid ? 1.f / Z : 0.f;
-    for (int u = 0; u < n_units; ++u) {
-        const omni_unit un = p.units[u];
+    const int per_y = (n_units + COMBINE_Y - 1) / COMBINE_Y;
+    const int u0 = blockIdx.y * per_y, u1 = min(n_units, u0 + per_y);
+    for (int u = u0; u < u1; ++u) {
         float v = 0.f;
         if (valid) {
-            const int s_first = (un.start / BLK) / bps, s_last = ((un.start + un.len - 1) / BLK) / bps;
-            for (int s = s_first; s <= s_last; ++s) {
-                const float2 ml = part[(size_t)(u + s) * BLK];
-                v += ml.y * exp2f((ml.x - M) * c);
+            for (int sp = s_first[u]; sp <= s_last[u]; ++sp) {
+                const float2 ml = part[(size_t)(u + sp) * BLK];
+                v += ml.y * tc::ex2_approx((ml.x - M) * c);
             }
             v *= inv_z;
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        if (lane == 0) red[wid] = v;
-        __syncthreads();
-        if (r == 0) tile_mass[(size_t)tile * p.n_units_max + u] = (red[0] + red[1]) + (red[2] + red[3]);
-        __syncthreads();
+        if (lane == 0) red[u * 4 + wid] = v;
     }
+    __syncthreads();
+    for (int u = u0 + r; u < u1; u += 128)
+        tile_mass[(size_t)tile * p.n_units_max + u] = (red[u * 4] + red[u * 4 + 1]) + (red[u * 4 + 2] + red[u * 4 + 3]);
 }
 
 // mass_u = sum over tiles (fixed order) / rows;  score_u = w[modality] * mass_u * N / len_u
@@ -474,7 +491,7 @@ omni_status omni_score_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q, int
     score_tc_kernel<<<base_items * p.n_splits, SC_THREADS, smem, st>>>(tm_q, tm_k, p);
     OMNI_CHECK_LAUNCH(ctx, "score_tc_kernel");
     const int n_tiles = p.n_row_tiles * g.h_q;
-    score_combine_kernel<<<n_tiles, 128, 0, st>>>(p, ctx->score_tile_mass);
+    score_combine_kernel<<<dim3(n_tiles, COMBINE_Y), 128, (size_t)n_units_max * 6 * sizeof(int), st>>>(p, ctx->score_tile_mass);
     OMNI_CHECK_LAUNCH(ctx, "score_combine_kernel");
     score_finalize_kernel<<<n_units_max, 128, 0, st>>>(ctx->score_tile_mass, n_tiles, units, n_units_dev, n_units_max,
                                                        w[0], w[1], w[2], 1.0f / ((float)t * g.h_q), scores_out, mass_out);
