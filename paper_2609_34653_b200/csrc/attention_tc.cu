@@ -30,6 +30,18 @@
 
 namespace {
 
+#ifndef ATT_POLY_EVERY
+#define ATT_POLY_EVERY 0       // every n-th pair of exponentials takes the polynomial path (0: none; 2-4 measured no gain here)
+#endif
+template <int PAIR>
+__device__ __forceinline__ uint64_t exp2_pair(uint64_t x2) {
+    // degree 3 (relative error 7.5e-5) is far below the bf16 rounding of the weights
+    if (ATT_POLY_EVERY > 0 && (PAIR % ATT_POLY_EVERY) == ATT_POLY_EVERY - 1) return tc::exp2_poly2<3>(x2);
+    float x0, x1;
+    tc::unpack2(x2, x0, x1);
+    return tc::pack2(tc::ex2_approx(x0), tc::ex2_approx(x1));
+}
+
 constexpr int BQ = 128;                  // rows per query tile
 constexpr int BK = 128;                  // keys per KV block
 constexpr int HK = 64;                   // keys per softmax warpgroup and block
@@ -386,13 +398,24 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         if (32 + i >= n_valid) sb[i] = 0xff800000u;
                     }
                 }
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+                // row maximum of the 64 logits: three-input maxima, four independent chains
+                float mx0 = tc::max3(__uint_as_float(sa[0]), __uint_as_float(sa[1]), __uint_as_float(sb[0]));
+                float mx1 = tc::max3(__uint_as_float(sa[2]), __uint_as_float(sa[3]), __uint_as_float(sb[1]));
+                float mx2 = tc::max3(__uint_as_float(sa[4]), __uint_as_float(sa[5]), __uint_as_float(sb[2]));
+                float mx3 = tc::max3(__uint_as_float(sa[6]), __uint_as_float(sa[7]), __uint_as_float(sb[3]));
 #pragma unroll
-                for (int i = 0; i < 32; i += 4) {
-                    mx0 = fmaxf(mx0, fmaxf(__uint_as_float(sa[i]), __uint_as_float(sb[i])));
-                    mx1 = fmaxf(mx1, fmaxf(__uint_as_float(sa[i + 1]), __uint_as_float(sb[i + 1])));
-                    mx2 = fmaxf(mx2, fmaxf(__uint_as_float(sa[i + 2]), __uint_as_float(sb[i + 2])));
-                    mx3 = fmaxf(mx3, fmaxf(__uint_as_float(sa[i + 3]), __uint_as_float(sb[i + 3])));
+                for (int i = 8; i < 32; i += 8) {
+                    mx0 = tc::max3(mx0, __uint_as_float(sa[i]), __uint_as_float(sa[i + 1]));
+                    mx1 = tc::max3(mx1, __uint_as_float(sa[i + 2]), __uint_as_float(sa[i + 3]));
+                    mx2 = tc::max3(mx2, __uint_as_float(sa[i + 4]), __uint_as_float(sa[i + 5]));
+                    mx3 = tc::max3(mx3, __uint_as_float(sa[i + 6]), __uint_as_float(sa[i + 7]));
+                }
+#pragma unroll
+                for (int i = 4; i < 32; i += 8) {
+                    mx0 = tc::max3(mx0, __uint_as_float(sb[i]), __uint_as_float(sb[i + 1]));
+                    mx1 = tc::max3(mx1, __uint_as_float(sb[i + 2]), __uint_as_float(sb[i + 3]));
+                    mx2 = tc::max3(mx2, __uint_as_float(sb[i + 4]), __uint_as_float(sb[i + 5]));
+                    mx3 = tc::max3(mx3, __uint_as_float(sb[i + 6]), __uint_as_float(sb[i + 7]));
                 }
                 const float bm = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
                 if ((warp & 3) == 0) TRACE(w, 1);
@@ -408,21 +431,25 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
                 // a row that has seen no key yet keeps m_ref = -inf; exponentiate against 0 so that P = 0, not NaN
                 const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref * p.scale_log2;
-                float rs0 = 0.f, rs1 = 0.f;
+                // pairs of columns: a packed FMA scales two logits and a packed add sums two weights
+                const uint64_t c2 = tc::pack2(p.scale_log2, p.scale_log2), nm2 = tc::pack2(neg_m, neg_m);
+                uint64_t rs0 = 0ull, rs1 = 0ull;
                 uint32_t pk[32];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const float a0 = tc::ex2_approx(fmaf(__uint_as_float(sa[2 * i]), p.scale_log2, neg_m));
-                    const float a1 = tc::ex2_approx(fmaf(__uint_as_float(sa[2 * i + 1]), p.scale_log2, neg_m));
-                    const float b0 = tc::ex2_approx(fmaf(__uint_as_float(sb[2 * i]), p.scale_log2, neg_m));
-                    const float b1 = tc::ex2_approx(fmaf(__uint_as_float(sb[2 * i + 1]), p.scale_log2, neg_m));
-                    pk[i] = tc::pack_bf16x2(a0, a1);
-                    pk[16 + i] = tc::pack_bf16x2(b0, b1);
-                    // the normaliser sums the ROUNDED weights the tensor core will use, so that the
-                    // weights of a row sum to one exactly and the rounding of a dominant weight cancels
-                    rs0 += __uint_as_float(pk[i] << 16) + __uint_as_float(pk[i] & 0xffff0000u);
-                    rs1 += __uint_as_float(pk[16 + i] << 16) + __uint_as_float(pk[16 + i] & 0xffff0000u);
-                }
+#define ATT_PAIR(src, i, dst, acc)                                                                            \
+    {                                                                                                         \
+        const uint64_t x2 = tc::fma2(tc::pack2(__uint_as_float(src[2 * (i)]), __uint_as_float(src[2 * (i) + 1])), c2, nm2); \
+        float e0, e1;                                                                                         \
+        tc::unpack2(exp2_pair<(dst)>(x2), e0, e1);                                                            \
+        pk[dst] = tc::pack_bf16x2(e0, e1);                                                                    \
+        /* the normaliser sums the ROUNDED weights the tensor core will use, so that the weights of a row */ \
+        /* sum to one exactly and the rounding of a dominant weight cancels */                                \
+        acc = tc::add2(acc, tc::pack2(__uint_as_float(pk[dst] << 16), __uint_as_float(pk[dst] & 0xffff0000u))); \
+    }
+#define ATT_PAIR4(i) ATT_PAIR(sa, i, i, rs0) ATT_PAIR(sb, i, 16 + (i), rs1)
+                ATT_PAIR4(0)  ATT_PAIR4(1)  ATT_PAIR4(2)  ATT_PAIR4(3)  ATT_PAIR4(4)  ATT_PAIR4(5)  ATT_PAIR4(6)  ATT_PAIR4(7)
+                ATT_PAIR4(8)  ATT_PAIR4(9)  ATT_PAIR4(10) ATT_PAIR4(11) ATT_PAIR4(12) ATT_PAIR4(13) ATT_PAIR4(14) ATT_PAIR4(15)
+#undef ATT_PAIR4
+#undef ATT_PAIR
                 tc::tmem_st32(s_tmem, pk);                   // P over the first 32 columns of this half of the S buffer
                 if ((warp & 3) == 0) TRACE(w, 2);
                 // O is touched only after the PVs of the previous block have completed (they have, by now, nearly always)
@@ -441,7 +468,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         tc::tmem_st32(o_own + c * 32, ov);
                     }
                 }
-                l_sum += rs0 + rs1;
+                {
+                    float r0, r1;
+                    tc::unpack2(tc::add2(rs0, rs1), r0, r1);
+                    l_sum += r0 + r1;
+                }
                 if ((warp & 3) == 0) TRACE(w, 3);
 
                 if (tail_partial && j == nhb - 1) {

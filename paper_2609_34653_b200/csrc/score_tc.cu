@@ -55,73 +55,14 @@ struct Barriers {
 
 constexpr int SMEM_FIXED = NT * TILE_BYTES + NSTAGE * TILE_BYTES + 1024 + 256;
 
-__device__ __forceinline__ float max3(float a, float b, float c) {
-    float d;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
+using tc::pack2; using tc::unpack2; using tc::fma2; using tc::add2; using tc::max3;
 
-// 2^x for x <= 0 on the FMA and integer pipes (no special-function unit): x is split into the nearest
-// integer n and f in [-0.5, 0.5], 2^f comes from a degree-4 minimax polynomial (relative error 2.7e-6),
-// and n is added to the exponent field.  Inputs below -125 (masked columns hold -inf) give about 2^-125.
-__device__ __forceinline__ float exp2_poly(float x) {
-    x = fmaxf(x, -125.f);
-    const float t = x + 12582912.f;                          // 1.5 * 2^23: the low mantissa bits now hold n
-    const float f = x - (t - 12582912.f);
-    float p = 0.009570031426846981f;
-    p = fmaf(p, f, 0.055917657911777496f);
-    p = fmaf(p, f, 0.240247443318367f);
-    p = fmaf(p, f, 0.6931218504905701f);
-    p = fmaf(p, f, 0.9999992847442627f);
-    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
-}
-// packed fp32 pairs (one instruction for two lanes of arithmetic)
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-    uint64_t d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-    uint64_t d;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-// the same for a packed pair
-__device__ __forceinline__ uint64_t exp2_poly2(uint64_t x2) {
-    float x0, x1;
-    unpack2(x2, x0, x1);
-    x2 = pack2(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
-    const uint64_t t2 = add2(x2, pack2(12582912.f, 12582912.f));
-    const uint64_t n2 = add2(t2, pack2(-12582912.f, -12582912.f));
-    const uint64_t f2 = fma2(n2, pack2(-1.f, -1.f), x2);
-    uint64_t p2 = pack2(0.009570031426846981f, 0.009570031426846981f);
-    p2 = fma2(p2, f2, pack2(0.055917657911777496f, 0.055917657911777496f));
-    p2 = fma2(p2, f2, pack2(0.240247443318367f, 0.240247443318367f));
-    p2 = fma2(p2, f2, pack2(0.6931218504905701f, 0.6931218504905701f));
-    p2 = fma2(p2, f2, pack2(0.9999992847442627f, 0.9999992847442627f));
-    float p0, p1, t0, t1;
-    unpack2(p2, p0, p1);
-    unpack2(t2, t0, t1);
-    return pack2(__int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23)),
-                 __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23)));
-}
-#ifndef SC_ROLL
-#define SC_ROLL 0
-#endif
 #ifndef SC_POLY_EVERY
 #define SC_POLY_EVERY 4        // every n-th pair of exponentials of a full chunk takes the polynomial path (0: none)
 #endif
 template <int PAIR>
 __device__ __forceinline__ uint64_t exp2_pair(uint64_t x2) {
-    if (SC_POLY_EVERY > 0 && (PAIR % SC_POLY_EVERY) == SC_POLY_EVERY - 1) return exp2_poly2(x2);
+    if (SC_POLY_EVERY > 0 && (PAIR % SC_POLY_EVERY) == SC_POLY_EVERY - 1) return tc::exp2_poly2<4>(x2);
     float x0, x1;
     unpack2(x2, x0, x1);
     return pack2(tc::ex2_approx(x0), tc::ex2_approx(x1));
@@ -324,11 +265,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     }
                 };
                 tc::tmem_ld32(s_tmem, sva);
-#if SC_ROLL
-#pragma unroll 1
-#else
 #pragma unroll
-#endif
                 for (int h = 0; h < 2; ++h) {
                     tc::tmem_wait_ld();
                     tc::tmem_ld32(s_tmem + h * 64 + 32, svb);

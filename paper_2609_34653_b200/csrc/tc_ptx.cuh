@@ -183,6 +183,63 @@ __device__ __forceinline__ float ex2_approx(float x) {
     asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// ---------------------------------------------------------------- packed fp32 pairs and a polynomial exp2
+// One instruction for two lanes of fp32 arithmetic (sm_100 f32x2 forms).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// 2^x for a pair of x <= 0 on the FMA and integer pipes (the special-function pipe, 16 results per clock
+// per SM, is the scarce unit of a softmax).  x is split into the nearest integer n and f in [-0.5, 0.5];
+// 2^f comes from a minimax polynomial (DEG 3: relative error 7.5e-5, DEG 4: 2.7e-6) and n is added to the
+// exponent field.  Inputs below -125 (masked columns hold -inf) give about 2^-125.
+template <int DEG>
+__device__ __forceinline__ uint64_t exp2_poly2(uint64_t x2) {
+    float x0, x1;
+    unpack2(x2, x0, x1);
+    x2 = pack2(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
+    const uint64_t t2 = add2(x2, pack2(12582912.f, 12582912.f));      // 1.5 * 2^23: the low mantissa bits hold n
+    const uint64_t n2 = add2(t2, pack2(-12582912.f, -12582912.f));
+    const uint64_t f2 = fma2(n2, pack2(-1.f, -1.f), x2);
+    uint64_t p2;
+    if (DEG == 3) {
+        p2 = pack2(0.055170927196741104f, 0.055170927196741104f);
+        p2 = fma2(p2, f2, pack2(0.24260930716991425f, 0.24260930716991425f));
+        p2 = fma2(p2, f2, pack2(0.6932609677314758f, 0.6932609677314758f));
+        p2 = fma2(p2, f2, pack2(0.9999281764030457f, 0.9999281764030457f));
+    } else {
+        p2 = pack2(0.009570031426846981f, 0.009570031426846981f);
+        p2 = fma2(p2, f2, pack2(0.055917657911777496f, 0.055917657911777496f));
+        p2 = fma2(p2, f2, pack2(0.240247443318367f, 0.240247443318367f));
+        p2 = fma2(p2, f2, pack2(0.6931218504905701f, 0.6931218504905701f));
+        p2 = fma2(p2, f2, pack2(0.9999992847442627f, 0.9999992847442627f));
+    }
+    float p0, p1, t0, t1;
+    unpack2(p2, p0, p1);
+    unpack2(t2, t0, t1);
+    return pack2(__int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23)),
+                 __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23)));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t r;
     asm volatile("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
