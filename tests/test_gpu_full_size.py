@@ -129,3 +129,75 @@ def test_sweep_cells_full_size(H, ob, P, t, ratio, page, cell, oracle_groups):
     _check_integer_path_and_sampled_attention(H, ob, P, w, res, rng)
     assert res["info"]["span_pages"] * page >= res["info"]["n_kept"]
     _check_scores_by_group(H, ob, P, w, res["scores"], oracle_groups=oracle_groups)
+
+
+def test_stream_loop_short(H, ob, P):
+    """Config 4 shape: chunks of one frame from {640, 1280, 2304} tokens plus 2 s of audio at 10-25 tok/s,
+    32/8 heads of 128, bf16, one layer, the cache carried on the device from chunk to chunk.  The budget
+    is scaled down so that eviction starts within a few chunks.  Every step is compared with the oracle
+    advanced from the same state: scores within tolerance, selection by the oracle's rule on the GPU's
+    scores, cache bytes and unit table exactly, attention within tolerance."""
+    sched = wl.loop_schedule(n_chunks=7)
+    budget, page, R, caps, w_mod = 3000, 64, 1, (-1, -1, -1), (1.0, 2.0, 2.0)
+    h_q, h_kv, d = 32, 8, 128
+    s_cap, u_cap, t_cap = 12288, 64, 2400
+    ctx = ob.Context(h_q, h_kv, d, "bf16", s_cap, u_cap, t_cap)
+    rng = np.random.Generator(np.random.PCG64(4242))
+    draw = lambda shape: wl.round_to_bf16(rng.standard_normal(shape, dtype=np.float32))
+    units = wl.loop_prefix_units()
+    k_cache, v_cache = draw((16, h_kv, d)), draw((16, h_kv, d))
+    dev = lambda a: ob.to_device(a, "bf16")
+    k_a = torch.zeros((s_cap, h_kv, d), dtype=torch.bfloat16, device="cuda")
+    v_a = torch.zeros_like(k_a)
+    k_b, v_b = torch.full_like(k_a, float("nan")), torch.full_like(v_a, float("nan"))
+    k_a[:16], v_a[:16] = dev(k_cache), dev(v_cache)
+    units_a = ob.units_to_device(units, u_cap)
+    units_b = torch.zeros_like(units_a)
+    n_hist_a, n_units_a = H.i32(16), H.i32(len(units))
+    n_hist_b, n_units_b = H.i32(-1), H.i32(-1)
+    params = ob.select_params(budget, R, caps)
+    evicted = False
+    for c, cu in enumerate(sched):
+        T = int(cu[:, 1].sum())
+        n, U = len(k_cache), len(units)
+        zs = np.exp(0.5 * rng.standard_normal(len(cu))).astype(np.float32)
+        q, v_chunk = draw((T, h_q, d)), draw((T, h_kv, d))
+        k_chunk = wl.round_to_bf16(rng.standard_normal((T, h_kv, d), dtype=np.float32) * np.repeat(zs, cu[:, 1])[:, None, None])
+        o = torch.full((T, h_q, d), float("nan"), dtype=torch.float32, device="cuda")
+        info = torch.zeros((8,), dtype=torch.int32, device="cuda")
+        qd = dev(q)
+        ctx.chunk_step(qd, dev(k_chunk), dev(v_chunk), T, ob.units_to_device(cu), len(cu), k_a, v_a, n_hist_a, n, units_a,
+                       n_units_a, U, w_mod, params, page, 0.0, k_b, v_b, units_b, n_hist_b, n_units_b, o, ob.DTYPE_FP32,
+                       info_out=info)
+        torch.cuda.synchronize()
+        assert ctx.poll_status() == 0
+        # the scores the step used (the work buffers are not part of the ABI: the scoring call is repeated)
+        scores = torch.zeros((U,), dtype=torch.float32, device="cuda")
+        ctx.score_units(qd, T, k_a, n_hist_a, n, units_a, n_units_a, U, w_mod, 0.0, scores, None)
+        torch.cuda.synchronize()
+        gpu_scores = scores.cpu().numpy()
+        s_ref, _ = oc.score_units(q, k_cache, units, w_mod)
+        rel = np.abs(gpu_scores - s_ref) / np.maximum(np.abs(s_ref), 1e-3 * np.abs(s_ref).max())
+        assert rel.max() <= P.SCORE_REL, (c, rel.max())
+        st = oc.stream_step(q, k_cache, v_cache, units, k_chunk, v_chunk, cu, w_mod, budget, R, caps, page,
+                            scores_override=gpu_scores)
+        P._selection_matches(units, st["select"]["unit_keep"], gpu_scores, s_ref, budget, R, caps)
+        n_new = len(st["k_cache"])
+        assert int(n_hist_b.item()) == n_new and int(n_units_b.item()) == len(st["units"])
+        assert np.array_equal(units_b[:len(st["units"])].cpu().numpy(), st["units"])
+        got = ob.info_to_dict(info)
+        cp = st["compact"]
+        assert got["n_kept"] == cp["n_kept"] and got["span_pages"] == cp["span_pages"] and got["rows_moved"] == cp["rows_moved"]
+        assert got["span_pages"] * page - got["n_kept"] < page
+        for gpu_c, ref_c in ((k_b, st["k_cache"]), (v_b, st["v_cache"])):
+            bits = H.bytes_of(gpu_c[:n_new]).reshape(n_new, -1).view(np.uint16).reshape(n_new, h_kv, d)
+            assert np.array_equal(bits, wl.bf16_bits(ref_c))
+        P._check_attention(o.cpu().numpy(), None, st["o"], None)
+        evicted |= cp["n_kept"] < n
+        # advance both states
+        k_cache, v_cache, units = st["k_cache"], st["v_cache"], st["units"]
+        k_a, k_b, v_a, v_b = k_b, k_a, v_b, v_a
+        units_a, units_b = units_b, units_a
+        n_hist_a, n_hist_b, n_units_a, n_units_b = n_hist_b, n_hist_a, n_units_b, n_units_a
+    assert evicted, "the schedule never exceeded the budget: the test did not exercise eviction"
+    ctx.close()
