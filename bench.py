@@ -121,6 +121,89 @@ class ClockSampler:
         return out
 
 
+def max_over_ranks(values, world, device):
+    """Element-wise maximum of a list of floats over all ranks (the job is as slow as its slowest replica)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.tolist()]
+
+
+def whole_job(per_replica_value, world):
+    """Replicas only: every rank runs the same independent stream, so the job's throughput is the sum."""
+    return per_replica_value * world
+
+
+def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=64):
+    """The 36-layer stream loop (frames of {640, 1280, 2304} tokens plus 2 s of audio at 10-25 tok/s per
+    chunk): per chunk and per layer one omnitide_chunk_step on a device-resident cache.  Returns the
+    mean milliseconds per chunk over the chunks whose history already exceeds the budget (CUDA events
+    around the 36 layer steps of a chunk; the chunk's inputs are drawn on the device before its timed
+    region) and the physical span against the kept count."""
+    from paper_2609_34653_b200 import workloads as wl
+    sched = wl.loop_schedule(n_chunks)
+    h_q, h_kv, d, t_cap, u_cap = 32, 8, 128, 2432, 96
+    s_cap = ((budget + 2 * t_cap + 255) // 256) * 256
+    ctx = ob.Context(h_q, h_kv, d, "bf16", s_cap, u_cap, t_cap)
+    gen = torch.Generator(device="cuda").manual_seed(4000 + rank)
+    randn = lambda *shape: torch.randn(*shape, generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    prefix = wl.loop_prefix_units()
+    layers = []
+    for l in range(n_layers):
+        ka = torch.zeros((s_cap, h_kv, d), dtype=torch.bfloat16, device="cuda")
+        va = torch.zeros_like(ka)
+        ka[:16], va[:16] = randn(16, h_kv, d), randn(16, h_kv, d)
+        layers.append(dict(k=[ka, torch.zeros_like(ka)], v=[va, torch.zeros_like(va)],
+                           units=[ob.units_to_device(prefix, u_cap), torch.zeros((u_cap, 6), dtype=torch.int32, device="cuda")],
+                           n_hist=[torch.tensor([16], dtype=torch.int32, device="cuda"), torch.zeros(1, dtype=torch.int32, device="cuda")],
+                           n_units=[torch.tensor([1], dtype=torch.int32, device="cuda"), torch.zeros(1, dtype=torch.int32, device="cuda")],
+                           info=torch.zeros(8, dtype=torch.int32, device="cuda")))
+    params = ob.select_params(budget, 1, (-1, -1, -1))
+    w_mod = (1.0, 2.0, 2.0)
+    hist_bound, units_bound = 16, 1
+    o = torch.empty((t_cap, h_q, d), dtype=torch.float32, device="cuda")
+    rows = []
+    for c, cu in enumerate(sched):
+        T = int(cu[:, 1].sum())
+        cu_dev = ob.units_to_device(cu)
+        zs = torch.exp(0.5 * torch.randn(len(cu), generator=gen, device="cuda"))
+        tok_scale = torch.repeat_interleave(zs, torch.from_numpy(cu[:, 1].astype(np.int64)).cuda())[:, None, None]
+        ins = [(randn(T, h_q, d), (torch.randn(T, h_kv, d, generator=gen, device="cuda") * tok_scale).to(torch.bfloat16),
+                randn(T, h_kv, d)) for _ in range(n_layers)]
+        a, b = c & 1, (c & 1) ^ 1
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for l, L in enumerate(layers):
+            q, kc, vc = ins[l]
+            ctx.chunk_step(q, kc, vc, T, cu_dev, len(cu), L["k"][a], L["v"][a], L["n_hist"][a], hist_bound, L["units"][a],
+                           L["n_units"][a], units_bound, w_mod, params, page, 0.0, L["k"][b], L["v"][b], L["units"][b],
+                           L["n_hist"][b], L["n_units"][b], o, ob.DTYPE_FP32, info_out=L["info"])
+        e1.record()
+        torch.cuda.synchronize()
+        assert ctx.poll_status() == 0, "device status word not clean inside the stream loop"
+        infos = torch.stack([L["info"] for L in layers]).cpu().numpy()
+        n_hist_new = int(max(int(L["n_hist"][b].item()) for L in layers))
+        rows.append(dict(ms=e0.elapsed_time(e1), hist=hist_bound, t=T, kept=float(infos[:, 0].mean()),
+                         span=float(infos[:, 1].mean()) * page, evicting=bool((infos[:, 0] < hist_bound).any())))
+        hist_bound = n_hist_new
+        units_bound = int(max(int(L["n_units"][b].item()) for L in layers))
+    launches = ctx.launch_count()
+    ctx.close()
+    steady = [r for r in rows if r["evicting"]] or rows[-max(1, len(rows) // 2):]
+    return {"ms_per_chunk": float(np.mean([r["ms"] for r in steady])), "layers": n_layers, "chunks": len(rows),
+            "chunks_timed": len(steady), "budget": budget, "page": page,
+            "mean_chunk_tokens": float(np.mean([r["t"] for r in steady])),
+            "mean_history_tokens": float(np.mean([r["hist"] for r in steady])),
+            "kept_rows_mean": float(np.mean([r["kept"] for r in steady])),
+            "span_slots_mean": float(np.mean([r["span"] for r in steady])),
+            "span_over_kept": float(np.mean([r["span"] / max(r["kept"], 1.0) for r in steady])),
+            "gpu_launches": int(launches),
+            "note": "36 layer steps per chunk timed with CUDA events; chunks counted once the history exceeds the budget"}
+
+
 def run_reference(args, rank, world):
     """CPU oracle timed on a bounded sample of the same workload (rank 0 only)."""
     if rank != 0:
@@ -165,6 +248,7 @@ def main():
     ap.add_argument("--workload", default="long_stream")
     ap.add_argument("--sets", type=int, default=8, help="distinct cache sets rotated so the working set exceeds L2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--loop-chunks", type=int, default=24, help="chunks of the 36-layer stream loop (0: skip it)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -297,11 +381,8 @@ def main():
 
     # ---- max over ranks
     ms_per_step = total_ms / args.steps
-    vec = torch.tensor([ms_per_step, per["attention"], per["compact"], per["score"], per["select"], per["append"], e2e_ms],
-                       dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(vec, op=dist.ReduceOp.MAX)
-    ms_per_step, att_ms, cp_ms, sc_ms, sel_ms, app_ms, e2e_ms = [float(x) for x in vec.tolist()]
+    ms_per_step, att_ms, cp_ms, sc_ms, sel_ms, app_ms, e2e_ms = max_over_ranks(
+        [ms_per_step, per["attention"], per["compact"], per["score"], per["select"], per["append"], e2e_ms], world, "cuda")
 
     peaks, peak_kind = load_peaks()
     tensor_peak = peaks["bf16_tflops_sustained"] if "bf16_tflops_sustained" in peaks else peaks["bf16_tflops"]
@@ -330,7 +411,7 @@ def main():
     roofline.update(kernel=dominant, peak_source=f"{peak_kind} ({'sustained' if 'bf16_tflops_sustained' in peaks else 'burst'} bf16 matmul / copy bandwidth)")
 
     line = {
-        "metric": METRIC, "value": att_tf * world, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": whole_job(att_tf, world), "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": args.workload, "h_q": w.h_q, "h_kv": w.h_kv, "head_dim": w.d, "n_hist": N, "chunk": T,
@@ -345,6 +426,13 @@ def main():
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                 "note": "attention FLOPs of the step over the whole host-buffer pass (copies + 5 stages)"},
     }
+    ctx.close()
+    del sets
+    torch.cuda.empty_cache()
+    if args.loop_chunks > 0:
+        loop = run_stream_loop(ob, torch, args.loop_chunks, rank)
+        loop["ms_per_chunk"] = max_over_ranks([loop["ms_per_chunk"]], world, "cuda")[0]
+        line["stream_loop"] = loop
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import omni_oracle as oc
         import threadpoolctl
@@ -358,7 +446,6 @@ def main():
                                 "sample": f"attention of 1 of {w.h_kv} KV groups ({G} query heads), T={T}, kept history {kept}"}
     if rank == 0:
         print(json.dumps(line), flush=True)
-    ctx.close()
     if world > 1:
         dist.destroy_process_group()
 
