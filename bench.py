@@ -66,7 +66,8 @@ def algorithmic_work(w, n_kept):
         "score_flop": 2.0 * w.d * w.h_q * T * N,
         "score_exp": 1.0 * w.h_q * T * N,
         "attn_flop": 4.0 * w.d * w.h_q * (T * n_kept + T * (T + 1) / 2.0),
-        "compact_bytes": 2.0 * n_kept * 2 * row + N + 4.0 * N,        # rows (R+W, K and V) + mask + slot map
+        "compact_bytes": 2.0 * n_kept * 2 * row + 25.0 * len(w.units),     # rows (R+W, K and V) + unit table and keep codes
+        "compact_mask_bytes": 2.0 * n_kept * 2 * row + N + 4.0 * N,        # token-mask entry point: + mask + slot map
         "select_bytes": 24.0 * len(w.units) + 5.0 * N,
         "append_bytes": 2.0 * T * 2 * row,
     }
@@ -248,6 +249,8 @@ def main():
     ap.add_argument("--workload", default="long_stream")
     ap.add_argument("--sets", type=int, default=8, help="distinct cache sets rotated so the working set exceeds L2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--mask-compaction", action="store_true",
+                    help="time omnipage_compact (token keep mask + slot map) instead of the unit-granular entry point")
     ap.add_argument("--loop-chunks", type=int, default=24, help="chunks of the 36-layer stream loop (0: skip it)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -315,10 +318,17 @@ def main():
         rec(0)
         ctx.score_units(s["q"], T, s["k_in"], n_hist_dev, N, units_in, n_units_dev, U, w.w_modality, 0.0, scores)
         rec(1)
-        ctx.select_units(units_in, n_units_dev, U, scores, params, unit_keep, keep_mask, N, n_kept, units_out, n_units_kept)
-        rec(2)
-        ctx.compact(s["k_in"], s["v_in"], s["k_out"], s["v_out"], keep_mask, n_hist_dev, N, w.page_size, units_out,
-                    n_units_kept, U, slot_map, info, None)
+        if args.mask_compaction:
+            ctx.select_units(units_in, n_units_dev, U, scores, params, unit_keep, keep_mask, N, n_kept, units_out, n_units_kept)
+            rec(2)
+            ctx.compact(s["k_in"], s["v_in"], s["k_out"], s["v_out"], keep_mask, n_hist_dev, N, w.page_size, units_out,
+                        n_units_kept, U, slot_map, info, None)
+        else:
+            # the pass keeps the decision per unit between selection and compaction (as omnitide_chunk_step does)
+            ctx.select_units(units_in, n_units_dev, U, scores, params, unit_keep, None, N, n_kept, units_out, n_units_kept)
+            rec(2)
+            ctx.compact_units(s["k_in"], s["v_in"], s["k_out"], s["v_out"], units_in, n_units_dev, U, unit_keep, N,
+                              w.page_size, units_out, n_units_kept, None, info, None)
         rec(3)
         ctx.chunk_attention(s["q"], T, s["k_out"], s["v_out"], n_kept, N, s["kc"], s["vc"], 0.0, s["o"], ob.DTYPE_FP32)
         rec(4)
@@ -388,7 +398,8 @@ def main():
     tensor_peak = peaks["bf16_tflops_sustained"] if "bf16_tflops_sustained" in peaks else peaks["bf16_tflops"]
     att_tf = work["attn_flop"] / (att_ms * 1e-3) / 1e12
     sc_tf = work["score_flop"] / (sc_ms * 1e-3) / 1e12
-    cp_gbs = work["compact_bytes"] / (cp_ms * 1e-3) / 1e9
+    cp_bytes = work["compact_mask_bytes"] if args.mask_compaction else work["compact_bytes"]
+    cp_gbs = cp_bytes / (cp_ms * 1e-3) / 1e9
     traffic = NCU_TRAFFIC_BYTES.get(args.workload, {})
     xu_peak = XU_PER_CLK_PER_SM * N_SM * SM_MAX_MHZ * 1e6 / 1e12   # Texp/s
     sc_texp = work["score_exp"] / (sc_ms * 1e-3) / 1e12
@@ -401,6 +412,7 @@ def main():
                   "note": "bound by the exponential rate of the special-function pipe (16 per clock per SM at the max SM clock)"},
         "compact": {"bound": "hbm", "achieved": cp_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": cp_gbs / peaks["hbm_gbs"], "frac_of_nominal": cp_gbs / NOMINAL["hbm_gbs"], "ms": cp_ms,
+                    "entry": "omnipage_compact" if args.mask_compaction else "omnipage_compact_units",
                     "traffic": traffic.get("compact")},
         "select": {"bound": "latency", "ms": sel_ms, "achieved": work["select_bytes"] / (sel_ms * 1e-3) / 1e9, "unit": "GB/s"},
         "append": {"bound": "hbm", "ms": app_ms, "achieved": work["append_bytes"] / (app_ms * 1e-3) / 1e9,

@@ -172,6 +172,26 @@ omni_status omnipage_compact(omnitide_ctx* ctx, void* stream,
                              int32_t* slot_map_out, omni_compact_info* info_out, uint8_t* page_class_out);
 
 /*
+ * (a3, unit-granular form) The same eager pack when the keep decision is one code per UNIT, which is what
+ * omnitide_select_units produces (Section 5.1: spans are never cut at a token position; Section 5.2: the unit
+ * records carry the layout).  Equivalent to omnipage_compact with
+ *   keep_mask[s] = (unit_keep[unit that holds s] != OMNI_KEEP_DROPPED),   s_span = end of the last unit,
+ * but no mask is read: the gather is a list of at most n_units contiguous runs, so no CTA has to wait for
+ * another one's count and the kernel starts copying after one round trip to the unit table.
+ *   units [dev] the history unit table (contiguous, in order), n_units_dev [dev, nullable] / n_units_max [host];
+ *   unit_keep [dev] n_units_max bytes (OMNI_KEEP_*); s_span_max [host] bound on the history length;
+ *   units_kept / n_units_kept_dev: the re-indexed table of the survivors (for part_begin; nullable);
+ *   slot_map_out [dev] s_span_max int32 (nullable), info_out [dev], page_class_out [dev] nullable, as above.
+ * A unit that reaches outside [0, s_span_max) sets OMNI_DEV_BAD_UNITS and is treated as dropped.
+ */
+omni_status omnipage_compact_units(omnitide_ctx* ctx, void* stream,
+                                   const void* k_src, const void* v_src, void* k_dst, void* v_dst,
+                                   const omni_unit* units, const int32_t* n_units_dev, int32_t n_units_max,
+                                   const uint8_t* unit_keep, int32_t s_span_max, int32_t page_size,
+                                   const omni_unit* units_kept, const int32_t* n_units_kept_dev,
+                                   int32_t* slot_map_out, omni_compact_info* info_out, uint8_t* page_class_out);
+
+/*
  * (a5) Append: new entries enter the recent-context class behind the retained history
  * (Section 6.1).  Copies the chunk's t K/V rows to cache slots [n_kept, n_kept + t), appends the
  * chunk's units to `units` with start += n_kept and group = recent-context, and writes

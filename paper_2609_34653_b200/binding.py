@@ -37,7 +37,7 @@ class CompactInfo(C.Structure):
 
 EXPORTS = [
     "omnitide_create", "omnitide_destroy", "omnitide_poll_status", "omnitide_last_error",
-    "omnitide_score_units", "omnitide_select_units", "omnipage_compact", "omnipage_append",
+    "omnitide_score_units", "omnitide_select_units", "omnipage_compact", "omnipage_compact_units", "omnipage_append",
     "omnitide_chunk_attention", "omnitide_chunk_step", "omnitide_chunk_step_host",
     "omnitide_set_option", "omnitide_launch_count", "omnitide_score_units_noalloc",
 ]
@@ -174,6 +174,15 @@ class Context:
                                               _ptr(units_kept), _ptr(n_units_kept_dev), n_units_max,
                                               _ptr(slot_map_out), _ptr(info_out), _ptr(page_class_out)),
                     "omnipage_compact")
+
+    def compact_units(self, k_src, v_src, k_dst, v_dst, units, n_units_dev, n_units_max, unit_keep, s_span_max,
+                      page_size, units_kept, n_units_kept_dev, slot_map_out, info_out, page_class_out):
+        self._check(self.lib.omnipage_compact_units(self._ctx, _stream(), _ptr(k_src), _ptr(v_src), _ptr(k_dst),
+                                                    _ptr(v_dst), _ptr(units), _ptr(n_units_dev), n_units_max,
+                                                    _ptr(unit_keep), s_span_max, page_size, _ptr(units_kept),
+                                                    _ptr(n_units_kept_dev), _ptr(slot_map_out), _ptr(info_out),
+                                                    _ptr(page_class_out)),
+                    "omnipage_compact_units")
 
     def append(self, k_cache, v_cache, n_kept_dev, k_chunk, v_chunk, t, units, n_units_dev, chunk_units,
                n_chunk_units, n_hist_out, n_units_out):

@@ -175,12 +175,12 @@ extern "C" omni_status omnitide_chunk_step(omnitide_ctx* ctx, void* stream, cons
     s = omnitide_score_units(ctx, stream, q, t, k_cache, n_hist_dev, n_hist_max, units, n_units_dev, n_units_max,
                              w_modality, scale, ctx->ws_scores, nullptr);
     if (s) return s;
+    // the keep decision stays per unit between the two steps: no token mask, no slot map inside the pass
     s = omnitide_select_units(ctx, stream, units, n_units_dev, n_units_max, ctx->ws_scores, params, ctx->ws_unit_keep,
-                              ctx->ws_keep_mask, n_hist_max, n_kept, units_out, n_units_kept);
+                              nullptr, n_hist_max, n_kept, units_out, n_units_kept);
     if (s) return s;
-    s = omnipage_compact(ctx, stream, k_cache, v_cache, k_cache_out, v_cache_out, ctx->ws_keep_mask, n_hist_dev,
-                         n_hist_max, page_size, OMNI_COMPACT_PACK, units_out, n_units_kept, n_units_max, ctx->ws_slot_map,
-                         info, nullptr);
+    s = omnipage_compact_units(ctx, stream, k_cache, v_cache, k_cache_out, v_cache_out, units, n_units_dev, n_units_max,
+                               ctx->ws_unit_keep, n_hist_max, page_size, units_out, n_units_kept, nullptr, info, nullptr);
     if (s) return s;
     s = omnitide_chunk_attention(ctx, stream, q, t, k_cache_out, v_cache_out, n_kept, n_hist_max, k_chunk, v_chunk, scale,
                                  o_out, out_dtype, nullptr);

@@ -197,6 +197,79 @@ __device__ __forceinline__ unsigned long long ld_relaxed_gpu(const unsigned long
     return v;
 }
 
+// Moves destination rows [d0, d0 + n_rows) of this CTA; src_list[r] is the source slot of row d0 + r.
+template <class Args>
+__device__ __forceinline__ void move_rows(const Args& a, const int* src_list, const int d0, const int n_rows, char* rowbuf,
+                                          uint64_t (*cbar)[CP_MAX_SLOTS], int* abort_flag_p) {
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    if (a.n_slots > 0) {
+        // bulk-copy path: lane 0 of every warp streams its rows HBM -> shared memory -> HBM with
+        // cp.async.bulk, `n_slots` rows in flight per warp; no per-vector instructions at all.
+        if (lane == 0) {
+            const int n_copies = 2 * n_rows;                         // copy i: row i >> 1, K (even) or V (odd)
+            const int mcp = n_copies > wid ? (n_copies - wid + CP_WARPS - 1) / CP_WARPS : 0;
+            const uint32_t buf0 = tc::smem_u32(rowbuf) + (uint32_t)(wid * a.n_slots) * a.row_bytes;
+            auto src_of = [&](int q) {
+                const int i = wid + q * CP_WARPS;
+                return ((i & 1) ? a.v_src : a.k_src) + (size_t)src_list[i >> 1] * a.row_bytes;
+            };
+            auto dst_of = [&](int q) {
+                const int i = wid + q * CP_WARPS;
+                return ((i & 1) ? a.v_dst : a.k_dst) + (size_t)(d0 + (i >> 1)) * a.row_bytes;
+            };
+            auto issue_load = [&](int q) {
+                const int slot = q % a.n_slots;
+                const uint32_t bar = tc::smem_u32(&cbar[wid][slot]);
+                tc::mbar_expect_tx(bar, a.row_bytes);
+                bulk_load(buf0 + slot * a.row_bytes, src_of(q), a.row_bytes, bar);
+            };
+            for (int q = 0; q < mcp && q < a.n_slots; ++q) issue_load(q);
+            bool ok = true;
+            for (int q = 0; q < mcp && ok; ++q) {
+                const int slot = q % a.n_slots;
+                ok = tc::mbar_wait(tc::smem_u32(&cbar[wid][slot]), (q / a.n_slots) & 1, abort_flag_p);
+                if (!ok) break;
+                bulk_store(dst_of(q), buf0 + slot * a.row_bytes, a.row_bytes);
+                // the buffer of copy q-1 is free once its store has read it: refill it
+                if (q >= 1 && q - 1 + a.n_slots < mcp) {
+                    asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    issue_load(q - 1 + a.n_slots);
+                }
+            }
+            asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+            if (!ok) atomicOr(a.status, OMNI_DEV_TIMEOUT);
+        }
+        return;
+    }
+    // vector path (rows too large for the buffers, or too small to be worth a bulk copy)
+    const int total = n_rows * 2 * a.vpr;                    // (row, K or V, vector)
+    for (int base = tid; base < total; base += CP_THREADS * CP_BATCH) {
+        uint4 buf[CP_BATCH];
+#pragma unroll
+        for (int u = 0; u < CP_BATCH; ++u) {
+            const int idx = base + u * CP_THREADS;
+            if (idx < total) {
+                int rw, v;
+                if (a.vpr_shift >= 0) { rw = idx >> a.vpr_shift; v = idx & (a.vpr - 1); }
+                else { rw = idx / a.vpr; v = idx - rw * a.vpr; }
+                const size_t so = (size_t)src_list[rw >> 1] * a.row_bytes + (size_t)v * 16;
+                buf[u] = ld_stream(reinterpret_cast<const uint4*>(((rw & 1) ? a.v_src : a.k_src) + so));
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < CP_BATCH; ++u) {
+            const int idx = base + u * CP_THREADS;
+            if (idx < total) {
+                int rw, v;
+                if (a.vpr_shift >= 0) { rw = idx >> a.vpr_shift; v = idx & (a.vpr - 1); }
+                else { rw = idx / a.vpr; v = idx - rw * a.vpr; }
+                const size_t dof = (size_t)(d0 + (rw >> 1)) * a.row_bytes + (size_t)v * 16;
+                st_stream(reinterpret_cast<uint4*>(((rw & 1) ? a.v_dst : a.k_dst) + dof), buf[u]);
+            }
+        }
+    }
+}
+
 // 16 mask bytes at slot `pos` (a multiple of 16) with the bytes at and beyond s zeroed
 __device__ __forceinline__ uint4 mask_at(const uint8_t* mask, int pos, int s) {
     uint4 v = make_uint4(0, 0, 0, 0);
@@ -418,73 +491,143 @@ __global__ void __launch_bounds__(CP_THREADS, 1) compact_pack_kernel(const Compa
     if (a.k_dst == nullptr) return;
     __syncthreads();                                        // the source list is complete
 
-    // ---- phase C: move the rows ---------------------------------------------------------------------
-    if (a.n_slots > 0) {
-        // bulk-copy path: lane 0 of every warp streams its rows HBM -> shared memory -> HBM with
-        // cp.async.bulk, `n_slots` rows in flight per warp; no per-vector instructions at all.
-        if (lane == 0) {
-            const int n_copies = 2 * n_rows;                         // copy i: row i >> 1, K (even) or V (odd)
-            const int mcp = n_copies > wid ? (n_copies - wid + CP_WARPS - 1) / CP_WARPS : 0;
-            const uint32_t buf0 = tc::smem_u32(rowbuf) + (uint32_t)(wid * a.n_slots) * a.row_bytes;
-            auto src_of = [&](int q) {
-                const int i = wid + q * CP_WARPS;
-                return ((i & 1) ? a.v_src : a.k_src) + (size_t)src_list[i >> 1] * a.row_bytes;
-            };
-            auto dst_of = [&](int q) {
-                const int i = wid + q * CP_WARPS;
-                return ((i & 1) ? a.v_dst : a.k_dst) + (size_t)(d0 + (i >> 1)) * a.row_bytes;
-            };
-            auto issue_load = [&](int q) {
-                const int slot = q % a.n_slots;
-                const uint32_t bar = tc::smem_u32(&cbar[wid][slot]);
-                tc::mbar_expect_tx(bar, a.row_bytes);
-                bulk_load(buf0 + slot * a.row_bytes, src_of(q), a.row_bytes, bar);
-            };
-            for (int q = 0; q < mcp && q < a.n_slots; ++q) issue_load(q);
-            bool ok = true;
-            for (int q = 0; q < mcp && ok; ++q) {
-                const int slot = q % a.n_slots;
-                ok = tc::mbar_wait(tc::smem_u32(&cbar[wid][slot]), (q / a.n_slots) & 1, &abort_flag);
-                if (!ok) break;
-                bulk_store(dst_of(q), buf0 + slot * a.row_bytes, a.row_bytes);
-                // the buffer of copy q-1 is free once its store has read it: refill it
-                if (q >= 1 && q - 1 + a.n_slots < mcp) {
-                    asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                    issue_load(q - 1 + a.n_slots);
-                }
-            }
-            asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-            if (!ok) atomicOr(a.status, OMNI_DEV_TIMEOUT);
-        }
-        return;
+    move_rows(a, src_list, d0, n_rows, rowbuf, cbar, &abort_flag);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Unit-granular compaction: the keep decision is one code per unit, so the gather is a list of at most
+// n_units contiguous runs and no mask is read.  No CTA needs anything from another: every CTA loads the
+// unit table (one round trip), scans the kept lengths, takes its share of the destination rows and
+// starts copying.
+struct CompactUnitsArgs {
+    const char* k_src; const char* v_src; char* k_dst; char* v_dst;
+    const omni_unit* units; const int32_t* n_units_dev; int n_units_max; const uint8_t* unit_keep;
+    int s_span_max; int page_size; int row_bytes; int vpr; int vpr_shift;
+    const omni_unit* units_kept; const int32_t* n_units_kept_dev;
+    int32_t* slot_map; omni_compact_info* info; uint8_t* page_class; int32_t* status;
+    int rows_cap; int n_slots;
+};
+
+__global__ void __launch_bounds__(CP_THREADS, 1) compact_units_kernel(const CompactUnitsArgs a) {
+    extern __shared__ __align__(128) int smem_i[];
+    int* ustart = smem_i;                                   // [n_units_max]
+    int* ulen = smem_i + a.n_units_max;                     // [n_units_max]: 0 for a unit outside the span
+    int* prefix = smem_i + 2 * a.n_units_max;               // [n_units_max + 1]: kept lengths, then their exclusive scan
+    int* src_list = prefix + a.n_units_max + 8;             // [rows_cap]
+    char* rowbuf = reinterpret_cast<char*>(smem_i) + ((((size_t)3 * a.n_units_max + 8 + a.rows_cap) * sizeof(int) + 127) & ~(size_t)127);
+    __shared__ int warp_tot[CP_WARPS + 1];
+    __shared__ int s_misc[4];
+    __shared__ uint64_t cbar[CP_WARPS][CP_MAX_SLOTS];
+    __shared__ int abort_flag;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int G = gridDim.x;
+
+    // ---- prologue: all loads that need no device-side count first ------------------------------------------
+    int nu = a.n_units_dev ? __ldg(a.n_units_dev) : a.n_units_max;
+    int u_start = 0, u_len = 0, u_keep = 0, k_len = 0, k_group = -1;
+    if (tid < a.n_units_max) {
+        u_start = __ldg(&a.units[tid].start);
+        u_len = __ldg(&a.units[tid].len);
+        u_keep = __ldg(a.unit_keep + tid);
     }
-    // vector path (rows too large for the buffers, or too small to be worth a bulk copy)
-    const int total = n_rows * 2 * a.vpr;                    // (row, K or V, vector)
-    for (int base = tid; base < total; base += CP_THREADS * CP_BATCH) {
-        uint4 buf[CP_BATCH];
-#pragma unroll
-        for (int u = 0; u < CP_BATCH; ++u) {
-            const int idx = base + u * CP_THREADS;
-            if (idx < total) {
-                int rw, v;
-                if (a.vpr_shift >= 0) { rw = idx >> a.vpr_shift; v = idx & (a.vpr - 1); }
-                else { rw = idx / a.vpr; v = idx - rw * a.vpr; }
-                const size_t so = (size_t)src_list[rw >> 1] * a.row_bytes + (size_t)v * 16;
-                buf[u] = ld_stream(reinterpret_cast<const uint4*>(((rw & 1) ? a.v_src : a.k_src) + so));
-            }
+    int nuk = 0;
+    if (a.units_kept) {
+        nuk = a.n_units_kept_dev ? __ldg(a.n_units_kept_dev) : a.n_units_max;
+        if (tid < a.n_units_max) { k_len = __ldg(&a.units_kept[tid].len); k_group = __ldg(&a.units_kept[tid].group); }
+    }
+    if (tid == 0) { s_misc[0] = 0; s_misc[1] = 0; s_misc[2] = 0x7fffffff; s_misc[3] = 0; abort_flag = 0; }
+    if (lane == 0 && a.n_slots > 0) {
+        for (int q = 0; q < a.n_slots; ++q) tc::mbar_init(tc::smem_u32(&cbar[wid][q]), 1);
+        tc::fence_barrier_init();
+    }
+    __syncthreads();
+    if (nu < 0 || nu > a.n_units_max) {
+        if (tid == 0 && blockIdx.x == 0) atomicOr(a.status, OMNI_DEV_BAD_COUNT);
+        nu = max(0, min(nu, a.n_units_max));
+    }
+    nuk = max(0, min(nuk, a.n_units_max));
+    // kept length per unit; a unit outside [0, s_span_max) is an error and counts as dropped
+    bool bad = false;
+    for (int u = tid; u < nu; u += CP_THREADS) {
+        if (u >= CP_THREADS) { u_start = a.units[u].start; u_len = a.units[u].len; u_keep = a.unit_keep[u]; }
+        const bool inside = u_start >= 0 && u_len > 0 && (long long)u_start + u_len <= a.s_span_max;
+        bad |= !inside;
+        const bool keep = inside && u_keep != OMNI_KEEP_DROPPED;
+        ustart[u] = u_start;
+        ulen[u] = inside ? u_len : 0;
+        prefix[u] = keep ? u_len : 0;
+        if (!keep) atomicMin(&s_misc[2], u);                 // first unit that is dropped (for rows_moved)
+        if (u == nu - 1) s_misc[3] = inside ? u_start + u_len : 0;   // end of the history
+    }
+    if (bad) atomicOr(a.status, OMNI_DEV_BAD_UNITS);
+    {
+        int p0 = 0, p1 = 0;
+        for (int u = tid; u < nuk; u += CP_THREADS) {
+            if (u >= CP_THREADS) { k_len = a.units_kept[u].len; k_group = a.units_kept[u].group; }
+            if (k_group == OMNI_GROUP_MUST_KEEP) p0 += k_len;
+            else if (k_group == OMNI_GROUP_SELECTED) p1 += k_len;
         }
-#pragma unroll
-        for (int u = 0; u < CP_BATCH; ++u) {
-            const int idx = base + u * CP_THREADS;
-            if (idx < total) {
-                int rw, v;
-                if (a.vpr_shift >= 0) { rw = idx >> a.vpr_shift; v = idx & (a.vpr - 1); }
-                else { rw = idx / a.vpr; v = idx - rw * a.vpr; }
-                const size_t dof = (size_t)(d0 + (rw >> 1)) * a.row_bytes + (size_t)v * 16;
-                st_stream(reinterpret_cast<uint4*>(((rw & 1) ? a.v_dst : a.k_dst) + dof), buf[u]);
-            }
+        p0 = __reduce_add_sync(0xffffffffu, p0);
+        p1 = __reduce_add_sync(0xffffffffu, p1);
+        if (lane == 0 && (p0 | p1)) { atomicAdd(&s_misc[0], p0); atomicAdd(&s_misc[1], p1); }
+    }
+    if (tid == 0) prefix[nu] = 0;
+    __syncthreads();
+    const int n_kept = block_excl_scan(prefix, nu, warp_tot);
+    const int n0 = s_misc[0], n1 = s_misc[1], u_open = s_misc[2], n_hist = s_misc[3];
+
+    // ---- destination share: the source slot of every row by a search over the scanned lengths --------------
+    const int rows_per = (n_kept + G - 1) / G;
+    const int d0 = min(n_kept, (int)blockIdx.x * rows_per);
+    const int d1 = min(n_kept, d0 + rows_per);
+    const int n_rows = min(d1 - d0, a.rows_cap);
+    for (int r = tid; r < n_rows; r += CP_THREADS) {
+        const int dd = d0 + r;
+        int lo = 0, hi = nu;                                 // largest u with prefix[u] <= dd (its kept length is > 0)
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (prefix[mid] <= dd) lo = mid; else hi = mid;
+        }
+        src_list[r] = ustart[lo] + (dd - prefix[lo]);
+    }
+    // ---- slot map (optional): unit u belongs to CTA u % G -----------------------------------------------------
+    if (a.slot_map) {
+        for (int u = blockIdx.x; u < nu; u += G) {
+            const int st = ustart[u], ln = ulen[u];
+            const bool keep = prefix[u + 1] > prefix[u];
+            const int base = prefix[u];
+            for (int i = tid; i < ln; i += CP_THREADS) a.slot_map[st + i] = keep ? base + i : -1;
         }
     }
+    // ---- integer summary and page classes ------------------------------------------------------------------
+    if (a.info && blockIdx.x == 0 && tid == 0) {
+        const int lead = u_open < nu ? ustart[u_open] : n_hist;      // retained rows before the first dropped slot
+        a.info->n_kept = n_kept;
+        a.info->span_pages = (n_kept + a.page_size - 1) / a.page_size;
+        a.info->rows_moved = n_kept - min(lead, n_kept);
+        a.info->part_begin[0] = 0;
+        a.info->part_begin[1] = a.units_kept ? n0 : 0;
+        a.info->part_begin[2] = a.units_kept ? n0 + n1 : 0;
+        a.info->part_begin[3] = n_kept;
+        a.info->reserved = 0;
+    }
+    if (a.page_class) {
+        const int n_pages = (a.s_span_max + a.page_size - 1) / a.page_size;
+        for (int p = blockIdx.x * CP_THREADS + tid; p < n_pages; p += G * CP_THREADS) {
+            const long long lo = (long long)p * a.page_size;
+            const long long hi = min(lo + a.page_size, (long long)n_kept);
+            uint8_t cls = OMNI_PAGE_EMPTY;
+            if (hi > lo) {
+                if (lo < n0) cls = OMNI_GROUP_MUST_KEEP;
+                else if (hi - lo == a.page_size) cls = OMNI_GROUP_SELECTED;
+                else cls = OMNI_GROUP_RECENT;
+            }
+            a.page_class[p] = cls;
+        }
+    }
+    if (a.k_dst == nullptr) return;
+    __syncthreads();                                        // the source list is complete
+    move_rows(a, src_list, d0, n_rows, rowbuf, cbar, &abort_flag);
 }
 
 // Dense copy of `n_rows` rows (device count) from staging back to the cache (in-place mode), and
@@ -545,6 +688,19 @@ __global__ void append_units_kernel(omni_unit* units, const int32_t* n_units_dev
 
 }  // namespace
 
+// Staging rows of the in-place mode, allocated on the first in-place call on a context (synchronous).
+static omni_status omni_inplace_staging(omnitide_ctx* ctx) {
+    if (ctx->inplace_rows >= (size_t)ctx->g.s_cap) return OMNI_OK;
+    if (ctx->inplace_k) cudaFree(ctx->inplace_k);
+    if (ctx->inplace_v) cudaFree(ctx->inplace_v);
+    ctx->inplace_k = ctx->inplace_v = nullptr;
+    ctx->inplace_rows = 0;
+    OMNI_CUDA(ctx, cudaMalloc(&ctx->inplace_k, (size_t)ctx->g.s_cap * ctx->row_bytes));
+    OMNI_CUDA(ctx, cudaMalloc(&ctx->inplace_v, (size_t)ctx->g.s_cap * ctx->row_bytes));
+    ctx->inplace_rows = ctx->g.s_cap;
+    return OMNI_OK;
+}
+
 extern "C" omni_status omnipage_compact(omnitide_ctx* ctx, void* stream, const void* k_src, const void* v_src,
                                         void* k_dst, void* v_dst, const uint8_t* keep_mask,
                                         const int32_t* s_span_dev, int32_t s_span_max, int32_t page_size, int32_t mode,
@@ -568,16 +724,8 @@ extern "C" omni_status omnipage_compact(omnitide_ctx* ctx, void* stream, const v
     void* kd = k_dst;
     void* vd = v_dst;
     if (in_place) {
-        if (ctx->inplace_rows < (size_t)ctx->g.s_cap) {
-            // first in-place call on this context: allocate the staging rows (synchronous)
-            if (ctx->inplace_k) cudaFree(ctx->inplace_k);
-            if (ctx->inplace_v) cudaFree(ctx->inplace_v);
-            ctx->inplace_k = ctx->inplace_v = nullptr;
-            ctx->inplace_rows = 0;
-            OMNI_CUDA(ctx, cudaMalloc(&ctx->inplace_k, (size_t)ctx->g.s_cap * ctx->row_bytes));
-            OMNI_CUDA(ctx, cudaMalloc(&ctx->inplace_v, (size_t)ctx->g.s_cap * ctx->row_bytes));
-            ctx->inplace_rows = ctx->g.s_cap;
-        }
+        const omni_status ss = omni_inplace_staging(ctx);
+        if (ss) return ss;
         kd = ctx->inplace_k;
         vd = ctx->inplace_v;
     }
@@ -625,6 +773,69 @@ extern "C" omni_status omnipage_compact(omnitide_ctx* ctx, void* stream, const v
     }
     if (in_place) {
         if (!info_out) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "compact: in-place mode needs info_out");
+        copy_rows_kernel<<<ctx->sm_count * 4, 256, 0, st>>>(
+            static_cast<const char*>(kd), static_cast<const char*>(vd), static_cast<char*>(k_dst),
+            static_cast<char*>(v_dst), &info_out->n_kept, s_span_max, nullptr, ctx->g.s_cap, (int)ctx->row_bytes,
+            ctx->status_dev);
+        OMNI_CHECK_LAUNCH(ctx, "copy_rows_kernel");
+    }
+    return OMNI_OK;
+}
+
+extern "C" omni_status omnipage_compact_units(omnitide_ctx* ctx, void* stream, const void* k_src, const void* v_src,
+                                              void* k_dst, void* v_dst, const omni_unit* units,
+                                              const int32_t* n_units_dev, int32_t n_units_max, const uint8_t* unit_keep,
+                                              int32_t s_span_max, int32_t page_size, const omni_unit* units_kept,
+                                              const int32_t* n_units_kept_dev, int32_t* slot_map_out,
+                                              omni_compact_info* info_out, uint8_t* page_class_out) {
+    if (!ctx) return OMNI_ERR_INVALID_ARG;
+    if (!units || !unit_keep || n_units_max <= 0 || s_span_max < 0 || page_size <= 0)
+        OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "compact_units: bad unit table/span/page");
+    if (s_span_max > ctx->g.s_cap) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "compact_units: s_span_max %d > s_cap %d", s_span_max, ctx->g.s_cap);
+    if (n_units_max > ctx->g.u_cap) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "compact_units: n_units_max > u_cap");
+    if ((k_src == nullptr) != (k_dst == nullptr) || (k_src == nullptr) != (v_src == nullptr) ||
+        (v_src == nullptr) != (v_dst == nullptr))
+        OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "compact_units: K/V source and destination must be given together");
+    if (!omni_aligned16(k_src) || !omni_aligned16(v_src) || !omni_aligned16(k_dst) || !omni_aligned16(v_dst))
+        OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "compact_units: pointers must be 16-byte aligned");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool in_place = k_src && (k_src == k_dst || v_src == v_dst);
+    void* kd = k_dst;
+    void* vd = v_dst;
+    if (in_place) {
+        if (!info_out) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "compact_units: in-place mode needs info_out");
+        const omni_status ss = omni_inplace_staging(ctx);
+        if (ss) return ss;
+        kd = ctx->inplace_k;
+        vd = ctx->inplace_v;
+    }
+    CompactUnitsArgs a;
+    a.k_src = static_cast<const char*>(k_src); a.v_src = static_cast<const char*>(v_src);
+    a.k_dst = static_cast<char*>(kd); a.v_dst = static_cast<char*>(vd);
+    a.units = units; a.n_units_dev = n_units_dev; a.n_units_max = n_units_max; a.unit_keep = unit_keep;
+    a.s_span_max = s_span_max; a.page_size = page_size; a.row_bytes = (int)ctx->row_bytes;
+    a.vpr = (int)(ctx->row_bytes >> 4); a.vpr_shift = -1;
+    for (int sft = 0; sft < 20; ++sft) if ((1 << sft) == a.vpr) a.vpr_shift = sft;
+    a.units_kept = units_kept; a.n_units_kept_dev = n_units_kept_dev;
+    a.slot_map = slot_map_out; a.info = info_out; a.page_class = page_class_out; a.status = ctx->status_dev;
+    const int grid = ctx->sm_count;
+    a.rows_cap = (((s_span_max + grid - 1) / grid + 1) + 3) & ~3;
+    const size_t smem_lists = ((size_t)3 * n_units_max + 8 + a.rows_cap) * sizeof(int);
+    const size_t smem_lists_al = (smem_lists + 127) & ~(size_t)127;
+    const size_t budget = 200 * 1024;
+    if (smem_lists_al > budget) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "compact_units: unit table too large for one launch");
+    a.n_slots = 0;
+    if (k_src && ctx->row_bytes >= 512) {
+        const size_t per_warp = (budget - smem_lists_al) / CP_WARPS;
+        a.n_slots = (int)std::min<size_t>(CP_MAX_SLOTS, per_warp / ctx->row_bytes);
+        if (a.n_slots < 2) a.n_slots = 0;
+    }
+    const size_t smem = smem_lists_al + (size_t)a.n_slots * CP_WARPS * ctx->row_bytes;
+    if (smem > 48 * 1024)
+        OMNI_CUDA(ctx, cudaFuncSetAttribute(compact_units_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    compact_units_kernel<<<grid, CP_THREADS, smem, st>>>(a);
+    OMNI_CHECK_LAUNCH(ctx, "compact_units_kernel");
+    if (in_place) {
         copy_rows_kernel<<<ctx->sm_count * 4, 256, 0, st>>>(
             static_cast<const char*>(kd), static_cast<const char*>(vd), static_cast<char*>(k_dst),
             static_cast<char*>(v_dst), &info_out->n_kept, s_span_max, nullptr, ctx->g.s_cap, (int)ctx->row_bytes,

@@ -97,3 +97,33 @@ def gpu_attention(ctx, w, k_hist, v_hist, n_hist, out_fp32=True, n_hist_max=None
 
 def bytes_of(t):
     return t.contiguous().view(torch.uint8).cpu().numpy()
+
+
+def gpu_compact_units(ctx, k, v, units_np, unit_keep_np, page, units_out_np=None, in_place=False, s_span_max=None,
+                      u_max=None, want_slot_map=True):
+    """omnipage_compact_units on a history unit table and one keep code per unit."""
+    U = len(units_np)
+    S = int(units_np[:, 1].sum()) if U else 0
+    smax = s_span_max or S
+    umax = u_max or max(U, 1)
+    du = ob.units_to_device(units_np, umax)
+    keep = torch.full((umax + 16,), 2, dtype=torch.uint8, device="cuda")      # stale codes beyond n_units are ignored
+    if U:
+        keep[:U] = torch.from_numpy(np.asarray(unit_keep_np, dtype=np.uint8)).cuda()
+    kd = k if in_place else torch.full_like(k, 0)
+    vd = v if in_place else torch.full_like(v, 0)
+    slot_map = torch.full((smax + 16,), -5, dtype=torch.int32, device="cuda") if want_slot_map else None
+    info = torch.full((8,), -5, dtype=torch.int32, device="cuda")
+    n_pages = (smax + page - 1) // page
+    page_class = torch.full((n_pages + 16,), 7, dtype=torch.uint8, device="cuda")
+    dk = nk = None
+    if units_out_np is not None and len(units_out_np):
+        dk = ob.units_to_device(units_out_np, umax)
+        nk = i32(len(units_out_np))
+    ctx.compact_units(k, v, kd, vd, du, i32(U), umax, keep, smax, page, dk, nk, slot_map, info, page_class)
+    torch.cuda.synchronize()
+    status = ctx.poll_status()
+    out = ob.info_to_dict(info)
+    out.update(k=kd, v=vd, slot_map=slot_map[:S].cpu().numpy() if want_slot_map else None,
+               page_class=page_class[:n_pages].cpu().numpy(), status=status)
+    return out

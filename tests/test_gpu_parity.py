@@ -103,6 +103,77 @@ def test_compact_edges_and_partitions(H, ob):
     ctx.close()
 
 
+@pytest.mark.parametrize("U,max_len,rowshape,dtype,page,density,seed", [
+    (1, 40, (1, 64), torch.float32, 16, 1.0, 0),
+    (12, 300, (2, 64), torch.bfloat16, 16, 0.5, 1),
+    (70, 2400, (8, 128), torch.bfloat16, 64, 0.15, 2),
+    (600, 90, (8, 128), torch.bfloat16, 256, 0.5, 3),         # more units than threads in a CTA
+    (37, 1000, (8, 128), torch.bfloat16, 64, 0.0, 4),          # nothing kept
+])
+@pytest.mark.parametrize("in_place", [False, True])
+def test_compact_units_bit_exact(H, ob, U, max_len, rowshape, dtype, page, density, seed, in_place):
+    """The unit-granular entry point equals the oracle's pack of the equivalent token mask, bit for bit."""
+    rng = np.random.default_rng(100 + seed)
+    units = _random_table(rng, U) if U > 1 else wl.make_units([(int(max_len), 0, 0)])
+    if U > 1:
+        units[:, 1] = rng.integers(1, max_len + 1, size=U)
+        units[:, 0] = np.concatenate([[0], np.cumsum(units[:-1, 1])])
+    S = int(units[:, 1].sum())
+    keep_u = np.where(rng.random(U) < density, 2, 0).astype(np.uint8)
+    mask = np.repeat(keep_u != 0, units[:, 1]).astype(np.uint8)
+    es = 2 if dtype == torch.bfloat16 else 4
+    raw = rng.integers(0, 256, size=(2, S, rowshape[0] * rowshape[1] * es), dtype=np.uint8)
+    k = torch.from_numpy(raw[0]).cuda().view(dtype).view(S, *rowshape).contiguous()
+    v = torch.from_numpy(raw[1]).cuda().view(dtype).view(S, *rowshape).contiguous()
+    # the survivors' table as the selection step writes it (start = kept tokens before the unit)
+    kept_idx = np.nonzero(keep_u)[0]
+    units_out = units[kept_idx].copy()
+    if len(units_out):
+        units_out[:, 0] = np.concatenate([[0], np.cumsum(units_out[:-1, 1])])
+        idx = np.arange(len(units_out))
+        units_out[:, 4] = np.where(idx == 0, 0, np.where(idx < (2 * len(units_out)) // 3, 1, 2))   # ordered groups
+    exp = oc.compact_pack(raw[0], raw[1], mask, page, units_out if len(units_out) else None)
+    ctx = ob.Context(4 * rowshape[0], rowshape[0], rowshape[1], "bf16" if es == 2 else "fp32", S + 64, U + 8, 16)
+    got = H.gpu_compact_units(ctx, k, v, units, keep_u, page, units_out_np=units_out, in_place=in_place, s_span_max=S + 40,
+                              u_max=U + 5)
+    assert got["status"] == 0
+    n = exp["n_kept"]
+    assert (got["n_kept"], got["span_pages"], got["rows_moved"]) == (n, exp["span_pages"], exp["rows_moved"])
+    assert np.array_equal(got["slot_map"], exp["slot_map"])
+    if n:
+        assert np.array_equal(H.bytes_of(got["k"][:n]).reshape(n, -1), exp["k"])
+        assert np.array_equal(H.bytes_of(got["v"][:n]).reshape(n, -1), exp["v"])
+    if len(units_out):
+        assert got["part_begin"] == exp["part_begin"].tolist()
+    n_pages = (S + 40 + page - 1) // page
+    exp_pc = np.full(n_pages, 255, np.uint8)
+    exp_pc[:len(exp["page_class"])] = exp["page_class"]
+    assert np.array_equal(got["page_class"], exp_pc)
+    # and it agrees with the mask entry point on the same decision
+    if not in_place:
+        got_m = H.gpu_compact(ctx, k, v, mask, page, units_out_np=units_out if len(units_out) else None)
+        assert np.array_equal(H.bytes_of(got_m["k"][:n]), H.bytes_of(got["k"][:n]))
+        assert np.array_equal(H.bytes_of(got_m["v"][:n]), H.bytes_of(got["v"][:n]))
+    ctx.close()
+
+
+def test_compact_units_rejects_bad_tables(H, ob):
+    rng = np.random.default_rng(5)
+    units = wl.make_units([(100, 0, 0), (50, 1, 1), (70, 0, 2)])
+    S = 220
+    k = torch.from_numpy(rng.standard_normal((S, 2, 64)).astype(np.float32)).cuda()
+    v = torch.from_numpy(rng.standard_normal((S, 2, 64)).astype(np.float32)).cuda()
+    ctx = ob.Context(4, 2, 64, "fp32", 512, 16, 16)
+    bad = units.copy()
+    bad[2, 1] = 4000                                          # reaches outside the span: flagged, treated as dropped
+    got = H.gpu_compact_units(ctx, k, v, bad, np.array([2, 0, 2], np.uint8), 16, s_span_max=S)
+    assert got["status"] & 2 and got["n_kept"] == 100
+    with pytest.raises(ob.OmniTideError):
+        ctx.compact_units(k, v, torch.empty_like(k), torch.empty_like(v), None, None, 3, None, S, 16, None, None, None,
+                          None, None)
+    ctx.close()
+
+
 # ------------------------------------------------------------------------------------- selection
 def _random_table(rng, U):
     lens = rng.integers(1, 400, size=U)
