@@ -360,6 +360,15 @@ def main():
     per = {n: float(np.mean([evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(args.steps)]))
            for j, n in enumerate(names)}
     assert ctx.poll_status() == 0, "device status word not clean after the timed region"
+    # what two CUDA events measure with nothing between them, behind a running kernel (the floor every
+    # per-kernel time above carries; a kernel launch adds about as much again)
+    floor_evs = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(20)]
+    for a_, b_ in floor_evs:
+        torch.cuda._sleep(200000)
+        a_.record()
+        b_.record()
+    torch.cuda.synchronize()
+    event_pair_floor_ms = float(np.mean([a_.elapsed_time(b_) for a_, b_ in floor_evs]))
 
     # ---- end to end through the host-buffer entry point: chunk H2D and output D2H inside the timed region
     hq = torch.from_numpy(w.q).to(tdt).contiguous().pin_memory()
@@ -433,6 +442,8 @@ def main():
         "attention_tflops": att_tf * world, "compaction_gbs": cp_gbs * world, "score_tflops": sc_tf * world,
         "ms_per_chunk": ms_per_step, "span_slots": ((kept + w.page_size - 1) // w.page_size) * w.page_size,
         "kept_rows": kept,
+        "timing_floor": {"empty_event_pair_ms": event_pair_floor_ms,
+                         "note": "two CUDA events recorded back to back; every per-kernel time includes this plus the launch latency"},
         "kernels": kernels, "roofline": roofline, "clocks": clocks, "gpu_launches": int(gpu_launches),
         "e2e": {"value": work["attn_flop"] * world / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_chunk": e2e_ms,
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),

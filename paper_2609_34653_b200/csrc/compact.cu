@@ -571,9 +571,24 @@ __global__ void __launch_bounds__(CP_THREADS, 1) compact_units_kernel(const Comp
         p1 = __reduce_add_sync(0xffffffffu, p1);
         if (lane == 0 && (p0 | p1)) { atomicAdd(&s_misc[0], p0); atomicAdd(&s_misc[1], p1); }
     }
-    if (tid == 0) prefix[nu] = 0;
-    __syncthreads();
-    const int n_kept = block_excl_scan(prefix, nu, warp_tot);
+    int n_kept;
+    if (nu < CP_THREADS) {
+        // one unit per thread: the scan runs on the registers (one barrier for the warp totals, one for the result)
+        const int mine = tid < nu ? prefix[tid] : 0;        // written by this thread above
+        int tot;
+        const int ex = warp_excl_scan(mine, lane, tot);
+        if (lane == 0) warp_tot[wid] = tot;
+        __syncthreads();
+        int base = 0;
+        for (int w = 0; w < wid; ++w) base += warp_tot[w];
+        if (tid <= nu) prefix[tid] = base + ex;
+        __syncthreads();
+        n_kept = prefix[nu];
+    } else {
+        if (tid == 0) prefix[nu] = 0;
+        __syncthreads();
+        n_kept = block_excl_scan(prefix, nu, warp_tot);
+    }
     const int n0 = s_misc[0], n1 = s_misc[1], u_open = s_misc[2], n_hist = s_misc[3];
 
     // ---- destination share: the source slot of every row by a search over the scanned lengths --------------
