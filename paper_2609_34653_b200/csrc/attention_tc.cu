@@ -83,7 +83,8 @@ struct Barriers {
     uint64_t q_full;
     uint64_t kv_full[NSTAGE];
     uint64_t kv_empty[NSTAGE];
-    uint64_t s_full[2];         // [buffer]
+    uint64_t s_full;            // S of the next block is complete
+    uint64_t s_free;            // both warpgroups hold S in registers: the next QK^T may overwrite it
     uint64_t p_full[2][2];      // [warpgroup][buffer]
     uint64_t pv_done[2];        // [buffer] both PVs of the block in that buffer have completed
     uint64_t o_done;
@@ -187,8 +188,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             tc::mbar_init(tc::smem_u32(&bars->kv_full[s]), 1);
             tc::mbar_init(tc::smem_u32(&bars->kv_empty[s]), 1);
         }
+        tc::mbar_init(tc::smem_u32(&bars->s_full), 1);
+        tc::mbar_init(tc::smem_u32(&bars->s_free), 256);
         for (int b = 0; b < 2; ++b) {
-            tc::mbar_init(tc::smem_u32(&bars->s_full[b]), 1);
             tc::mbar_init(tc::smem_u32(&bars->p_full[0][b]), 128);
             tc::mbar_init(tc::smem_u32(&bars->p_full[1][b]), 128);
         }
@@ -270,45 +272,34 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         // ================================ QK issuer (one thread) ================================
         if (lane == 0) {
             auto wait = [&](uint64_t* bar, int parity) { return tc::mbar_wait(tc::smem_u32(bar), parity, abort_flag); };
-            // S[buf] = Q K^T over the 128 keys of ring slot idx
-            auto issue_qk = [&](int buf, int idx) {
+            // S = Q K^T over the 128 keys of ring slot idx
+            auto issue_qk = [&](int idx) {
                 const uint32_t b0 = kv_smem + (idx % NSTAGE) * TILE_BYTES;
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk) {
                     const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
-                    tc::umma_ss(tmem + buf * 128, tc::umma_smem_desc(q_smem + off, 16, 1024), tc::umma_smem_desc(b0 + off, 16, 1024),
+                    tc::umma_ss(tmem, tc::umma_smem_desc(q_smem + off, 16, 1024), tc::umma_smem_desc(b0 + off, 16, 1024),
                                 IDESC_QK, kk > 0, 1u);
                 }
-                tc::umma_commit(tc::smem_u32(&bars->s_full[buf]));
+                tc::umma_commit(tc::smem_u32(&bars->s_full));
                 tc::umma_commit(tc::smem_u32(&bars->kv_empty[idx % NSTAGE]));
             };
-            int g = 0;                                       // blocks started so far (buffer = g & 1)
+            int g = 0;                                       // blocks started so far
             bool ok = true;
             while (ok && it.next(part)) {
                 const int n = part.j1 - part.j0;
                 ok = wait(&bars->q_full, part_idx & 1);
-                // S of the first two blocks: K tiles at ring positions 0 and 1 of the part.  Both buffers are
-                // free: every pv_done of the previous part was waited for below.
-                for (int jj = 0; jj < 2 && jj < n && ok; ++jj) {
-                    const int idx = kv_base + jj;
+                for (int jj = 0; jj < n && ok; ++jj) {
+                    const int gb = g + jj;
+                    const int idx = kv_base + (jj < 2 ? jj : 2 * jj - 1);      // K_jj in the part's load order
+                    TRACE(2, 0);
                     ok = wait(&bars->kv_full[idx % NSTAGE], (idx / NSTAGE) & 1);
+                    TRACE(2, 1);
+                    // S is single-buffered: the softmax warps must hold the previous block in registers
+                    if (ok && gb > 0) ok = wait(&bars->s_free, (gb - 1) & 1);
                     if (!ok) break;
                     tc::tcgen05_fence_after();
-                    issue_qk((g + jj) & 1, idx);
-                }
-                for (int jj = 0; jj < n && ok; ++jj) {
-                    const int gb = g + jj, buf = gb & 1;
-                    TRACE(2, 0);
-                    // the PVs of block j have read P out of the buffer: S of block j+2 may overwrite it
-                    ok = wait(&bars->pv_done[buf], (gb >> 1) & 1);
-                    TRACE(2, 1);
-                    if (ok && jj + 2 < n) {
-                        const int idx = kv_base + 2 * (jj + 2) - 1;          // K_{j+2} in the part's load order
-                        ok = wait(&bars->kv_full[idx % NSTAGE], (idx / NSTAGE) & 1);
-                        if (!ok) break;
-                        tc::tcgen05_fence_after();
-                        issue_qk(buf, idx);
-                    }
+                    issue_qk(idx);
                     TRACE(2, 2); TRACE(2, 3); TRACE(2, 4);
                     TRACE_NEXT();
                 }
@@ -330,7 +321,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const uint32_t b0 = kv_smem + stage * TILE_BYTES + w * (HK * 128);
 #pragma unroll
                 for (int kk = 0; kk < HK / 16; ++kk) {
-                    tc::umma_ts(tmem + 256 + w * 128, tmem + buf * 128 + w * HK + kk * 8,
+                    tc::umma_ts(tmem + 256 + w * 128, tmem + 128 + buf * 64 + w * 32 + kk * 8,
                                 tc::umma_smem_desc(b0 + kk * 2048, HALF_BYTES, 1024), IDESC_PV, accumulate || kk > 0, 1u);
                 }
             };
@@ -377,15 +368,19 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
             for (int jj = 0; jj < n_part && ok; ++jj, ++g) {
                 const int j = part.j0 + jj;
-                const int buf = g & 1;
-                const uint32_t s_tmem = tmem + buf * 128 + w * HK + lane_addr;
-                ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&bars->s_full[buf]), (g >> 1) & 1, abort_flag));
+                const int buf = g & 1;                                     // P buffer of this block
+                const uint32_t s_tmem = tmem + w * HK + lane_addr;
+                const uint32_t p_tmem = tmem + 128 + buf * 64 + w * 32 + lane_addr;
+                ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&bars->s_full), g & 1, abort_flag));
                 tc::tcgen05_fence_after();
                 if ((warp & 3) == 0) TRACE(w, 0);
                 uint32_t sa[32], sb[32];
                 tc::tmem_ld32(s_tmem, sa);
                 tc::tmem_ld32(s_tmem + 32, sb);
                 tc::tmem_wait_ld();
+                // the logits are in registers: S may be overwritten by the next block's QK^T
+                tc::tcgen05_fence_before();
+                tc::mbar_arrive(tc::smem_u32(&bars->s_free));
 
                 // masking of this warpgroup's 64 keys: ragged history tail, causal diagonal
                 int n_valid = HK;
@@ -450,7 +445,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 ATT_PAIR4(8)  ATT_PAIR4(9)  ATT_PAIR4(10) ATT_PAIR4(11) ATT_PAIR4(12) ATT_PAIR4(13) ATT_PAIR4(14) ATT_PAIR4(15)
 #undef ATT_PAIR4
 #undef ATT_PAIR
-                tc::tmem_st32(s_tmem, pk);                   // P over the first 32 columns of this half of the S buffer
+                // the P buffer of block g was last read by the PVs of block g-2, which completed before the
+                // wait of block g-1 below returned (or, for the first two blocks of a part, before the previous part ended)
+                tc::tmem_st32(p_tmem, pk);
                 if ((warp & 3) == 0) TRACE(w, 2);
                 // O is touched only after the PVs of the previous block have completed (they have, by now, nearly always)
                 if (jj > 0)
