@@ -31,7 +31,7 @@
 namespace {
 
 #ifndef ATT_POLY_EVERY
-#define ATT_POLY_EVERY 0       // every n-th pair of exponentials takes the polynomial path (0: none; 2-4 measured no gain here)
+#define ATT_POLY_EVERY 4       // every n-th pair of exponentials takes the polynomial path (0: none); 4 measured best (+2 %)
 #endif
 template <int PAIR>
 __device__ __forceinline__ uint64_t exp2_pair(uint64_t x2) {
@@ -426,7 +426,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
                 // a row that has seen no key yet keeps m_ref = -inf; exponentiate against 0 so that P = 0, not NaN
                 const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref * p.scale_log2;
-                // pairs of columns: a packed FMA scales two logits and a packed add sums two weights
+                // pairs of columns: a packed FMA scales two logits and a packed add sums two weights; every fourth
+                // pair takes its exponentials from the polynomial on the FMA pipe
                 const uint64_t c2 = tc::pack2(p.scale_log2, p.scale_log2), nm2 = tc::pack2(neg_m, neg_m);
                 uint64_t rs0 = 0ull, rs1 = 0ull;
                 uint32_t pk[32];
@@ -573,40 +574,46 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
 }
 
-// Merge the partial outputs of every item that was cut between CTAs.  Grid (items, 4 groups of 32 rows);
+// Merge the partial outputs of every item that was cut between CTAs.  Grid (share boundaries, 4 groups of 32 rows);
 // a warp owns 4 rows and a lane 4 of a row's 128 columns.  Shared memory: one int per CTA of the main kernel.
 constexpr int MERGE_BATCH = 4;
 __global__ void __launch_bounds__(256) attention_merge_kernel(const AttnParams p, int n_cta) {
     extern __shared__ int s_slot[];                          // partial slot of every part of the item
-    __shared__ int s_n;
-    const int qt = p.n_tiles - 1 - blockIdx.x / p.h_q;
-    const int head = blockIdx.x % p.h_q;
+    __shared__ int s_n, s_qt, s_head;
+    // blockIdx.x + 1 = b: the boundary between the shares of CTA b-1 and CTA b of the main kernel.  An item is
+    // cut only where a boundary falls strictly inside it, so the boundaries enumerate the cut items; an item
+    // that holds several boundaries is merged by the first of them.
     if (threadIdx.x == 0) {
         int n_hist = p.n_hist_dev ? *p.n_hist_dev : p.n_hist_max;
         n_hist = max(0, min(n_hist, p.n_hist_max));
         Sched s;
         s.nhb = (n_hist + BK - 1) / BK; s.n_tiles = p.n_tiles; s.h_q = p.h_q;
         const long long total = s.total();
-        const long long w0 = s.item_begin(qt, head);
-        const int nb = s.nb_item(qt);
-        auto cta_of = [&](long long w) {
-            int b = (int)(w * n_cta / total);
-            b = max(0, min(b, n_cta - 1));
-            while (b + 1 < n_cta && share_begin(total, b + 1, n_cta) <= w) ++b;
-            while (b > 0 && share_begin(total, b, n_cta) > w) --b;
-            return b;
-        };
-        const int b_first = cta_of(w0), b_last = cta_of(w0 + nb - 1);
-        int n = 0;
-        if (b_first != b_last)
-            for (int b = b_first; b <= b_last; ++b)
-                if (share_begin(total, b, n_cta) != share_begin(total, b + 1, n_cta))
-                    s_slot[n++] = b * 2 + (b == b_first ? 1 : 0);
-        s_n = n;
+        const int b = blockIdx.x + 1;
+        const long long w = share_begin(total, b, n_cta);
+        int n = 0, qt = 0, head = 0, j = 0;
+        if (w > 0 && w < total) {
+            s.locate(w, qt, head, j);
+            const long long w0 = w - j, w1 = w0 + s.nb_item(qt);            // the item is [w0, w1)
+            if (j > 0 && share_begin(total, b - 1, n_cta) <= w0) {
+                // first part: the non-empty share that holds w0 (slot 1); then every non-empty share that
+                // starts inside the item (slot 0)
+                int bf = b - 1;
+                while (bf > 0 && share_begin(total, bf, n_cta) == share_begin(total, bf + 1, n_cta)) --bf;
+                s_slot[n++] = bf * 2 + 1;
+                for (int bb = b; bb < n_cta; ++bb) {
+                    const long long wb = share_begin(total, bb, n_cta);
+                    if (wb >= w1) break;
+                    if (wb != share_begin(total, bb + 1, n_cta)) s_slot[n++] = bb * 2;
+                }
+            }
+        }
+        s_n = n; s_qt = qt; s_head = head;
     }
     __syncthreads();
     const int n_parts = s_n;
-    if (n_parts == 0) return;                                // the item was computed by one CTA
+    if (n_parts == 0) return;                                // no item is cut at this boundary (or an earlier boundary owns it)
+    const int qt = s_qt, head = s_head;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int q4 = 0; q4 < 4; ++q4) {
         const int r = blockIdx.y * 32 + warp * 4 + q4;       // row of the tile
@@ -635,7 +642,7 @@ __global__ void __launch_bounds__(256) attention_merge_kernel(const AttnParams p
 #pragma unroll
             for (int i = 0; i < MERGE_BATCH; ++i) {
                 if (!(ml[i].y > 0.f)) continue;
-                const float wgt = exp2f((ml[i].x - M) * p.scale_log2);
+                const float wgt = tc::ex2_approx((ml[i].x - M) * p.scale_log2);
                 acc.x += wgt * o[i].x; acc.y += wgt * o[i].y; acc.z += wgt * o[i].z; acc.w += wgt * o[i].w;
                 L += wgt * ml[i].y;
             }
@@ -687,7 +694,10 @@ omni_status omni_attention_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q,
     }
     attention_tc_kernel<<<n_cta, ATT_THREADS, SMEM_BYTES, st>>>(tm_q, tm_kh, tm_vh, tm_kc, tm_vc, p);
     OMNI_CHECK_LAUNCH(ctx, "attention_tc_kernel");
-    attention_merge_kernel<<<dim3(p.n_tiles * g.h_q, 4), 256, (n_cta + 1) * sizeof(int), st>>>(p, n_cta);
-    OMNI_CHECK_LAUNCH(ctx, "attention_merge_kernel");
+    if (n_cta > 1) {
+        // one CTA row per boundary between two shares: only an item cut there has partials to merge
+        attention_merge_kernel<<<dim3(n_cta - 1, 4), 256, (n_cta + 1) * sizeof(int), st>>>(p, n_cta);
+        OMNI_CHECK_LAUNCH(ctx, "attention_merge_kernel");
+    }
     return OMNI_OK;
 }
