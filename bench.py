@@ -374,14 +374,14 @@ def main():
     hq = torch.from_numpy(w.q).to(tdt).contiguous().pin_memory()
     hk = torch.from_numpy(w.k_chunk).to(tdt).contiguous().pin_memory()
     hv = torch.from_numpy(w.v_chunk).to(tdt).contiguous().pin_memory()
-    ho = torch.empty((T, w.h_q, w.d), dtype=torch.float32).pin_memory()
+    ho = torch.empty((T, w.h_q, w.d), dtype=tdt).pin_memory()       # the output in the storage dtype, as a model consumes it
     hcu = np.ascontiguousarray(w.chunk_units, dtype=np.int32)
     e2e_steps = max(3, min(args.steps, 20))
 
     def e2e_step(s):
         ctx.chunk_step_host(hq, hk, hv, T, hcu, len(hcu), s["k_in"], s["v_in"], n_hist_dev, N, units_in, n_units_dev, U,
                             w.w_modality, params, w.page_size, 0.0, s["k_out"], s["v_out"], units_out, n_hist_out,
-                            n_units_out, ho, ob.DTYPE_FP32)
+                            n_units_out, ho, ob.DTYPE_BF16 if w.dtype == "bf16" else ob.DTYPE_FP32)
         torch.cuda.current_stream().synchronize()       # the caller reads o_host after every step
 
     for i in range(3):
@@ -461,12 +461,13 @@ def main():
         import threadpoolctl
         G = w.h_q // w.h_kv
         t0 = time.perf_counter()
-        oc.chunk_attention(w.q[:, :G], w.k_hist[:kept, :1], w.v_hist[:kept, :1], w.k_chunk[:, :1], w.v_chunk[:, :1])
+        oc.chunk_attention(w.q, w.k_hist[:kept], w.v_hist[:kept], w.k_chunk, w.v_chunk)
         dt = time.perf_counter() - t0
         cores = max([p.get("num_threads", 1) for p in threadpoolctl.threadpool_info()] + [1])
-        line["cpu_baseline"] = {"value": work["attn_flop"] / w.h_kv / dt / 1e12, "unit": "TFLOP/s", "cores": cores,
+        line["cpu_baseline"] = {"value": work["attn_flop"] / dt / 1e12, "unit": "TFLOP/s", "cores": cores,
                                 "kind": "oracle", "seconds": dt,
-                                "sample": f"attention of 1 of {w.h_kv} KV groups ({G} query heads), T={T}, kept history {kept}"}
+                                "sample": f"the attention step of the workload, all {w.h_q} query heads, T={T}, kept history {kept} "
+                                          "(scoring, selection and compaction of the oracle are not in the sample)"}
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:

@@ -21,6 +21,9 @@ void free_all(omnitide_ctx* c) {
                     c->st_k, c->st_v, c->st_o, c->st_units, c->attn_part_o, c->attn_part_ml, c->cp_words};
     for (void* p : ptrs)
         if (p) cudaFree(p);
+    if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+    if (c->ev_kv) cudaEventDestroy(c->ev_kv);
+    if (c->aux_stream) cudaStreamDestroy(c->aux_stream);
 }
 
 }  // namespace
@@ -52,6 +55,9 @@ extern "C" omni_status omnitide_create(omnitide_ctx** ctx_out, const omni_geomet
     ok &= alloc(&c->score_part, row_tiles * ((size_t)g->u_cap + 64) * 128) == cudaSuccess;   // + split boundaries
     ok &= alloc(&c->score_tile_mass, row_tiles * g->u_cap) == cudaSuccess;
     ok &= alloc(&c->score_mass64, (size_t)g->u_cap) == cudaSuccess;
+    ok &= cudaStreamCreateWithFlags(&c->aux_stream, cudaStreamNonBlocking) == cudaSuccess;
+    ok &= cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
+    ok &= cudaEventCreateWithFlags(&c->ev_kv, cudaEventDisableTiming) == cudaSuccess;
     ok &= alloc(&c->cp_words, (size_t)c->sm_count + 1) == cudaSuccess;
     ok = ok && cudaMemset(c->cp_words, 0, ((size_t)c->sm_count + 1) * sizeof(unsigned long long)) == cudaSuccess;
     ok &= alloc(&c->ws_scores, (size_t)g->u_cap) == cudaSuccess;
@@ -155,7 +161,7 @@ extern "C" omni_status omnitide_chunk_attention(omnitide_ctx* ctx, void* stream,
                                  out_dtype, lse_out);
 }
 
-extern "C" omni_status omnitide_chunk_step(omnitide_ctx* ctx, void* stream, const void* q, const void* k_chunk,
+static omni_status chunk_step_impl(cudaEvent_t chunk_kv_ready, omnitide_ctx* ctx, void* stream, const void* q, const void* k_chunk,
                                            const void* v_chunk, int32_t t, const omni_unit* chunk_units,
                                            int32_t n_chunk_units, const void* k_cache, const void* v_cache,
                                            const int32_t* n_hist_dev, int32_t n_hist_max, const omni_unit* units,
@@ -182,11 +188,27 @@ extern "C" omni_status omnitide_chunk_step(omnitide_ctx* ctx, void* stream, cons
     s = omnipage_compact_units(ctx, stream, k_cache, v_cache, k_cache_out, v_cache_out, units, n_units_dev, n_units_max,
                                ctx->ws_unit_keep, n_hist_max, page_size, units_out, n_units_kept, nullptr, info, nullptr);
     if (s) return s;
+    // the chunk's K/V rows are first read here (scoring reads only Q and the cached keys)
+    if (chunk_kv_ready) OMNI_CUDA(ctx, cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), chunk_kv_ready, 0));
     s = omnitide_chunk_attention(ctx, stream, q, t, k_cache_out, v_cache_out, n_kept, n_hist_max, k_chunk, v_chunk, scale,
                                  o_out, out_dtype, nullptr);
     if (s) return s;
     return omnipage_append(ctx, stream, k_cache_out, v_cache_out, n_kept, k_chunk, v_chunk, t, units_out, n_units_kept,
                            chunk_units, n_chunk_units, n_hist_out, n_units_out);
+}
+
+extern "C" omni_status omnitide_chunk_step(omnitide_ctx* ctx, void* stream, const void* q, const void* k_chunk,
+                                           const void* v_chunk, int32_t t, const omni_unit* chunk_units,
+                                           int32_t n_chunk_units, const void* k_cache, const void* v_cache,
+                                           const int32_t* n_hist_dev, int32_t n_hist_max, const omni_unit* units,
+                                           const int32_t* n_units_dev, int32_t n_units_max, const float* w_modality,
+                                           const omni_select_params* params, int32_t page_size, float scale,
+                                           void* k_cache_out, void* v_cache_out, omni_unit* units_out, int32_t* n_hist_out,
+                                           int32_t* n_units_out, void* o_out, int32_t out_dtype,
+                                           omni_compact_info* info_out) {
+    return chunk_step_impl(nullptr, ctx, stream, q, k_chunk, v_chunk, t, chunk_units, n_chunk_units, k_cache, v_cache,
+                           n_hist_dev, n_hist_max, units, n_units_dev, n_units_max, w_modality, params, page_size, scale,
+                           k_cache_out, v_cache_out, units_out, n_hist_out, n_units_out, o_out, out_dtype, info_out);
 }
 
 extern "C" omni_status omnitide_chunk_step_host(omnitide_ctx* ctx, void* stream, const void* q_host,
@@ -207,16 +229,21 @@ extern "C" omni_status omnitide_chunk_step_host(omnitide_ctx* ctx, void* stream,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t q_bytes = (size_t)t * ctx->g.h_q * ctx->g.d * ctx->es;
     const size_t kv_bytes = (size_t)t * ctx->row_bytes;
+    // Q goes up on the caller's stream and scoring starts behind it; the chunk's K/V rows and unit records,
+    // first needed by the attention step, go up on a second stream beside the scoring kernels.
+    OMNI_CUDA(ctx, cudaEventRecord(ctx->ev_fork, st));       // orders the upload behind the previous call's readers of the staging
     OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->st_q, q_host, q_bytes, cudaMemcpyHostToDevice, st));
-    OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->st_k, k_chunk_host, kv_bytes, cudaMemcpyHostToDevice, st));
-    OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->st_v, v_chunk_host, kv_bytes, cudaMemcpyHostToDevice, st));
+    OMNI_CUDA(ctx, cudaStreamWaitEvent(ctx->aux_stream, ctx->ev_fork, 0));
+    OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->st_k, k_chunk_host, kv_bytes, cudaMemcpyHostToDevice, ctx->aux_stream));
+    OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->st_v, v_chunk_host, kv_bytes, cudaMemcpyHostToDevice, ctx->aux_stream));
     if (n_chunk_units)
         OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->st_units, chunk_units_host, sizeof(omni_unit) * n_chunk_units,
-                                       cudaMemcpyHostToDevice, st));
-    omni_status s = omnitide_chunk_step(ctx, stream, ctx->st_q, ctx->st_k, ctx->st_v, t, ctx->st_units, n_chunk_units,
-                                        k_cache, v_cache, n_hist_dev, n_hist_max, units, n_units_dev, n_units_max,
-                                        w_modality, params, page_size, scale, k_cache_out, v_cache_out, units_out,
-                                        n_hist_out, n_units_out, ctx->st_o, out_dtype, info_out);
+                                       cudaMemcpyHostToDevice, ctx->aux_stream));
+    OMNI_CUDA(ctx, cudaEventRecord(ctx->ev_kv, ctx->aux_stream));
+    omni_status s = chunk_step_impl(ctx->ev_kv, ctx, stream, ctx->st_q, ctx->st_k, ctx->st_v, t, ctx->st_units, n_chunk_units,
+                                    k_cache, v_cache, n_hist_dev, n_hist_max, units, n_units_dev, n_units_max,
+                                    w_modality, params, page_size, scale, k_cache_out, v_cache_out, units_out,
+                                    n_hist_out, n_units_out, ctx->st_o, out_dtype, info_out);
     if (s) return s;
     const size_t o_bytes = (size_t)t * ctx->g.h_q * ctx->g.d * (out_dtype == OMNI_DTYPE_FP32 ? 4 : 2);
     OMNI_CUDA(ctx, cudaMemcpyAsync(o_host, ctx->st_o, o_bytes, cudaMemcpyDeviceToHost, st));

@@ -36,6 +36,8 @@ struct omnitide_ctx {
     omni_compact_info* ws_info;
     // staging of omnitide_chunk_step_host
     void* st_q; void* st_k; void* st_v; void* st_o; omni_unit* st_units;
+    cudaStream_t aux_stream;      // carries the K/V chunk upload of chunk_step_host beside the scoring kernels
+    cudaEvent_t ev_fork, ev_kv;
     // attention split-KV partials
     float* attn_part_o;           // allocated on first use
     float* attn_part_ml;
