@@ -687,10 +687,9 @@ omni_status omni_attention_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q,
     const long long w_max = (long long)g.h_q * ((long long)p.n_tiles * (nhb_max + 1) + (long long)p.n_tiles * (p.n_tiles - 1) / 2);
     const int n_cta = (int)std::max(1ll, std::min((long long)ctx->sm_count, w_max / 4));
     p.part_o = ctx->attn_part_o; p.part_ml = reinterpret_cast<float2*>(ctx->attn_part_ml);
-    static bool attr_set = false;
-    if (!attr_set) {
+    if (!ctx->attn_attr_set) {                               // per context, hence per device
         OMNI_CUDA(ctx, cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
-        attr_set = true;
+        ctx->attn_attr_set = true;
     }
     attention_tc_kernel<<<n_cta, ATT_THREADS, SMEM_BYTES, st>>>(tm_q, tm_kh, tm_vh, tm_kc, tm_vc, p);
     OMNI_CHECK_LAUNCH(ctx, "attention_tc_kernel");

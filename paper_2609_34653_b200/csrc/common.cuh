@@ -42,6 +42,7 @@ struct omnitide_ctx {
     float* attn_part_o;           // allocated on first use
     float* attn_part_ml;
     size_t attn_part_cap;
+    bool attn_attr_set;           // the attention kernel's shared-memory limit has been raised on this device
     // -----------------------------------------------------------------------------------
     void* encode_tiled;           // cuTensorMapEncodeTiled, resolved through the runtime
     int64_t launches;

@@ -39,7 +39,7 @@ struct ScoreParams {
     float scale_log2;
     float2* part;             // [tile][seg_cap][128]
     int seg_cap;
-    int n_pairs, n_row_tiles, n_splits;
+    int ctas_per_kv, n_row_tiles, n_splits;                   // CTAs per KV head and split: ceil(n_row_tiles * G / NT)
     int32_t* status;
 };
 
@@ -68,7 +68,7 @@ __device__ __forceinline__ uint64_t exp2_pair(uint64_t x2) {
     return pack2(tc::ex2_approx(x0), tc::ex2_approx(x1));
 }
 
-__device__ __forceinline__ int blocks_per_split(int nkb, int n_splits) { return (nkb + n_splits - 1) / n_splits; }
+__host__ __device__ __forceinline__ int blocks_per_split(int nkb, int n_splits) { return (nkb + n_splits - 1) / n_splits; }
 
 __global__ void __launch_bounds__(SC_THREADS, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, const ScoreParams p) {
@@ -82,12 +82,17 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     volatile int* abort_flag = &bars->abort_flag;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    const int per_split = p.n_pairs * p.h_q;
+    // The four tiles of a CTA share one KV head (hence one K stream): the (row tile, query head of the group)
+    // pairs of a KV head are numbered row-tile-major and a CTA takes four consecutive ones, so no tile slot is
+    // idle unless n_row_tiles * G is not a multiple of four (G = 4: one row tile, the four heads of the group).
+    const int G = p.h_q / p.h_kv;
+    const int per_split = p.ctas_per_kv * p.h_kv;
     const int split = blockIdx.x / per_split;
     const int rem = blockIdx.x % per_split;
-    const int pair = rem / p.h_q;
-    const int head = rem % p.h_q;
-    const int kvh = head / (p.h_q / p.h_kv);
+    const int kvh = rem / p.ctas_per_kv;
+    const int c_in_kv = rem % p.ctas_per_kv;
+    auto row_of = [&](int tt) { return (c_in_kv * NT + tt) / G; };
+    auto head_of = [&](int tt) { return kvh * G + (c_in_kv * NT + tt) % G; };
 
     int n_units = p.n_units_dev ? *p.n_units_dev : p.n_units_max;
     n_units = max(0, min(n_units, p.n_units_max));
@@ -104,7 +109,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     if (nb <= 0) return;
     bool active[NT];
 #pragma unroll
-    for (int tt = 0; tt < NT; ++tt) active[tt] = (NT * pair + tt) * BLK < p.t;
+    for (int tt = 0; tt < NT; ++tt) active[tt] = row_of(tt) < p.n_row_tiles;
 
     for (int u = threadIdx.x; u < n_units; u += SC_THREADS) unit_end[u] = p.units[u].start + p.units[u].len;
     if (threadIdx.x == 0) {
@@ -135,7 +140,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             tc::mbar_expect_tx(tc::smem_u32(&bars->q_full), n_active * TILE_BYTES);
             for (int tt = 0; tt < NT; ++tt) {
                 if (!active[tt]) continue;
-                const int row0 = (NT * pair + tt) * BLK;
+                const int row0 = row_of(tt) * BLK, head = head_of(tt);
                 tc::tma_load_2d(q_smem + tt * TILE_BYTES, &tm_q, head * HD, row0, tc::smem_u32(&bars->q_full));
                 tc::tma_load_2d(q_smem + tt * TILE_BYTES + HALF_BYTES, &tm_q, head * HD + 64, row0, tc::smem_u32(&bars->q_full));
             }
@@ -185,7 +190,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (active[tt]) {
             const int r = (warp & 3) * 32 + lane;
             const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-            const int tile = head * p.n_row_tiles + NT * pair + tt;
+            const int tile = head_of(tt) * p.n_row_tiles + row_of(tt);
             float2* part = p.part + (size_t)tile * p.seg_cap * BLK + r;
             const float c = p.scale_log2;
             // unit that holds the first key of this split
@@ -407,19 +412,21 @@ omni_status omni_score_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q, int
     p.units = units; p.n_units_dev = n_units_dev; p.n_units_max = n_units_max;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.part = ctx->score_part; p.seg_cap = g.u_cap + MAX_SPLITS;
-    p.n_pairs = (t + NT * BLK - 1) / (NT * BLK);
     p.n_row_tiles = (t + BLK - 1) / BLK;
     p.status = ctx->status_dev;
     // split the key range so that the grid fills whole waves of SMs and a split keeps >= 8 key blocks
     const int nkb_max = (n_hist_max + BLK - 1) / BLK;
-    const int base_items = p.n_pairs * g.h_q;
+    p.ctas_per_kv = (p.n_row_tiles * (g.h_q / g.h_kv) + NT - 1) / NT;
+    const int base_items = p.ctas_per_kv * g.h_kv;
+    // cost of a choice = waves x (key blocks per CTA + a start-up allowance: Q load, pipeline fill, partial writes)
+    constexpr int STARTUP_BLOCKS = 3;
     int best = 1;
-    double best_eff = 0.0;
+    long long best_cost = -1;
     for (int ks = 1; ks <= MAX_SPLITS && (ks == 1 || nkb_max / ks >= 8); ++ks) {
         const long long items = (long long)base_items * ks;
         const long long waves = (items + ctx->sm_count - 1) / ctx->sm_count;
-        const double eff = (double)items / (double)(waves * ctx->sm_count);
-        if (eff > best_eff + 1e-3) { best_eff = eff; best = ks; }
+        const long long cost = waves * (blocks_per_split(nkb_max, ks) + STARTUP_BLOCKS);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = ks; }
     }
     p.n_splits = best;
     const int smem = SMEM_FIXED + n_units_max * (int)sizeof(int);
