@@ -192,6 +192,22 @@ omni_status omnipage_compact_units(omnitide_ctx* ctx, void* stream,
                                    int32_t* slot_map_out, omni_compact_info* info_out, uint8_t* page_class_out);
 
 /*
+ * (next row: cross-layer batching) The unit-granular pack applied to n_layers caches in ONE launch with one shared
+ * source -> destination map (Section 6.2 "Executing accepted moves": the mapping is planned once from metadata and
+ * every layer's K and V rows follow it).  k_src / v_src / k_dst / v_dst [dev] are device arrays of n_layers
+ * device pointers (caller-owned; out of place only: no k_dst[l] may overlap any source).  All other arguments
+ * and all outputs are those of omnipage_compact_units (the integer outputs describe the shared map once).
+ * Turns the launch-bound single-layer copy into one bandwidth-bound launch.  2 * s_span_max * n_layers < 2^31.
+ */
+omni_status omnipage_compact_units_batched(omnitide_ctx* ctx, void* stream,
+                                           const void* const* k_src, const void* const* v_src,
+                                           void* const* k_dst, void* const* v_dst, int32_t n_layers,
+                                           const omni_unit* units, const int32_t* n_units_dev, int32_t n_units_max,
+                                           const uint8_t* unit_keep, int32_t s_span_max, int32_t page_size,
+                                           const omni_unit* units_kept, const int32_t* n_units_kept_dev,
+                                           int32_t* slot_map_out, omni_compact_info* info_out, uint8_t* page_class_out);
+
+/*
  * (a5) Append: new entries enter the recent-context class behind the retained history
  * (Section 6.1).  Copies the chunk's t K/V rows to cache slots [n_kept, n_kept + t), appends the
  * chunk's units to `units` with start += n_kept and group = recent-context, and writes

@@ -37,7 +37,7 @@ class CompactInfo(C.Structure):
 
 EXPORTS = [
     "omnitide_create", "omnitide_destroy", "omnitide_poll_status", "omnitide_last_error",
-    "omnitide_score_units", "omnitide_select_units", "omnipage_compact", "omnipage_compact_units", "omnipage_append",
+    "omnitide_score_units", "omnitide_select_units", "omnipage_compact", "omnipage_compact_units", "omnipage_compact_units_batched", "omnipage_append",
     "omnitide_chunk_attention", "omnitide_chunk_step", "omnitide_chunk_step_host",
     "omnitide_set_option", "omnitide_launch_count", "omnitide_score_units_noalloc",
 ]
@@ -183,6 +183,16 @@ class Context:
                                                     _ptr(n_units_kept_dev), _ptr(slot_map_out), _ptr(info_out),
                                                     _ptr(page_class_out)),
                     "omnipage_compact_units")
+
+    def compact_units_batched(self, k_src_ptrs, v_src_ptrs, k_dst_ptrs, v_dst_ptrs, n_layers, units, n_units_dev,
+                              n_units_max, unit_keep, s_span_max, page_size, units_kept, n_units_kept_dev, slot_map_out,
+                              info_out, page_class_out):
+        """k_src_ptrs ...: int64 CUDA tensors holding n_layers device pointers each."""
+        self._check(self.lib.omnipage_compact_units_batched(
+            self._ctx, _stream(), _ptr(k_src_ptrs), _ptr(v_src_ptrs), _ptr(k_dst_ptrs), _ptr(v_dst_ptrs), n_layers,
+            _ptr(units), _ptr(n_units_dev), n_units_max, _ptr(unit_keep), s_span_max, page_size, _ptr(units_kept),
+            _ptr(n_units_kept_dev), _ptr(slot_map_out), _ptr(info_out), _ptr(page_class_out)),
+            "omnipage_compact_units_batched")
 
     def append(self, k_cache, v_cache, n_kept_dev, k_chunk, v_chunk, t, units, n_units_dev, chunk_units,
                n_chunk_units, n_hist_out, n_units_out):

@@ -197,6 +197,40 @@ __device__ __forceinline__ unsigned long long ld_relaxed_gpu(const unsigned long
     return v;
 }
 
+// element i of a device array of pointers, through the read-only path
+template <class T, class P>
+__device__ __forceinline__ T* ldg_ptr(P table, int i) {
+    return reinterpret_cast<T*>(__ldg(reinterpret_cast<const unsigned long long*>(table) + i));
+}
+
+// One lane streams `mcp` row copies HBM -> shared memory -> HBM with cp.async.bulk, `n_slots` rows in flight:
+// copy q reads src_of(q) and writes dst_of(q) (both called in increasing q).  Returns false after a timeout.
+template <class SrcOf, class DstOf>
+__device__ __forceinline__ bool bulk_copy_loop(const int mcp, SrcOf src_of, DstOf dst_of, const uint32_t row_bytes,
+                                               const int n_slots, const uint32_t buf0, uint64_t* bars, int* abort_flag_p) {
+    auto issue_load = [&](int q) {
+        const int slot = q % n_slots;
+        const uint32_t bar = tc::smem_u32(&bars[slot]);
+        tc::mbar_expect_tx(bar, row_bytes);
+        bulk_load(buf0 + slot * row_bytes, src_of(q), row_bytes, bar);
+    };
+    for (int q = 0; q < mcp && q < n_slots; ++q) issue_load(q);
+    bool ok = true;
+    for (int q = 0; q < mcp && ok; ++q) {
+        const int slot = q % n_slots;
+        ok = tc::mbar_wait(tc::smem_u32(&bars[slot]), (q / n_slots) & 1, abort_flag_p);
+        if (!ok) break;
+        bulk_store(dst_of(q), buf0 + slot * row_bytes, row_bytes);
+        // the buffer of copy q-1 is free once its store has read it: refill it
+        if (q >= 1 && q - 1 + n_slots < mcp) {
+            asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            issue_load(q - 1 + n_slots);
+        }
+    }
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    return ok;
+}
+
 // Moves destination rows [d0, d0 + n_rows) of this CTA; src_list[r] is the source slot of row d0 + r.
 template <class Args>
 __device__ __forceinline__ void move_rows(const Args& a, const int* src_list, const int d0, const int n_rows, char* rowbuf,
@@ -217,26 +251,7 @@ __device__ __forceinline__ void move_rows(const Args& a, const int* src_list, co
                 const int i = wid + q * CP_WARPS;
                 return ((i & 1) ? a.v_dst : a.k_dst) + (size_t)(d0 + (i >> 1)) * a.row_bytes;
             };
-            auto issue_load = [&](int q) {
-                const int slot = q % a.n_slots;
-                const uint32_t bar = tc::smem_u32(&cbar[wid][slot]);
-                tc::mbar_expect_tx(bar, a.row_bytes);
-                bulk_load(buf0 + slot * a.row_bytes, src_of(q), a.row_bytes, bar);
-            };
-            for (int q = 0; q < mcp && q < a.n_slots; ++q) issue_load(q);
-            bool ok = true;
-            for (int q = 0; q < mcp && ok; ++q) {
-                const int slot = q % a.n_slots;
-                ok = tc::mbar_wait(tc::smem_u32(&cbar[wid][slot]), (q / a.n_slots) & 1, abort_flag_p);
-                if (!ok) break;
-                bulk_store(dst_of(q), buf0 + slot * a.row_bytes, a.row_bytes);
-                // the buffer of copy q-1 is free once its store has read it: refill it
-                if (q >= 1 && q - 1 + a.n_slots < mcp) {
-                    asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                    issue_load(q - 1 + a.n_slots);
-                }
-            }
-            asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+            const bool ok = bulk_copy_loop(mcp, src_of, dst_of, a.row_bytes, a.n_slots, buf0, cbar[wid], abort_flag_p);
             if (!ok) atomicOr(a.status, OMNI_DEV_TIMEOUT);
         }
         return;
@@ -506,8 +521,12 @@ struct CompactUnitsArgs {
     const omni_unit* units_kept; const int32_t* n_units_kept_dev;
     int32_t* slot_map; omni_compact_info* info; uint8_t* page_class; int32_t* status;
     int rows_cap; int n_slots;
+    // batched form: n_layers caches share the one source -> destination map (device arrays of n_layers pointers)
+    int n_layers;
+    const char* const* k_src_l; const char* const* v_src_l; char* const* k_dst_l; char* const* v_dst_l;
 };
 
+template <bool BATCHED>
 __global__ void __launch_bounds__(CP_THREADS, 1) compact_units_kernel(const CompactUnitsArgs a) {
     extern __shared__ __align__(128) int smem_i[];
     int* ustart = smem_i;                                   // [n_units_max]
@@ -592,18 +611,21 @@ __global__ void __launch_bounds__(CP_THREADS, 1) compact_units_kernel(const Comp
     const int n0 = s_misc[0], n1 = s_misc[1], u_open = s_misc[2], n_hist = s_misc[3];
 
     // ---- destination share: the source slot of every row by a search over the scanned lengths --------------
-    const int rows_per = (n_kept + G - 1) / G;
-    const int d0 = min(n_kept, (int)blockIdx.x * rows_per);
-    const int d1 = min(n_kept, d0 + rows_per);
-    const int n_rows = min(d1 - d0, a.rows_cap);
-    for (int r = tid; r < n_rows; r += CP_THREADS) {
-        const int dd = d0 + r;
-        int lo = 0, hi = nu;                                 // largest u with prefix[u] <= dd (its kept length is > 0)
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (prefix[mid] <= dd) lo = mid; else hi = mid;
+    int d0 = 0, n_rows = 0;
+    if (!BATCHED) {
+        const int rows_per = (n_kept + G - 1) / G;
+        d0 = min(n_kept, (int)blockIdx.x * rows_per);
+        const int d1 = min(n_kept, d0 + rows_per);
+        n_rows = min(d1 - d0, a.rows_cap);
+        for (int r = tid; r < n_rows; r += CP_THREADS) {
+            const int dd = d0 + r;
+            int lo = 0, hi = nu;                             // largest u with prefix[u] <= dd (its kept length is > 0)
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (prefix[mid] <= dd) lo = mid; else hi = mid;
+            }
+            src_list[r] = ustart[lo] + (dd - prefix[lo]);
         }
-        src_list[r] = ustart[lo] + (dd - prefix[lo]);
     }
     // ---- slot map (optional): unit u belongs to CTA u % G -----------------------------------------------------
     if (a.slot_map) {
@@ -640,9 +662,50 @@ __global__ void __launch_bounds__(CP_THREADS, 1) compact_units_kernel(const Comp
             a.page_class[p] = cls;
         }
     }
-    if (a.k_dst == nullptr) return;
-    __syncthreads();                                        // the source list is complete
-    move_rows(a, src_list, d0, n_rows, rowbuf, cbar, &abort_flag);
+    if (!BATCHED) {
+        if (a.k_dst == nullptr) return;
+        __syncthreads();                                    // the source list is complete
+        move_rows(a, src_list, d0, n_rows, rowbuf, cbar, &abort_flag);
+        return;
+    }
+    // ---- batched form: copies are numbered layer-major, (layer, destination row, K or V), and every CTA takes an
+    // equal contiguous range of them; a lane walks its copies in increasing order, so the unit that holds a
+    // destination row is found by stepping forward (a binary search only when the layer changes)
+    __syncthreads();
+    if (lane == 0 && n_kept > 0) {
+        const int total = 2 * n_kept * a.n_layers;           // the host bounds this below 2^31
+        const int per = (total + G - 1) / G;
+        const int c0 = min(total, (int)blockIdx.x * per), c1 = min(total, c0 + per);
+        const int mine = c1 - c0;
+        const int mcp = mine > wid ? (mine - wid + CP_WARPS - 1) / CP_WARPS : 0;
+        const uint32_t buf0 = tc::smem_u32(rowbuf) + (uint32_t)(wid * a.n_slots) * a.row_bytes;
+        int u_cur = 0, layer_cur = -1;
+        auto src_of = [&](int q) {
+            const int c = c0 + wid + q * CP_WARPS;
+            const int f = c >> 1, layer = f / n_kept, dd = f - layer * n_kept;
+            if (layer != layer_cur) {
+                int lo = 0, hi = nu;
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (prefix[mid] <= dd) lo = mid; else hi = mid;
+                }
+                u_cur = lo;
+                layer_cur = layer;
+            } else {
+                while (dd >= prefix[u_cur + 1]) ++u_cur;     // also steps over dropped units (equal prefixes)
+            }
+            const char* base = ldg_ptr<const char>((c & 1) ? a.v_src_l : a.k_src_l, layer);
+            return base + (size_t)(ustart[u_cur] + (dd - prefix[u_cur])) * a.row_bytes;
+        };
+        auto dst_of = [&](int q) {
+            const int c = c0 + wid + q * CP_WARPS;
+            const int f = c >> 1, layer = f / n_kept, dd = f - layer * n_kept;
+            char* base = ldg_ptr<char>((c & 1) ? a.v_dst_l : a.k_dst_l, layer);
+            return base + (size_t)dd * a.row_bytes;
+        };
+        if (!bulk_copy_loop(mcp, src_of, dst_of, a.row_bytes, a.n_slots, buf0, cbar[wid], &abort_flag))
+            atomicOr(a.status, OMNI_DEV_TIMEOUT);
+    }
 }
 
 // Dense copy of `n_rows` rows (device count) from staging back to the cache (in-place mode), and
@@ -834,6 +897,7 @@ extern "C" omni_status omnipage_compact_units(omnitide_ctx* ctx, void* stream, c
     a.units_kept = units_kept; a.n_units_kept_dev = n_units_kept_dev;
     a.slot_map = slot_map_out; a.info = info_out; a.page_class = page_class_out; a.status = ctx->status_dev;
     const int grid = ctx->sm_count;
+    a.n_layers = 1; a.k_src_l = a.v_src_l = nullptr; a.k_dst_l = a.v_dst_l = nullptr;
     a.rows_cap = (((s_span_max + grid - 1) / grid + 1) + 3) & ~3;
     const size_t smem_lists = ((size_t)3 * n_units_max + 8 + a.rows_cap) * sizeof(int);
     const size_t smem_lists_al = (smem_lists + 127) & ~(size_t)127;
@@ -847,8 +911,8 @@ extern "C" omni_status omnipage_compact_units(omnitide_ctx* ctx, void* stream, c
     }
     const size_t smem = smem_lists_al + (size_t)a.n_slots * CP_WARPS * ctx->row_bytes;
     if (smem > 48 * 1024)
-        OMNI_CUDA(ctx, cudaFuncSetAttribute(compact_units_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    compact_units_kernel<<<grid, CP_THREADS, smem, st>>>(a);
+        OMNI_CUDA(ctx, cudaFuncSetAttribute(compact_units_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    compact_units_kernel<false><<<grid, CP_THREADS, smem, st>>>(a);
     OMNI_CHECK_LAUNCH(ctx, "compact_units_kernel");
     if (in_place) {
         copy_rows_kernel<<<ctx->sm_count * 4, 256, 0, st>>>(
@@ -857,6 +921,50 @@ extern "C" omni_status omnipage_compact_units(omnitide_ctx* ctx, void* stream, c
             ctx->status_dev);
         OMNI_CHECK_LAUNCH(ctx, "copy_rows_kernel");
     }
+    return OMNI_OK;
+}
+
+extern "C" omni_status omnipage_compact_units_batched(omnitide_ctx* ctx, void* stream, const void* const* k_src,
+                                                      const void* const* v_src, void* const* k_dst, void* const* v_dst,
+                                                      int32_t n_layers, const omni_unit* units, const int32_t* n_units_dev,
+                                                      int32_t n_units_max, const uint8_t* unit_keep, int32_t s_span_max,
+                                                      int32_t page_size, const omni_unit* units_kept,
+                                                      const int32_t* n_units_kept_dev, int32_t* slot_map_out,
+                                                      omni_compact_info* info_out, uint8_t* page_class_out) {
+    if (!ctx) return OMNI_ERR_INVALID_ARG;
+    if (!units || !unit_keep || n_units_max <= 0 || s_span_max < 0 || page_size <= 0 || n_layers <= 0 || !k_src || !v_src ||
+        !k_dst || !v_dst)
+        OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "compact_units_batched: bad unit table/span/page/layers");
+    if (s_span_max > ctx->g.s_cap) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "compact_units_batched: s_span_max %d > s_cap %d", s_span_max, ctx->g.s_cap);
+    if (n_units_max > ctx->g.u_cap) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "compact_units_batched: n_units_max > u_cap");
+    if (2ll * s_span_max * n_layers >= (1ll << 31))
+        OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "compact_units_batched: 2 * s_span_max * n_layers must stay below 2^31");
+    if (ctx->row_bytes < 512 || (ctx->row_bytes & 15))
+        OMNI_FAIL(ctx, OMNI_ERR_UNSUPPORTED, "compact_units_batched: rows of at least 512 bytes (a multiple of 16) only");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CompactUnitsArgs a;
+    a.k_src = a.v_src = nullptr; a.k_dst = a.v_dst = nullptr;
+    a.units = units; a.n_units_dev = n_units_dev; a.n_units_max = n_units_max; a.unit_keep = unit_keep;
+    a.s_span_max = s_span_max; a.page_size = page_size; a.row_bytes = (int)ctx->row_bytes;
+    a.vpr = (int)(ctx->row_bytes >> 4); a.vpr_shift = -1;
+    a.units_kept = units_kept; a.n_units_kept_dev = n_units_kept_dev;
+    a.slot_map = slot_map_out; a.info = info_out; a.page_class = page_class_out; a.status = ctx->status_dev;
+    a.n_layers = n_layers;
+    a.k_src_l = reinterpret_cast<const char* const*>(k_src); a.v_src_l = reinterpret_cast<const char* const*>(v_src);
+    a.k_dst_l = reinterpret_cast<char* const*>(k_dst); a.v_dst_l = reinterpret_cast<char* const*>(v_dst);
+    const int grid = ctx->sm_count;
+    a.rows_cap = 4;                                          // no per-row source list in the batched form
+    const size_t smem_lists_al = ((((size_t)3 * n_units_max + 8 + a.rows_cap) * sizeof(int)) + 127) & ~(size_t)127;
+    const size_t budget = 200 * 1024;
+    if (smem_lists_al + 2 * CP_WARPS * ctx->row_bytes > budget)
+        OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "compact_units_batched: unit table or rows too large for one launch");
+    const size_t per_warp = (budget - smem_lists_al) / CP_WARPS;
+    a.n_slots = (int)std::min<size_t>(CP_MAX_SLOTS, per_warp / ctx->row_bytes);
+    const size_t smem = smem_lists_al + (size_t)a.n_slots * CP_WARPS * ctx->row_bytes;
+    if (smem > 48 * 1024)
+        OMNI_CUDA(ctx, cudaFuncSetAttribute(compact_units_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    compact_units_kernel<true><<<grid, CP_THREADS, smem, st>>>(a);
+    OMNI_CHECK_LAUNCH(ctx, "compact_units_kernel(batched)");
     return OMNI_OK;
 }
 

@@ -157,6 +157,46 @@ def test_compact_units_bit_exact(H, ob, U, max_len, rowshape, dtype, page, densi
     ctx.close()
 
 
+@pytest.mark.parametrize("n_layers,U,max_len,density,seed", [(1, 9, 200, 0.5, 0), (3, 40, 700, 0.3, 1), (5, 70, 300, 0.9, 2),
+                                                             (4, 12, 500, 0.0, 3)])
+def test_compact_units_batched_bit_exact(H, ob, n_layers, U, max_len, density, seed):
+    """Cross-layer batching: every layer's packed cache equals the oracle's pack of that layer with the shared mask."""
+    rng = np.random.default_rng(200 + seed)
+    units = _random_table(rng, U)
+    units[:, 1] = rng.integers(1, max_len + 1, size=U)
+    units[:, 0] = np.concatenate([[0], np.cumsum(units[:-1, 1])])
+    S = int(units[:, 1].sum())
+    keep_u = np.where(rng.random(U) < density, 2, 0).astype(np.uint8)
+    mask = np.repeat(keep_u != 0, units[:, 1]).astype(np.uint8)
+    rowshape, page = (8, 128), 64
+    raw = rng.integers(0, 256, size=(n_layers, 2, S, rowshape[0] * rowshape[1] * 2), dtype=np.uint8)
+    ks = [torch.from_numpy(raw[l, 0]).cuda().view(torch.bfloat16).view(S, *rowshape).contiguous() for l in range(n_layers)]
+    vs = [torch.from_numpy(raw[l, 1]).cuda().view(torch.bfloat16).view(S, *rowshape).contiguous() for l in range(n_layers)]
+    kd = [torch.zeros_like(k) for k in ks]
+    vd = [torch.zeros_like(v) for v in vs]
+    ptrs = lambda ts: torch.tensor([t.data_ptr() for t in ts], dtype=torch.int64, device="cuda")
+    ctx = ob.Context(32, 8, 128, "bf16", S + 64, U + 8, 16)
+    du = ob.units_to_device(units, U + 4)
+    keep = torch.full((U + 20,), 2, dtype=torch.uint8, device="cuda")
+    keep[:U] = torch.from_numpy(keep_u).cuda()
+    slot_map = torch.full((S + 16,), -5, dtype=torch.int32, device="cuda")
+    info = torch.full((8,), -5, dtype=torch.int32, device="cuda")
+    ctx.compact_units_batched(ptrs(ks), ptrs(vs), ptrs(kd), ptrs(vd), n_layers, du, H.i32(U), U + 4, keep, S, page, None, None,
+                              slot_map, info, None)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    got = ob.info_to_dict(info)
+    for l in range(n_layers):
+        exp = oc.compact_pack(raw[l, 0], raw[l, 1], mask, page)
+        n = exp["n_kept"]
+        assert (got["n_kept"], got["span_pages"], got["rows_moved"]) == (n, exp["span_pages"], exp["rows_moved"])
+        if n:
+            assert np.array_equal(H.bytes_of(kd[l][:n]).reshape(n, -1), exp["k"]), l
+            assert np.array_equal(H.bytes_of(vd[l][:n]).reshape(n, -1), exp["v"]), l
+        assert np.array_equal(slot_map[:S].cpu().numpy(), exp["slot_map"])
+    ctx.close()
+
+
 def test_compact_units_rejects_bad_tables(H, ob):
     rng = np.random.default_rng(5)
     units = wl.make_units([(100, 0, 0), (50, 1, 1), (70, 0, 2)])
