@@ -451,6 +451,26 @@ def main():
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                 "note": "attention FLOPs of the step over the whole host-buffer pass (copies + 5 stages)"},
     }
+    # ---- decode-phase attention: one new token against the compacted history (GQA-packed tile path), cache sets rotated
+    d_reps = max(8, min(args.steps, 40))
+    devs = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(d_reps)]
+    o1 = torch.empty((1, w.h_q, w.d), dtype=torch.float32, device="cuda")
+    for i in range(3 + d_reps):
+        s_ = sets[i % R]
+        if i >= 3:
+            devs[i - 3][0].record()
+        ctx.chunk_attention(s_["q"][:1], 1, s_["k_out"], s_["v_out"], n_kept, N, s_["kc"][:1], s_["vc"][:1], 0.0, o1, ob.DTYPE_FP32)
+        if i >= 3:
+            devs[i - 3][1].record()
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0, "device status word not clean after the decode steps"
+    dec_ms = max_over_ranks([float(np.mean([a_.elapsed_time(b_) for a_, b_ in devs]))], world, "cuda")[0]
+    dec_bytes = 2.0 * (kept + 1) * w.h_kv * w.d * 2 + 2.0 * w.h_q * w.d * 2 + w.h_q * w.d * 4
+    line["kernels"]["decode_attention"] = {
+        "bound": "hbm", "achieved": dec_bytes / (dec_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+        "frac": dec_bytes / (dec_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "ms": dec_ms, "bytes": dec_bytes,
+        "note": f"omnitide_chunk_attention with t = 1 over {kept} retained rows (K and V read once per KV group), merge kernel included"}
+
     # ---- cross-layer batched compaction: the same unit decision applied to the K/V caches of 36 layers in one launch
     batched = None
     if args.batch_layers > 0:

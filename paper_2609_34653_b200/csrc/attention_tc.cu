@@ -75,6 +75,7 @@ struct AttnParams {
     void* o_out; int out_dtype; float* lse_out;
     int32_t* status;
     int n_tiles;          // query tiles of 128 rows
+    int pack_shift;       // >= 0: GQA-packed single tile, row r = (token r >> pack_shift, head of the group r & (G-1)); -1: off
     float* part_o;        // [cta][2 slots][128 rows][128] un-normalised partial outputs
     float2* part_ml;      // [cta][2 slots][128 rows] (running max, sum)
 };
@@ -174,7 +175,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const bool tail_partial = nhb > 0 && hist_tail < BK;
 
     PartIter it;
-    it.s.nhb = nhb; it.s.n_tiles = p.n_tiles; it.s.h_q = p.h_q;
+    // GQA-packed mode (few queries, e.g. decode): one tile holds all query heads of a KV group, items are KV heads
+    const bool packed = p.pack_shift >= 0;
+    it.s.nhb = nhb; it.s.n_tiles = p.n_tiles; it.s.h_q = packed ? p.h_kv : p.h_q;
     {
         const long long total = it.s.total();
         it.w = share_begin(total, blockIdx.x, gridDim.x);
@@ -246,10 +249,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 // the Q tile is free once every MMA of the previous part has completed
                 if (part_idx > 0) ok = tc::mbar_wait(tc::smem_u32(&bars->o_done), (part_idx - 1) & 1, abort_flag);
                 if (!ok) break;
-                kvh = part.head / (p.h_q / p.h_kv);
+                kvh = packed ? part.head : part.head / (p.h_q / p.h_kv);
                 tc::mbar_expect_tx(tc::smem_u32(&bars->q_full), TILE_BYTES);
-                tc::tma_load_2d(q_smem, &tm_q, part.head * HD, part.qt * BQ, tc::smem_u32(&bars->q_full));
-                tc::tma_load_2d(q_smem + HALF_BYTES, &tm_q, part.head * HD + 64, part.qt * BQ, tc::smem_u32(&bars->q_full));
+                if (packed) {
+                    const int h0 = kvh << p.pack_shift;      // first query head of the group
+                    tc::tma_load_3d(q_smem, &tm_q, 0, h0, 0, tc::smem_u32(&bars->q_full));
+                    tc::tma_load_3d(q_smem + HALF_BYTES, &tm_q, 64, h0, 0, tc::smem_u32(&bars->q_full));
+                } else {
+                    tc::tma_load_2d(q_smem, &tm_q, part.head * HD, part.qt * BQ, tc::smem_u32(&bars->q_full));
+                    tc::tma_load_2d(q_smem + HALF_BYTES, &tm_q, part.head * HD + 64, part.qt * BQ, tc::smem_u32(&bars->q_full));
+                }
                 const int n = part.j1 - part.j0;
                 load_tile(part.j0, false);
                 if (ok && n > 1) load_tile(part.j0 + 1, false);
@@ -385,7 +394,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 // masking of this warpgroup's 64 keys: ragged history tail, causal diagonal
                 int n_valid = HK;
                 if (j == nhb - 1 && tail_partial) n_valid = hist_tail - w * HK;
-                if (j == diag_block) n_valid = r + 1 - w * HK;             // <= 0: the row sees nothing of this half
+                if (j == diag_block) n_valid = (packed ? (r >> p.pack_shift) : r) + 1 - w * HK;   // <= 0: the row sees nothing of this half
                 if (n_valid < HK) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
@@ -504,7 +513,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const float L = w_own * l_sum + w_oth * other.y;
             const float inv = part.final_ ? 1.f / L : 1.f;
             const uint32_t o_oth = tmem + 256 + (w ^ 1) * 128 + lane_addr;
-            const int row = part.qt * BQ + r;
+            // output row and head of this TMEM lane
+            const int row = packed ? (r >> p.pack_shift) : part.qt * BQ + r;
+            const int out_head = packed ? (part.head << p.pack_shift) + (r & ((1 << p.pack_shift) - 1)) : part.head;
             const size_t pslot = (size_t)blockIdx.x * 2 + part.slot;
             // this warpgroup writes output columns [64 w, 64 w + 64)
 #pragma unroll
@@ -523,12 +534,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     v[i] = (va + vb) * inv;
                 }
                 const int col = w * 64 + c * 32;
+                if (row >= p.t) continue;                    // padding row of the tile: nothing reads it
                 if (!part.final_) {
                     float4* dst = reinterpret_cast<float4*>(p.part_o + (pslot * BQ + r) * HD + col);
 #pragma unroll
                     for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-                } else if (row < p.t) {
-                    const size_t off = ((size_t)row * p.h_q + part.head) * HD + col;
+                } else {
+                    const size_t off = ((size_t)row * p.h_q + out_head) * HD + col;
                     if (p.out_dtype == OMNI_DTYPE_FP32) {
                         float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o_out) + off);
 #pragma unroll
@@ -543,8 +555,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
             }
             if (ok && w == 0) {
-                if (!part.final_) p.part_ml[pslot * BQ + r] = make_float2(M, L);
-                else if (p.lse_out && row < p.t) p.lse_out[(size_t)row * p.h_q + part.head] = M * p.scale + logf(L);
+                if (!part.final_) { if (row < p.t) p.part_ml[pslot * BQ + r] = make_float2(M, L); }
+                else if (p.lse_out && row < p.t) p.lse_out[(size_t)row * p.h_q + out_head] = M * p.scale + logf(L);
             }
             // O (and the part's Q tile) may be reused; the exchange buffer too, once both warpgroups are here
             tc::tcgen05_fence_before();
@@ -578,33 +590,42 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 // a warp owns 4 rows and a lane 4 of a row's 128 columns.  Shared memory: one int per CTA of the main kernel.
 constexpr int MERGE_BATCH = 4;
 __global__ void __launch_bounds__(256) attention_merge_kernel(const AttnParams p, int n_cta) {
-    extern __shared__ int s_slot[];                          // partial slot of every part of the item
+    extern __shared__ __align__(16) int s_slot[];            // partial slot of every part of the item
     __shared__ int s_n, s_qt, s_head;
     // blockIdx.x + 1 = b: the boundary between the shares of CTA b-1 and CTA b of the main kernel.  An item is
     // cut only where a boundary falls strictly inside it, so the boundaries enumerate the cut items; an item
     // that holds several boundaries is merged by the first of them.
+    // rows of this CTA's group of 32 that exist at all (a packed tile of a short chunk is mostly padding)
+    {
+        const int r_first = blockIdx.y * 32;
+        const int row_first = p.pack_shift >= 0 ? (r_first >> p.pack_shift) : 0;
+        if (p.pack_shift >= 0 && row_first >= p.t) return;
+    }
+    int n_hist = p.n_hist_dev ? *p.n_hist_dev : p.n_hist_max;
+    n_hist = max(0, min(n_hist, p.n_hist_max));
+    Sched s;
+    s.nhb = (n_hist + BK - 1) / BK; s.n_tiles = p.n_tiles; s.h_q = p.pack_shift >= 0 ? p.h_kv : p.h_q;
+    const long long total = s.total();
+    // share boundaries, one per thread (the divisions run in parallel), kept behind the slot list
+    long long* s_begin = reinterpret_cast<long long*>(s_slot + ((n_cta + 2) & ~1));         // [n_cta + 1]
+    for (int bb = threadIdx.x; bb <= n_cta; bb += blockDim.x) s_begin[bb] = share_begin(total, bb, n_cta);
+    __syncthreads();
     if (threadIdx.x == 0) {
-        int n_hist = p.n_hist_dev ? *p.n_hist_dev : p.n_hist_max;
-        n_hist = max(0, min(n_hist, p.n_hist_max));
-        Sched s;
-        s.nhb = (n_hist + BK - 1) / BK; s.n_tiles = p.n_tiles; s.h_q = p.h_q;
-        const long long total = s.total();
         const int b = blockIdx.x + 1;
-        const long long w = share_begin(total, b, n_cta);
+        const long long w = s_begin[b];
         int n = 0, qt = 0, head = 0, j = 0;
         if (w > 0 && w < total) {
             s.locate(w, qt, head, j);
             const long long w0 = w - j, w1 = w0 + s.nb_item(qt);            // the item is [w0, w1)
-            if (j > 0 && share_begin(total, b - 1, n_cta) <= w0) {
+            if (j > 0 && s_begin[b - 1] <= w0) {
                 // first part: the non-empty share that holds w0 (slot 1); then every non-empty share that
                 // starts inside the item (slot 0)
                 int bf = b - 1;
-                while (bf > 0 && share_begin(total, bf, n_cta) == share_begin(total, bf + 1, n_cta)) --bf;
+                while (bf > 0 && s_begin[bf] == s_begin[bf + 1]) --bf;
                 s_slot[n++] = bf * 2 + 1;
                 for (int bb = b; bb < n_cta; ++bb) {
-                    const long long wb = share_begin(total, bb, n_cta);
-                    if (wb >= w1) break;
-                    if (wb != share_begin(total, bb + 1, n_cta)) s_slot[n++] = bb * 2;
+                    if (s_begin[bb] >= w1) break;
+                    if (s_begin[bb] != s_begin[bb + 1]) s_slot[n++] = bb * 2;
                 }
             }
         }
@@ -617,7 +638,9 @@ __global__ void __launch_bounds__(256) attention_merge_kernel(const AttnParams p
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int q4 = 0; q4 < 4; ++q4) {
         const int r = blockIdx.y * 32 + warp * 4 + q4;       // row of the tile
-        const int row = qt * BQ + r;
+        const bool packed = p.pack_shift >= 0;
+        const int row = packed ? (r >> p.pack_shift) : qt * BQ + r;
+        const int out_head = packed ? (head << p.pack_shift) + (r & ((1 << p.pack_shift) - 1)) : head;
         if (row >= p.t) continue;
         float M = -INFINITY;
         for (int i = 0; i < n_parts; ++i) {
@@ -648,7 +671,7 @@ __global__ void __launch_bounds__(256) attention_merge_kernel(const AttnParams p
             }
         }
         const float inv = 1.f / L;
-        const size_t off = ((size_t)row * p.h_q + head) * HD + lane * 4;
+        const size_t off = ((size_t)row * p.h_q + out_head) * HD + lane * 4;
         if (p.out_dtype == OMNI_DTYPE_FP32) {
             *reinterpret_cast<float4*>(static_cast<float*>(p.o_out) + off) =
                 make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
@@ -658,7 +681,7 @@ __global__ void __launch_bounds__(256) attention_merge_kernel(const AttnParams p
             v.y = tc::pack_bf16x2(acc.z * inv, acc.w * inv);
             *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.o_out) + off) = v;
         }
-        if (p.lse_out && lane == 0) p.lse_out[(size_t)row * p.h_q + head] = M * p.scale + logf(L);
+        if (p.lse_out && lane == 0) p.lse_out[(size_t)row * p.h_q + out_head] = M * p.scale + logf(L);
     }
 }
 
@@ -670,7 +693,14 @@ omni_status omni_attention_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q,
     const omni_geometry& g = ctx->g;
     CUtensorMap tm_q, tm_kh, tm_vh, tm_kc, tm_vc;
     const uint64_t q_inner = (uint64_t)g.h_q * HD, kv_inner = (uint64_t)g.h_kv * HD;
-    bool ok = omni_make_map_bf16(ctx->encode_tiled, &tm_q, q, t, q_inner, BQ);
+    // few queries (decode, short chunks): all query heads of a KV group share one 128-row tile, so K and V are read
+    // once per group and the tile is not 127/128 padding
+    const int G = g.h_q / g.h_kv;
+    int pack_shift = -1;
+    if ((G & (G - 1)) == 0 && G <= BQ && (long long)t * G <= BQ)
+        for (int sft = 0; sft < 8; ++sft) if ((1 << sft) == G) pack_shift = sft;
+    bool ok = pack_shift >= 0 ? omni_make_map_q_packed(ctx->encode_tiled, &tm_q, q, t, g.h_q, G)
+                              : omni_make_map_bf16(ctx->encode_tiled, &tm_q, q, t, q_inner, BQ);
     ok &= omni_make_map_bf16(ctx->encode_tiled, &tm_kc, k_chunk, t, kv_inner, BK);
     ok &= omni_make_map_bf16(ctx->encode_tiled, &tm_vc, v_chunk, t, kv_inner, BK);
     // with an empty history the history maps are never used; point them at the chunk to stay valid
@@ -681,10 +711,12 @@ omni_status omni_attention_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q,
     p.t = t; p.h_q = g.h_q; p.h_kv = g.h_kv; p.n_hist_dev = n_hist_dev; p.n_hist_max = n_hist_max;
     p.scale = scale; p.scale_log2 = scale * 1.4426950408889634f;
     p.o_out = o_out; p.out_dtype = out_dtype; p.lse_out = lse_out; p.status = ctx->status_dev;
-    p.n_tiles = (t + BQ - 1) / BQ;
+    p.pack_shift = pack_shift;
+    p.n_tiles = pack_shift >= 0 ? 1 : (t + BQ - 1) / BQ;
+    const int n_items_heads = pack_shift >= 0 ? g.h_kv : g.h_q;
     // one CTA per SM, fewer when the whole job is small (at least 4 block steps per CTA)
     const long long nhb_max = (n_hist_max + BK - 1) / BK;
-    const long long w_max = (long long)g.h_q * ((long long)p.n_tiles * (nhb_max + 1) + (long long)p.n_tiles * (p.n_tiles - 1) / 2);
+    const long long w_max = (long long)n_items_heads * ((long long)p.n_tiles * (nhb_max + 1) + (long long)p.n_tiles * (p.n_tiles - 1) / 2);
     const int n_cta = (int)std::max(1ll, std::min((long long)ctx->sm_count, w_max / 4));
     p.part_o = ctx->attn_part_o; p.part_ml = reinterpret_cast<float2*>(ctx->attn_part_ml);
     if (!ctx->attn_attr_set) {                               // per context, hence per device
@@ -695,7 +727,7 @@ omni_status omni_attention_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q,
     OMNI_CHECK_LAUNCH(ctx, "attention_tc_kernel");
     if (n_cta > 1) {
         // one CTA row per boundary between two shares: only an item cut there has partials to merge
-        attention_merge_kernel<<<dim3(n_cta - 1, 4), 256, (n_cta + 1) * sizeof(int), st>>>(p, n_cta);
+        attention_merge_kernel<<<dim3(n_cta - 1, 4), 256, (n_cta + 2) * sizeof(int) + (n_cta + 1) * sizeof(long long), st>>>(p, n_cta);
         OMNI_CHECK_LAUNCH(ctx, "attention_merge_kernel");
     }
     return OMNI_OK;

@@ -72,6 +72,11 @@ __device__ __forceinline__ void tma_load_2d(uint32_t smem_dst, const CUtensorMap
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t smem_dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
@@ -261,6 +266,21 @@ static inline bool omni_make_map_bf16(void* encode_fn, CUtensorMap* map, const v
     cuuint32_t estr[2] = {1, 1};
     CUresult r = reinterpret_cast<omni_encode_tiled_fn>(encode_fn)(
         map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+// Q [T][h_q][128] bf16 seen as (dim, head, token): a box of {64 dims, g heads, 128 / g tokens} lands in shared memory as
+// 128 rows of 128 bytes ordered (token, head of the group), the tile of the GQA-packed attention path.
+static inline bool omni_make_map_q_packed(void* encode_fn, CUtensorMap* map, const void* base, uint64_t t, uint64_t h_q,
+                                          uint32_t g) {
+    cuuint64_t dims[3] = {128, h_q, t ? t : 1};
+    cuuint64_t strides[2] = {128 * 2, h_q * 128 * 2};
+    cuuint32_t box[3] = {64, g, 128 / g};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = reinterpret_cast<omni_encode_tiled_fn>(encode_fn)(
+        map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;

@@ -295,6 +295,14 @@ def test_attention_cuda_core_bf16(H, ob, seed, d, t, n_hist):
     (256, 0, 4, 4),         # no history: plain causal self-attention
     (690, 4080, 8, 2),      # config-2 chunk and kept-history sizes
     (1, 1, 4, 2),
+    # few queries: the GQA-packed tile (all query heads of a KV group in one 128-row tile)
+    (1, 8191, 32, 8),       # decode over the config-3 retained history
+    (1, 0, 8, 2),           # decode with an empty history: the token attends to itself
+    (4, 5000, 32, 8),       # 4 tokens x 4 heads = 16 rows of the tile
+    (32, 1000, 32, 8),      # exactly fills the packed tile
+    (33, 1000, 32, 8),      # one token too many: falls back to one tile per head
+    (16, 300, 8, 1),        # G = 8
+    (5, 129, 12, 4),        # G = 3 is not a power of two: not packed
 ])
 def test_attention_tensor_core(H, ob, t, n_hist, h_q, h_kv):
     rng = np.random.default_rng(t * 7 + n_hist)
