@@ -29,6 +29,15 @@ What follows the paper and what does not
                        score-ordered greedy fill that the paper does NOT
                        define.  PARITY UNPINNED for the greedy order; pinned
                        only by invariants, special cases and brute force.
+* plan_structural   -- OmniPick as the paper describes it (Section 5.1): no
+                       scores; recent events whole, older events reduced to
+                       boundary spans, per-modality sink prefixes and text under
+                       a shared budget, then whole events dropped oldest first
+                       (partially retained before complete) down to the low
+                       watermark.  Prefix lengths, budgets and what counts as a
+                       boundary span are parameters the paper leaves open;
+                       pinned by a hand-worked example, an independent
+                       token-level replay and invariants.
 * score_units       -- the paper's OmniPick collects no attention scores at
                        run time; the statistic scored here is the one its
                        design study measures offline (attention weight from
@@ -46,7 +55,9 @@ import numpy as np
 # unit-table columns
 U_START, U_LEN, U_MOD, U_EVENT, U_GROUP, U_FLAGS = range(6)
 GRP_MUST_KEEP, GRP_SELECTED, GRP_RECENT = 0, 1, 2
-KEEP_DROPPED, KEEP_WHOLE = 0, 2          # code 1 (sink prefix only) is reserved
+KEEP_DROPPED, KEEP_SINK_PREFIX, KEEP_WHOLE = 0, 1, 2
+FLAG_BOUNDARY = 1                         # unit.flags bit 0: a boundary span (kept whole while its event survives)
+MOD_VIDEO, MOD_AUDIO, MOD_TEXT = 0, 1, 2
 PAGE_EMPTY = 255
 
 
@@ -173,6 +184,98 @@ def select_units(units, scores, budget, n_recent_events=1, modality_cap=(-1, -1,
             pos += ln
     units_out = np.asarray(units_out, dtype=np.int32).reshape(-1, 6)
     return dict(unit_keep=keep, keep_mask=keep_mask, n_kept=pos, units_out=units_out, order=order)
+
+
+# ---------------------------------------------------------------------------
+# P -- structure-aware, score-free retention planning (OmniPick as written)
+# ---------------------------------------------------------------------------
+def plan_structural(units, high_watermark, low_watermark, n_recent_events, sink_prefix, text_budget):
+    """The paper's retention plan, from unit metadata alone (Section 5.1).
+
+    An *event* (the paper's "unit": one input chunk or one response) is the run
+    of typed spans (rows of `units`) that share an event id.
+
+    0. Retention starts only when the history exceeds the high watermark;
+       otherwise everything is kept.
+    1. Spans of the must-keep group (the protected system prefix) are kept
+       whole and never dropped.  The `n_recent_events` newest events are kept
+       whole ("keeping recent units intact").
+    2. Older events, oldest to newest ("selecting spans from older units"):
+       a boundary span is kept whole; an image/video or audio span keeps only
+       its first `sink_prefix[modality]` tokens (a candidate sink); text spans
+       are kept whole, oldest to newest, until their shared token budget is
+       exhausted (the first text span that does not fit and all later ones of
+       the older events are dropped).
+    3. If the selection still exceeds the low watermark, whole events are
+       dropped oldest first, partially retained events before complete ones;
+       the walk stops when the target is met or only one event remains: the
+       low watermark is a trimming target, not a strict bound.
+    4. Survivors are re-indexed as in `select_units` (Section 5.2); a shortened
+       span keeps its modality, event and flags with its new length.
+
+    Returns dict(unit_keep[U] u8 (0 dropped, 1 sink prefix only, 2 whole),
+    unit_kept_len[U] i32, keep_mask[N] u8, n_kept, units_out[U', 6]).
+    """
+    units = np.asarray(units, dtype=np.int64)
+    U = len(units)
+    lens = units[:, U_LEN]
+    events = units[:, U_EVENT]
+    if U > 1 and np.any(np.diff(events) < 0):
+        raise ValueError("event ids must be non-decreasing in unit order")
+    n_hist = int(lens.sum())
+    kept = lens.copy()
+    must = units[:, U_GROUP] == GRP_MUST_KEEP
+    distinct = sorted(set(int(e) for e in events))
+    recent = set(distinct[max(0, len(distinct) - n_recent_events):]) if n_recent_events > 0 else set()
+    is_recent = np.array([int(e) in recent for e in events], dtype=bool)
+
+    if n_hist > high_watermark:
+        text_used = 0
+        text_open = True
+        for u in range(U):                                   # oldest to newest
+            if must[u] or is_recent[u]:
+                continue
+            mod = int(units[u, U_MOD])
+            if int(units[u, U_FLAGS]) & FLAG_BOUNDARY:
+                continue                                     # kept whole
+            if mod == MOD_TEXT:
+                if text_open and text_used + int(lens[u]) <= text_budget:
+                    text_used += int(lens[u])
+                else:
+                    text_open = False
+                    kept[u] = 0
+            else:
+                kept[u] = min(int(lens[u]), int(sink_prefix[mod]))
+        total = int(kept.sum())
+        if total > low_watermark:
+            # events that can be dropped, with what they hold outside the protected prefix
+            ev_units = {e: [u for u in range(U) if int(events[u]) == e and not must[u]] for e in distinct}
+            alive = [e for e in distinct if sum(int(kept[u]) for u in ev_units[e]) > 0]
+            partial = [e for e in alive if any(kept[u] < lens[u] for u in ev_units[e])]
+            complete = [e for e in alive if e not in partial]
+            n_alive = len(alive)
+            for e in partial + complete:                     # oldest first within each class
+                if total <= low_watermark or n_alive <= 1:
+                    break
+                for u in ev_units[e]:
+                    total -= int(kept[u])
+                    kept[u] = 0
+                n_alive -= 1
+
+    keep = np.where(kept == 0, KEEP_DROPPED, np.where(kept == lens, KEEP_WHOLE, KEEP_SINK_PREFIX)).astype(np.uint8)
+    keep_mask = np.zeros(n_hist, dtype=np.uint8)
+    units_out = []
+    pos = 0
+    for u in range(U):
+        k = int(kept[u])
+        if k > 0:
+            st = int(units[u, U_START])
+            keep_mask[st:st + k] = 1
+            g = GRP_MUST_KEEP if must[u] else (GRP_RECENT if is_recent[u] else GRP_SELECTED)
+            units_out.append((pos, k, int(units[u, U_MOD]), int(events[u]), g, int(units[u, U_FLAGS])))
+            pos += k
+    units_out = np.asarray(units_out, dtype=np.int32).reshape(-1, 6)
+    return dict(unit_keep=keep, unit_kept_len=kept.astype(np.int32), keep_mask=keep_mask, n_kept=pos, units_out=units_out)
 
 
 # ---------------------------------------------------------------------------

@@ -437,3 +437,144 @@ def test_tiny_config_ranking_is_nontrivial():
     assert sel["n_kept"] <= w.budget
     cp = oc.compact_pack(w.k_hist, w.v_hist, sel["keep_mask"], w.page_size, sel["units_out"])
     assert 0 <= cp["span_pages"] * w.page_size - cp["n_kept"] < w.page_size
+
+
+# ------------------------------------------------------------------ structural retention planning
+def _toy_stream():
+    """4-token protected prefix, then four events of (video 10, audio 6[, text 3])."""
+    return np.array([[0, 4, 2, 0, 0, 0],
+                     [4, 10, 0, 1, 2, 0], [14, 6, 1, 1, 2, 0], [20, 3, 2, 1, 2, 0],
+                     [23, 10, 0, 2, 2, 0], [33, 6, 1, 2, 2, 0], [39, 3, 2, 2, 2, 0],
+                     [42, 10, 0, 3, 2, 0], [52, 6, 1, 3, 2, 0],
+                     [58, 10, 0, 4, 2, 0], [68, 6, 1, 4, 2, 0]], dtype=np.int32)
+
+
+def test_plan_structural_hand_worked():
+    """Section 5.1 worked by hand on an 11-span stream of 74 tokens: the two newest events stay whole, older
+    image/audio spans shrink to sink prefixes of 2 / 1 tokens, older text is kept oldest first under a shared
+    budget of 4 (the first 3-token span fits, the second does not), then whole events go, oldest first."""
+    u = _toy_stream()
+    # no drop phase needed: 4 + (2+1+3) + (2+1+0) + 16 + 16 = 45 <= 45
+    r = oc.plan_structural(u, 40, 45, 2, (2, 1, 0), 4)
+    assert r["unit_kept_len"].tolist() == [4, 2, 1, 3, 2, 1, 0, 10, 6, 10, 6]
+    assert r["unit_keep"].tolist() == [2, 1, 1, 2, 1, 1, 0, 2, 2, 2, 2]
+    assert r["n_kept"] == 45
+    assert r["units_out"][:, 0].tolist() == [0, 4, 6, 7, 10, 12, 13, 23, 29, 39]
+    assert r["units_out"][:, 4].tolist() == [0, 1, 1, 1, 1, 1, 2, 2, 2, 2]           # must-keep | selected | recent
+    mask = r["keep_mask"]
+    assert mask[:4].all() and mask[4:6].all() and not mask[6:14].any()               # image span keeps its first 2 tokens
+    assert mask[14] and not mask[15:20].any() and mask[20:23].all()                  # audio sink, then the text span
+    assert not mask[39:42].any() and mask[42:].all()
+    # target 40: one partially retained event (the oldest) is dropped, 45 - 6 = 39
+    r = oc.plan_structural(u, 40, 40, 2, (2, 1, 0), 4)
+    assert r["unit_kept_len"].tolist() == [4, 0, 0, 0, 2, 1, 0, 10, 6, 10, 6] and r["n_kept"] == 39
+    # target 30: both partially retained events go (36 left), then complete events oldest first: 20
+    r = oc.plan_structural(u, 40, 30, 2, (2, 1, 0), 4)
+    assert r["unit_kept_len"].tolist() == [4, 0, 0, 0, 0, 0, 0, 0, 0, 10, 6] and r["n_kept"] == 20
+    # target 5 cannot be met: the walk stops when one event remains; the prefix is never dropped
+    r = oc.plan_structural(u, 40, 5, 2, (2, 1, 0), 4)
+    assert r["unit_kept_len"].tolist() == [4, 0, 0, 0, 0, 0, 0, 0, 0, 10, 6]
+    # below the high watermark nothing happens
+    r = oc.plan_structural(u, 74, 10, 1, (0, 0, 0), 0)
+    assert r["unit_kept_len"].tolist() == u[:, 1].tolist() and r["keep_mask"].all() and (r["unit_keep"] == 2).all()
+    # a boundary span of an older event is kept whole while its event survives
+    ub = u.copy()
+    ub[1, 5] = oc.FLAG_BOUNDARY
+    r = oc.plan_structural(ub, 40, 60, 2, (2, 1, 0), 4)
+    assert r["unit_kept_len"].tolist() == [4, 10, 1, 3, 2, 1, 0, 10, 6, 10, 6]
+
+
+def _random_stream(rng, n_events, with_prefix=True):
+    spans = [(int(rng.integers(1, 9)), 2, 0)] if with_prefix else []
+    for e in range(1, n_events + 1):
+        for mod in (0, 1, 2):
+            if rng.random() < (0.9, 0.8, 0.4)[mod]:
+                spans.append((int(rng.integers(1, 40)), mod, e))
+        if not spans or spans[-1][2] != e:
+            spans.append((int(rng.integers(1, 40)), 0, e))
+    u = wl.make_units(spans, group_of_first=0 if with_prefix else None)
+    for i in range(len(u)):
+        if rng.random() < 0.1 and u[i, 4] != 0:
+            u[i, 5] |= oc.FLAG_BOUNDARY
+    return u
+
+
+def _token_level_replay(u, H, L, R, sink, Tb):
+    """The same rules replayed per TOKEN with array operations (a second derivation, no shared code)."""
+    lens = u[:, 1]
+    n = int(lens.sum())
+    tok_unit = np.repeat(np.arange(len(u)), lens)
+    tok_off = np.arange(n) - np.repeat(u[:, 0], lens)
+    if n <= H:
+        return np.ones(n, dtype=bool)
+    ev = u[tok_unit, 3]
+    mod = u[tok_unit, 2]
+    must = u[tok_unit, 4] == 0
+    bnd = (u[tok_unit, 5] & 1) == 1
+    ids = np.unique(u[:, 3])
+    recent_ids = ids[max(0, len(ids) - R):] if R > 0 else ids[:0]
+    rec = np.isin(ev, recent_ids)
+    keep = must | rec | (~must & ~rec & bnd)
+    older = ~must & ~rec & ~bnd
+    for m in (0, 1):
+        keep |= older & (mod == m) & (tok_off < sink[m])
+    # text: cumulative length of older text spans in time order, span by span
+    t_units = [i for i in range(len(u)) if u[i, 2] == 2 and u[i, 4] != 0 and u[i, 3] not in recent_ids and not (u[i, 5] & 1)]
+    csum = np.cumsum([int(u[i, 1]) for i in t_units]) if t_units else np.array([], dtype=int)
+    fits = csum <= Tb
+    if len(fits) and not fits.all():
+        fits[np.argmin(fits):] = False
+    for i, ok in zip(t_units, fits):
+        if ok:
+            keep[tok_unit == i] = True
+    # whole events, oldest first, partially retained ones before complete ones
+    full = np.array([keep[(tok_unit == i)].all() for i in range(len(u))])
+    droppable = lambda e: (ev == e) & ~must
+    alive = [e for e in ids if keep[droppable(e)].any()]
+    part = [e for e in alive if not all(full[i] for i in range(len(u)) if u[i, 3] == e and u[i, 4] != 0)]
+    comp = [e for e in alive if e not in part]
+    left = len(alive)
+    for e in part + comp:
+        if keep.sum() <= L or left <= 1:
+            break
+        keep[droppable(e)] = False
+        left -= 1
+    return keep
+
+
+def test_plan_structural_matches_token_level_replay_and_invariants():
+    rng = np.random.default_rng(515)
+    for trial in range(300):
+        u = _random_stream(rng, int(rng.integers(1, 9)), with_prefix=rng.random() < 0.8)
+        n = int(u[:, 1].sum())
+        H = int(rng.integers(0, n + 10))
+        L = int(rng.integers(0, H + 1))
+        R = int(rng.integers(0, 4))
+        sink = (int(rng.integers(0, 12)), int(rng.integers(0, 12)), 0)
+        Tb = int(rng.integers(0, 60))
+        r = oc.plan_structural(u, H, L, R, sink, Tb)
+        ref = _token_level_replay(u, H, L, R, sink, Tb)
+        assert np.array_equal(r["keep_mask"].astype(bool), ref), trial
+        kept, lens = r["unit_kept_len"], u[:, 1]
+        # a span survives as a prefix of itself; the mask is that prefix
+        assert ((kept >= 0) & (kept <= lens)).all()
+        for i in range(len(u)):
+            st = int(u[i, 0])
+            assert r["keep_mask"][st:st + kept[i]].all() and not r["keep_mask"][st + kept[i]:st + lens[i]].any()
+        # the protected prefix always survives whole
+        assert (kept[u[:, 4] == 0] == lens[u[:, 4] == 0]).all()
+        # survivors are re-indexed contiguously, in order, with their new lengths
+        uo = r["units_out"]
+        assert uo[:, 1].tolist() == [int(k) for k in kept if k > 0]
+        assert uo[:, 0].tolist() == np.concatenate([[0], np.cumsum(uo[:-1, 1])]).astype(int).tolist() if len(uo) else True
+        assert r["n_kept"] == int(kept.sum()) == int(r["keep_mask"].sum())
+        if n > H:
+            # stop rule: the target is met, or a single event is left beside the prefix
+            ev_alive = {int(u[i, 3]) for i in range(len(u)) if kept[i] > 0 and u[i, 4] != 0}
+            assert r["n_kept"] <= L or len(ev_alive) <= 1
+            # an older image/audio span keeps nothing or exactly its sink prefix
+            ids = np.unique(u[:, 3])
+            rec = set(ids[max(0, len(ids) - R):].tolist()) if R > 0 else set()
+            for i in range(len(u)):
+                if u[i, 4] != 0 and int(u[i, 3]) not in rec and not (u[i, 5] & 1) and u[i, 2] in (0, 1):
+                    assert kept[i] in (0, min(int(lens[i]), sink[int(u[i, 2])]))
