@@ -55,6 +55,7 @@ enum { OMNI_MOD_VIDEO = 0, OMNI_MOD_AUDIO = 1, OMNI_MOD_TEXT = 2 };
 enum { OMNI_GROUP_MUST_KEEP = 0, OMNI_GROUP_SELECTED = 1, OMNI_GROUP_RECENT = 2 };
 enum { OMNI_KEEP_DROPPED = 0, OMNI_KEEP_SINK_PREFIX = 1 /* reserved */, OMNI_KEEP_WHOLE = 2 };
 enum { OMNI_PAGE_EMPTY = 255 };
+enum { OMNI_FLAG_BOUNDARY = 1 };  /* omni_unit.flags bit 0: a boundary span (Section 5.1), kept whole while its event survives */
 enum { OMNI_COMPACT_PACK = 0 };
 
 typedef struct {
@@ -72,7 +73,7 @@ typedef struct {
     int32_t modality;   /* OMNI_MOD_* */
     int32_t event;      /* streaming event the span belongs to */
     int32_t group;      /* OMNI_GROUP_* */
-    int32_t flags;      /* opaque, carried through */
+    int32_t flags;      /* bit 0 = OMNI_FLAG_BOUNDARY; the other bits are opaque; carried through */
 } omni_unit;
 
 typedef struct {
@@ -80,6 +81,15 @@ typedef struct {
     int32_t n_recent_events;    /* newest events kept whole */
     int32_t modality_cap[3];    /* per-modality token cap on selected (non-protected) units; <0 = none */
 } omni_select_params;
+
+/* Parameters of the paper's own score-free retention plan (Section 5.1).  The paper leaves the values open. */
+typedef struct {
+    int32_t high_watermark;     /* retention starts only when the history exceeds it */
+    int32_t low_watermark;      /* trimming target (not a strict bound) */
+    int32_t n_recent_events;    /* newest events kept whole */
+    int32_t sink_prefix[3];     /* tokens kept at the start of an older image/video or audio span (text entry unused) */
+    int32_t text_budget;        /* tokens of older text spans kept, oldest first */
+} omni_structural_params;
 
 /* Integer results of one compaction, written to device memory. */
 typedef struct {
@@ -146,6 +156,29 @@ omni_status omnitide_select_units(omnitide_ctx* ctx, void* stream,
                                   int32_t* n_kept_out, omni_unit* units_out, int32_t* n_units_out);
 
 /*
+ * (next row: OmniPick as the paper describes it, Section 5.1 "Structure-aware retention planning") Score-free
+ * retention plan from unit metadata alone.  An event (the paper's "unit") is the run of spans that share an
+ * event id.
+ *   0. nothing happens unless the history exceeds high_watermark;
+ *   1. must-keep spans and the n_recent_events newest events are kept whole;
+ *   2. older events, oldest to newest: a boundary span (OMNI_FLAG_BOUNDARY) is kept whole, an image/video or
+ *      audio span keeps its first sink_prefix[modality] tokens, text spans are kept whole, oldest first, until
+ *      text_budget is exhausted (the first one that does not fit ends it);
+ *   3. while the plan still exceeds low_watermark, whole events are dropped oldest first, partially retained
+ *      events before complete ones, until the target is met or one event remains;
+ *   4. survivors are re-indexed (Section 5.2) as in omnitide_select_units; a shortened span keeps its record
+ *      with the new length.
+ * Outputs [dev]: unit_keep_out[n_units] (0 dropped, 1 sink prefix only, 2 whole), unit_kept_len_out[n_units]
+ * (nullable), keep_mask_out[n_hist] (nullable, 16-byte aligned), n_kept_out, units_out, n_units_out.
+ * Together with omnipage_compact_units(..., unit_kept_len, ...) this is the path with no scoring at all.
+ */
+omni_status omnitide_plan_structural(omnitide_ctx* ctx, void* stream,
+                                     const omni_unit* units, const int32_t* n_units_dev, int32_t n_units_max,
+                                     const omni_structural_params* params /*[host]*/,
+                                     uint8_t* unit_keep_out, int32_t* unit_kept_len_out, uint8_t* keep_mask_out,
+                                     int32_t n_hist_max, int32_t* n_kept_out, omni_unit* units_out, int32_t* n_units_out);
+
+/*
  * (a3) OmniPage eager compaction (Section 6, "Compaction-movement trade-off": pack every retained
  * entry into a contiguous prefix; Section 6.1 for allocation classes and page promotion; Section 6.2
  * for the page-rounded span and for copy semantics: reads of all sources precede all writes).
@@ -179,7 +212,9 @@ omni_status omnipage_compact(omnitide_ctx* ctx, void* stream,
  * but no mask is read: the gather is a list of at most n_units contiguous runs, so no CTA has to wait for
  * another one's count and the kernel starts copying after one round trip to the unit table.
  *   units [dev] the history unit table (contiguous, in order), n_units_dev [dev, nullable] / n_units_max [host];
- *   unit_keep [dev] n_units_max bytes (OMNI_KEEP_*); s_span_max [host] bound on the history length;
+ *   unit_keep [dev] n_units_max bytes (OMNI_KEEP_*); unit_kept_len [dev, nullable] n_units_max int32: the number of
+ *   tokens kept at the START of every unit (sink prefixes of omnitide_plan_structural; NULL = kept units are whole);
+ *   s_span_max [host] bound on the history length;
  *   units_kept / n_units_kept_dev: the re-indexed table of the survivors (for part_begin; nullable);
  *   slot_map_out [dev] s_span_max int32 (nullable), info_out [dev], page_class_out [dev] nullable, as above.
  * A unit that reaches outside [0, s_span_max) sets OMNI_DEV_BAD_UNITS and is treated as dropped.
@@ -187,7 +222,8 @@ omni_status omnipage_compact(omnitide_ctx* ctx, void* stream,
 omni_status omnipage_compact_units(omnitide_ctx* ctx, void* stream,
                                    const void* k_src, const void* v_src, void* k_dst, void* v_dst,
                                    const omni_unit* units, const int32_t* n_units_dev, int32_t n_units_max,
-                                   const uint8_t* unit_keep, int32_t s_span_max, int32_t page_size,
+                                   const uint8_t* unit_keep, const int32_t* unit_kept_len,
+                                   int32_t s_span_max, int32_t page_size,
                                    const omni_unit* units_kept, const int32_t* n_units_kept_dev,
                                    int32_t* slot_map_out, omni_compact_info* info_out, uint8_t* page_class_out);
 
@@ -203,7 +239,8 @@ omni_status omnipage_compact_units_batched(omnitide_ctx* ctx, void* stream,
                                            const void* const* k_src, const void* const* v_src,
                                            void* const* k_dst, void* const* v_dst, int32_t n_layers,
                                            const omni_unit* units, const int32_t* n_units_dev, int32_t n_units_max,
-                                           const uint8_t* unit_keep, int32_t s_span_max, int32_t page_size,
+                                           const uint8_t* unit_keep, const int32_t* unit_kept_len,
+                                           int32_t s_span_max, int32_t page_size,
                                            const omni_unit* units_kept, const int32_t* n_units_kept_dev,
                                            int32_t* slot_map_out, omni_compact_info* info_out, uint8_t* page_class_out);
 

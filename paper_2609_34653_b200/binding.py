@@ -30,6 +30,11 @@ class SelectParams(C.Structure):
     _fields_ = [("budget", C.c_int32), ("n_recent_events", C.c_int32), ("modality_cap", C.c_int32 * 3)]
 
 
+class StructuralParams(C.Structure):
+    _fields_ = [("high_watermark", C.c_int32), ("low_watermark", C.c_int32), ("n_recent_events", C.c_int32),
+                ("sink_prefix", C.c_int32 * 3), ("text_budget", C.c_int32)]
+
+
 class CompactInfo(C.Structure):
     _fields_ = [("n_kept", C.c_int32), ("span_pages", C.c_int32), ("rows_moved", C.c_int32),
                 ("part_begin", C.c_int32 * 4), ("reserved", C.c_int32)]
@@ -37,7 +42,7 @@ class CompactInfo(C.Structure):
 
 EXPORTS = [
     "omnitide_create", "omnitide_destroy", "omnitide_poll_status", "omnitide_last_error",
-    "omnitide_score_units", "omnitide_select_units", "omnipage_compact", "omnipage_compact_units", "omnipage_compact_units_batched", "omnipage_append",
+    "omnitide_score_units", "omnitide_select_units", "omnitide_plan_structural", "omnipage_compact", "omnipage_compact_units", "omnipage_compact_units_batched", "omnipage_append",
     "omnitide_chunk_attention", "omnitide_chunk_step", "omnitide_chunk_step_host",
     "omnitide_set_option", "omnitide_launch_count", "omnitide_score_units_noalloc",
 ]
@@ -62,6 +67,10 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.omnitide_score_units.argtypes = [vp, vp, vp, i32, vp, vp, i32, vp, vp, i32, C.POINTER(f32), f32, vp, vp]
     lib.omnitide_select_units.argtypes = [vp, vp, vp, vp, i32, vp, C.POINTER(SelectParams), vp, vp, i32, vp, vp, vp]
     lib.omnipage_compact.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, i32, vp, vp, vp]
+    lib.omnitide_plan_structural.argtypes = [vp, vp, vp, vp, i32, C.POINTER(StructuralParams), vp, vp, vp, i32, vp, vp, vp]
+    lib.omnipage_compact_units.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, i32, i32, vp, vp, vp, vp, vp]
+    lib.omnipage_compact_units_batched.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, vp, i32, vp, vp, i32, i32, vp, vp, vp,
+                                                   vp, vp]
     lib.omnipage_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, i32, vp, vp]
     lib.omnitide_chunk_attention.argtypes = [vp, vp, vp, i32, vp, vp, vp, i32, vp, vp, f32, vp, i32, vp]
     lib.omnitide_score_units_noalloc.argtypes = [vp, i32, i32, i32, i32, vp, i32, vp, i32, vp, i32, C.POINTER(f32), f32,
@@ -107,6 +116,12 @@ def _host_ptr(a):
 
 def _stream():
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def structural_params(high_watermark, low_watermark, n_recent_events, sink_prefix, text_budget) -> StructuralParams:
+    sp = [int(x) for x in sink_prefix] + [0] * (3 - len(sink_prefix))
+    return StructuralParams(int(high_watermark), int(low_watermark), int(n_recent_events), (C.c_int32 * 3)(*sp[:3]),
+                            int(text_budget))
 
 
 def select_params(budget, n_recent_events=1, modality_cap=(-1, -1, -1)) -> SelectParams:
@@ -167,6 +182,13 @@ class Context:
                                                    _ptr(keep_mask_out), n_hist_max, _ptr(n_kept_out), _ptr(units_out),
                                                    _ptr(n_units_out)), "omnitide_select_units")
 
+    def plan_structural(self, units, n_units_dev, n_units_max, params, unit_keep_out, unit_kept_len_out, keep_mask_out,
+                        n_hist_max, n_kept_out, units_out, n_units_out):
+        self._check(self.lib.omnitide_plan_structural(self._ctx, _stream(), _ptr(units), _ptr(n_units_dev), n_units_max,
+                                                      C.byref(params), _ptr(unit_keep_out), _ptr(unit_kept_len_out),
+                                                      _ptr(keep_mask_out), n_hist_max, _ptr(n_kept_out), _ptr(units_out),
+                                                      _ptr(n_units_out)), "omnitide_plan_structural")
+
     def compact(self, k_src, v_src, k_dst, v_dst, keep_mask, s_span_dev, s_span_max, page_size, units_kept,
                 n_units_kept_dev, n_units_max, slot_map_out, info_out, page_class_out, mode=0):
         self._check(self.lib.omnipage_compact(self._ctx, _stream(), _ptr(k_src), _ptr(v_src), _ptr(k_dst), _ptr(v_dst),
@@ -176,22 +198,22 @@ class Context:
                     "omnipage_compact")
 
     def compact_units(self, k_src, v_src, k_dst, v_dst, units, n_units_dev, n_units_max, unit_keep, s_span_max,
-                      page_size, units_kept, n_units_kept_dev, slot_map_out, info_out, page_class_out):
+                      page_size, units_kept, n_units_kept_dev, slot_map_out, info_out, page_class_out, unit_kept_len=None):
         self._check(self.lib.omnipage_compact_units(self._ctx, _stream(), _ptr(k_src), _ptr(v_src), _ptr(k_dst),
                                                     _ptr(v_dst), _ptr(units), _ptr(n_units_dev), n_units_max,
-                                                    _ptr(unit_keep), s_span_max, page_size, _ptr(units_kept),
+                                                    _ptr(unit_keep), _ptr(unit_kept_len), s_span_max, page_size, _ptr(units_kept),
                                                     _ptr(n_units_kept_dev), _ptr(slot_map_out), _ptr(info_out),
                                                     _ptr(page_class_out)),
                     "omnipage_compact_units")
 
     def compact_units_batched(self, k_src_ptrs, v_src_ptrs, k_dst_ptrs, v_dst_ptrs, n_layers, units, n_units_dev,
                               n_units_max, unit_keep, s_span_max, page_size, units_kept, n_units_kept_dev, slot_map_out,
-                              info_out, page_class_out):
+                              info_out, page_class_out, unit_kept_len=None):
         """k_src_ptrs ...: int64 CUDA tensors holding n_layers device pointers each."""
         self._check(self.lib.omnipage_compact_units_batched(
             self._ctx, _stream(), _ptr(k_src_ptrs), _ptr(v_src_ptrs), _ptr(k_dst_ptrs), _ptr(v_dst_ptrs), n_layers,
-            _ptr(units), _ptr(n_units_dev), n_units_max, _ptr(unit_keep), s_span_max, page_size, _ptr(units_kept),
-            _ptr(n_units_kept_dev), _ptr(slot_map_out), _ptr(info_out), _ptr(page_class_out)),
+            _ptr(units), _ptr(n_units_dev), n_units_max, _ptr(unit_keep), _ptr(unit_kept_len), s_span_max, page_size,
+            _ptr(units_kept), _ptr(n_units_kept_dev), _ptr(slot_map_out), _ptr(info_out), _ptr(page_class_out)),
             "omnipage_compact_units_batched")
 
     def append(self, k_cache, v_cache, n_kept_dev, k_chunk, v_chunk, t, units, n_units_dev, chunk_units,

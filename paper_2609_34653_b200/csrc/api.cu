@@ -186,7 +186,8 @@ static omni_status chunk_step_impl(cudaEvent_t chunk_kv_ready, omnitide_ctx* ctx
                               nullptr, n_hist_max, n_kept, units_out, n_units_kept);
     if (s) return s;
     s = omnipage_compact_units(ctx, stream, k_cache, v_cache, k_cache_out, v_cache_out, units, n_units_dev, n_units_max,
-                               ctx->ws_unit_keep, n_hist_max, page_size, units_out, n_units_kept, nullptr, info, nullptr);
+                               ctx->ws_unit_keep, nullptr, n_hist_max, page_size, units_out, n_units_kept, nullptr, info,
+                               nullptr);
     if (s) return s;
     // the chunk's K/V rows are first read here (scoring reads only Q and the cached keys)
     if (chunk_kv_ready) OMNI_CUDA(ctx, cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), chunk_kv_ready, 0));

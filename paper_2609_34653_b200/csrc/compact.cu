@@ -517,6 +517,7 @@ __global__ void __launch_bounds__(CP_THREADS, 1) compact_pack_kernel(const Compa
 struct CompactUnitsArgs {
     const char* k_src; const char* v_src; char* k_dst; char* v_dst;
     const omni_unit* units; const int32_t* n_units_dev; int n_units_max; const uint8_t* unit_keep;
+    const int32_t* unit_kept_len;   // nullable: tokens kept at the start of every unit (sink prefixes); else whole units
     int s_span_max; int page_size; int row_bytes; int vpr; int vpr_shift;
     const omni_unit* units_kept; const int32_t* n_units_kept_dev;
     int32_t* slot_map; omni_compact_info* info; uint8_t* page_class; int32_t* status;
@@ -543,11 +544,12 @@ __global__ void __launch_bounds__(CP_THREADS, 1) compact_units_kernel(const Comp
 
     // ---- prologue: all loads that need no device-side count first ------------------------------------------
     int nu = a.n_units_dev ? __ldg(a.n_units_dev) : a.n_units_max;
-    int u_start = 0, u_len = 0, u_keep = 0, k_len = 0, k_group = -1;
+    int u_start = 0, u_len = 0, u_keep = 0, u_klen = -1, k_len = 0, k_group = -1;
     if (tid < a.n_units_max) {
         u_start = __ldg(&a.units[tid].start);
         u_len = __ldg(&a.units[tid].len);
         u_keep = __ldg(a.unit_keep + tid);
+        if (a.unit_kept_len) u_klen = __ldg(a.unit_kept_len + tid);
     }
     int nuk = 0;
     if (a.units_kept) {
@@ -568,14 +570,19 @@ __global__ void __launch_bounds__(CP_THREADS, 1) compact_units_kernel(const Comp
     // kept length per unit; a unit outside [0, s_span_max) is an error and counts as dropped
     bool bad = false;
     for (int u = tid; u < nu; u += CP_THREADS) {
-        if (u >= CP_THREADS) { u_start = a.units[u].start; u_len = a.units[u].len; u_keep = a.unit_keep[u]; }
+        if (u >= CP_THREADS) {
+            u_start = a.units[u].start; u_len = a.units[u].len; u_keep = a.unit_keep[u];
+            u_klen = a.unit_kept_len ? a.unit_kept_len[u] : -1;
+        }
         const bool inside = u_start >= 0 && u_len > 0 && (long long)u_start + u_len <= a.s_span_max;
         bad |= !inside;
         const bool keep = inside && u_keep != OMNI_KEEP_DROPPED;
+        // tokens kept at the start of the unit: all of it, or the given prefix length
+        const int klen = !keep ? 0 : (a.unit_kept_len ? max(0, min(u_klen, u_len)) : u_len);
         ustart[u] = u_start;
         ulen[u] = inside ? u_len : 0;
-        prefix[u] = keep ? u_len : 0;
-        if (!keep) atomicMin(&s_misc[2], u);                 // first unit that is dropped (for rows_moved)
+        prefix[u] = klen;
+        if (klen < u_len) atomicMin(&s_misc[2], u);          // first unit with a dropped slot (for rows_moved)
         if (u == nu - 1) s_misc[3] = inside ? u_start + u_len : 0;   // end of the history
     }
     if (bad) atomicOr(a.status, OMNI_DEV_BAD_UNITS);
@@ -631,14 +638,14 @@ __global__ void __launch_bounds__(CP_THREADS, 1) compact_units_kernel(const Comp
     if (a.slot_map) {
         for (int u = blockIdx.x; u < nu; u += G) {
             const int st = ustart[u], ln = ulen[u];
-            const bool keep = prefix[u + 1] > prefix[u];
-            const int base = prefix[u];
-            for (int i = tid; i < ln; i += CP_THREADS) a.slot_map[st + i] = keep ? base + i : -1;
+            const int base = prefix[u], klen = prefix[u + 1] - prefix[u];
+            for (int i = tid; i < ln; i += CP_THREADS) a.slot_map[st + i] = i < klen ? base + i : -1;
         }
     }
     // ---- integer summary and page classes ------------------------------------------------------------------
     if (a.info && blockIdx.x == 0 && tid == 0) {
-        const int lead = u_open < nu ? ustart[u_open] : n_hist;      // retained rows before the first dropped slot
+        // retained rows before the first dropped slot: the units before the first shortened one, plus its kept prefix
+        const int lead = u_open < nu ? ustart[u_open] + (prefix[u_open + 1] - prefix[u_open]) : n_hist;
         a.info->n_kept = n_kept;
         a.info->span_pages = (n_kept + a.page_size - 1) / a.page_size;
         a.info->rows_moved = n_kept - min(lead, n_kept);
@@ -863,7 +870,8 @@ extern "C" omni_status omnipage_compact(omnitide_ctx* ctx, void* stream, const v
 extern "C" omni_status omnipage_compact_units(omnitide_ctx* ctx, void* stream, const void* k_src, const void* v_src,
                                               void* k_dst, void* v_dst, const omni_unit* units,
                                               const int32_t* n_units_dev, int32_t n_units_max, const uint8_t* unit_keep,
-                                              int32_t s_span_max, int32_t page_size, const omni_unit* units_kept,
+                                              const int32_t* unit_kept_len, int32_t s_span_max, int32_t page_size,
+                                              const omni_unit* units_kept,
                                               const int32_t* n_units_kept_dev, int32_t* slot_map_out,
                                               omni_compact_info* info_out, uint8_t* page_class_out) {
     if (!ctx) return OMNI_ERR_INVALID_ARG;
@@ -891,6 +899,7 @@ extern "C" omni_status omnipage_compact_units(omnitide_ctx* ctx, void* stream, c
     a.k_src = static_cast<const char*>(k_src); a.v_src = static_cast<const char*>(v_src);
     a.k_dst = static_cast<char*>(kd); a.v_dst = static_cast<char*>(vd);
     a.units = units; a.n_units_dev = n_units_dev; a.n_units_max = n_units_max; a.unit_keep = unit_keep;
+    a.unit_kept_len = unit_kept_len;
     a.s_span_max = s_span_max; a.page_size = page_size; a.row_bytes = (int)ctx->row_bytes;
     a.vpr = (int)(ctx->row_bytes >> 4); a.vpr_shift = -1;
     for (int sft = 0; sft < 20; ++sft) if ((1 << sft) == a.vpr) a.vpr_shift = sft;
@@ -927,7 +936,8 @@ extern "C" omni_status omnipage_compact_units(omnitide_ctx* ctx, void* stream, c
 extern "C" omni_status omnipage_compact_units_batched(omnitide_ctx* ctx, void* stream, const void* const* k_src,
                                                       const void* const* v_src, void* const* k_dst, void* const* v_dst,
                                                       int32_t n_layers, const omni_unit* units, const int32_t* n_units_dev,
-                                                      int32_t n_units_max, const uint8_t* unit_keep, int32_t s_span_max,
+                                                      int32_t n_units_max, const uint8_t* unit_keep,
+                                                      const int32_t* unit_kept_len, int32_t s_span_max,
                                                       int32_t page_size, const omni_unit* units_kept,
                                                       const int32_t* n_units_kept_dev, int32_t* slot_map_out,
                                                       omni_compact_info* info_out, uint8_t* page_class_out) {
@@ -945,6 +955,7 @@ extern "C" omni_status omnipage_compact_units_batched(omnitide_ctx* ctx, void* s
     CompactUnitsArgs a;
     a.k_src = a.v_src = nullptr; a.k_dst = a.v_dst = nullptr;
     a.units = units; a.n_units_dev = n_units_dev; a.n_units_max = n_units_max; a.unit_keep = unit_keep;
+    a.unit_kept_len = unit_kept_len;
     a.s_span_max = s_span_max; a.page_size = page_size; a.row_bytes = (int)ctx->row_bytes;
     a.vpr = (int)(ctx->row_bytes >> 4); a.vpr_shift = -1;
     a.units_kept = units_kept; a.n_units_kept_dev = n_units_kept_dev;

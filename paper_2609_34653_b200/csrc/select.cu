@@ -245,6 +245,206 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) select_units_kernel(const Sele
     }
 }
 
+// ---------------------------------------------------------------------------------------------------
+// Structure-aware, score-free retention planning (Section 5.1): metadata only.  One CTA: the per-span rules
+// run in parallel (the text budget is a prefix sum in time order), the event walk of the drop phase is
+// sequential by definition and runs on one thread over the event runs of the table.
+struct PlanArgs {
+    const omni_unit* units; const int32_t* n_units_dev; int n_units_max;
+    omni_structural_params p;
+    uint8_t* unit_keep; int32_t* unit_kept_len; uint8_t* keep_mask; int n_hist_max;
+    int32_t* n_kept_out; omni_unit* units_out; int32_t* n_units_out; int32_t* status;
+};
+
+__global__ void __launch_bounds__(SEL_THREADS, 1) plan_structural_kernel(const PlanArgs a) {
+    extern __shared__ int sm_plan[];
+    const int cap = a.n_units_max;
+    int* s_start = sm_plan;                 // [cap + 1]
+    int* s_len = s_start + cap + 1;         // [cap]
+    int* s_meta = s_len + cap;              // [cap]  modality | must << 8 | boundary << 9 | recent << 10
+    int* s_event = s_meta + cap;            // [cap]
+    int* s_kept = s_event + cap;            // [cap]  kept tokens per span
+    int* s_scan = s_kept + cap;             // [cap + 1] scan scratch (text prefix sums, new starts)
+    int* s_idx = s_scan + cap + 1;          // [cap + 1] kept spans before a span
+    int* s_drop = s_idx + cap + 1;          // [cap]  1: the span's event is dropped in the last phase
+    __shared__ int red[33];
+    __shared__ int s_thr_event, s_all_recent, s_bad;
+    const int tid = threadIdx.x;
+
+    int U = a.n_units_dev ? *a.n_units_dev : a.n_units_max;
+    if (U < 0 || U > a.n_units_max) {
+        if (tid == 0) atomicOr(a.status, OMNI_DEV_BAD_COUNT);
+        U = max(0, min(U, a.n_units_max));
+    }
+    if (tid == 0) { s_bad = 0; s_all_recent = 0; s_thr_event = 0; }
+    __syncthreads();
+    for (int u = tid; u < U; u += SEL_THREADS) {
+        const omni_unit un = a.units[u];
+        s_start[u] = un.start; s_len[u] = un.len; s_event[u] = un.event;
+        s_meta[u] = (un.modality & 0xff) | ((un.group == OMNI_GROUP_MUST_KEEP) << 8) | ((un.flags & OMNI_FLAG_BOUNDARY) ? (1 << 9) : 0);
+        s_drop[u] = 0;
+        bool bad = un.len <= 0 || un.modality < 0 || un.modality > 2;
+        if (u == 0) bad |= un.start != 0;
+        if (u + 1 < U) {
+            const omni_unit nx = a.units[u + 1];
+            bad |= (nx.start != un.start + un.len) || (nx.event < un.event);
+        }
+        if (bad) s_bad = 1;
+    }
+    __syncthreads();
+    const int n_hist = U ? s_start[U - 1] + s_len[U - 1] : 0;
+    if (s_bad || n_hist > a.n_hist_max) {
+        if (tid == 0) {
+            atomicOr(a.status, s_bad ? OMNI_DEV_BAD_UNITS : OMNI_DEV_BAD_COUNT);
+            *a.n_kept_out = 0; *a.n_units_out = 0;
+        }
+        return;
+    }
+    if (tid == 0) {
+        s_start[U] = n_hist;
+        // the oldest of the newest R events
+        const int R = a.p.n_recent_events;
+        if (R <= 0 || U == 0) {
+            s_all_recent = -1;
+        } else {
+            int distinct = 1, u = U - 1, ev = s_event[U - 1];
+            while (u > 0) {
+                const int e2 = s_event[u - 1];
+                if (e2 != ev) {
+                    if (distinct == R) break;
+                    ++distinct;
+                    ev = e2;
+                }
+                --u;
+            }
+            s_thr_event = ev;
+        }
+    }
+    __syncthreads();
+    const bool any_recent = s_all_recent == 0;
+    const int thr = s_thr_event;
+    const bool round = n_hist > a.p.high_watermark;          // retention starts above the high watermark only
+
+    // ---- per-span rules -----------------------------------------------------------------------------
+    for (int u = tid; u < U; u += SEL_THREADS) {
+        const int meta = s_meta[u], mod = meta & 0xff, ln = s_len[u];
+        const bool recent = any_recent && s_event[u] >= thr;
+        if (recent) s_meta[u] = meta | (1 << 10);
+        const bool whole = !round || (meta & (1 << 8)) || recent || (meta & (1 << 9));
+        int kept = ln, text = 0;
+        if (!whole) {
+            if (mod == OMNI_MOD_TEXT) text = ln;             // decided by the shared budget below
+            else kept = min(ln, max(0, mod == OMNI_MOD_VIDEO ? a.p.sink_prefix[0] : a.p.sink_prefix[1]));
+        }
+        s_kept[u] = kept;
+        s_scan[u] = text;
+    }
+    __syncthreads();
+    if (round) {
+        // older text spans, oldest first, while the running total fits the budget: the first misfit ends it
+        block_excl_scan(s_scan, U, red);
+        for (int u = tid; u < U; u += SEL_THREADS) {
+            const int meta = s_meta[u];
+            const bool older_text = !(meta & ((1 << 8) | (1 << 9) | (1 << 10))) && (meta & 0xff) == OMNI_MOD_TEXT;
+            if (older_text && s_scan[u] + s_len[u] > a.p.text_budget) s_kept[u] = 0;
+        }
+        __syncthreads();
+    }
+    int my = 0;
+    for (int u = tid; u < U; u += SEL_THREADS) my += s_kept[u];
+    const int total0 = block_sum(my, red);
+
+    // ---- drop whole events, oldest first, partially retained ones before complete ones ------------------
+    if (round && total0 > a.p.low_watermark && tid == 0) {
+        int total = total0, n_alive = 0;
+        // pass 1: classify the event runs (s_scan[first span of the run] = kept tokens outside the prefix,
+        // s_idx[first span] = 1 if partially retained)
+        for (int u0 = 0; u0 < U;) {
+            int u1 = u0, ev_kept = 0, partial = 0;
+            while (u1 < U && s_event[u1] == s_event[u0]) {
+                if (!(s_meta[u1] & (1 << 8))) { ev_kept += s_kept[u1]; partial |= s_kept[u1] < s_len[u1]; }
+                ++u1;
+            }
+            s_scan[u0] = ev_kept;
+            s_idx[u0] = partial;
+            n_alive += ev_kept > 0;
+            u0 = u1;
+        }
+        for (int cls = 1; cls >= 0; --cls) {
+            for (int u0 = 0; u0 < U;) {
+                int u1 = u0;
+                while (u1 < U && s_event[u1] == s_event[u0]) ++u1;
+                if (s_scan[u0] > 0 && s_idx[u0] == cls) {
+                    if (total <= a.p.low_watermark || n_alive <= 1) { cls = -1; break; }
+                    total -= s_scan[u0];
+                    --n_alive;
+                    for (int u = u0; u < u1; ++u) s_drop[u] = 1;
+                }
+                u0 = u1;
+            }
+        }
+    }
+    __syncthreads();
+
+    // ---- codes, re-indexed survivors ---------------------------------------------------------------------
+    for (int u = tid; u < U; u += SEL_THREADS) {
+        if (s_drop[u] && !(s_meta[u] & (1 << 8))) s_kept[u] = 0;
+        s_scan[u] = s_kept[u];
+        s_idx[u] = s_kept[u] > 0;
+    }
+    __syncthreads();
+    const int n_kept = block_excl_scan(s_scan, U, red);       // s_scan[u] = kept tokens before span u
+    const int n_units_kept = block_excl_scan(s_idx, U, red);  // s_idx[u] = kept spans before span u
+    for (int u = tid; u < U; u += SEL_THREADS) {
+        const int kept = s_kept[u], ln = s_len[u], meta = s_meta[u];
+        a.unit_keep[u] = kept == 0 ? OMNI_KEEP_DROPPED : (kept == ln ? OMNI_KEEP_WHOLE : OMNI_KEEP_SINK_PREFIX);
+        if (a.unit_kept_len) a.unit_kept_len[u] = kept;
+        if (kept > 0) {
+            omni_unit un = a.units[u];
+            un.group = (meta & (1 << 8)) ? OMNI_GROUP_MUST_KEEP : ((meta & (1 << 10)) ? OMNI_GROUP_RECENT : OMNI_GROUP_SELECTED);
+            un.start = s_scan[u];
+            un.len = kept;
+            a.units_out[s_idx[u]] = un;
+        }
+    }
+    if (tid == 0) { *a.n_kept_out = n_kept; *a.n_units_out = n_units_kept; }
+
+    // ---- per-token keep mask: the first kept tokens of every span ----------------------------------------
+    if (a.keep_mask) {
+        const int n_vec = (n_hist + 15) >> 4;
+        for (int vi = tid; vi < n_vec; vi += SEL_THREADS) {
+            const int pos = vi << 4;
+            int lo = 0, hi = U;                   // largest u with s_start[u] <= pos
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (s_start[mid] <= pos) lo = mid; else hi = mid;
+            }
+            int u = lo;
+            uint32_t w0 = 0, w1 = 0, w2 = 0, w3 = 0;
+#pragma unroll
+            for (int b = 0; b < 16; ++b) {
+                const int p = pos + b;
+                if (p < n_hist) {
+                    while (p >= s_start[u + 1]) ++u;
+                    if (p - s_start[u] < s_kept[u]) {
+                        const uint32_t bit = 1u << ((b & 3) * 8);
+                        if (b < 4) w0 |= bit; else if (b < 8) w1 |= bit; else if (b < 12) w2 |= bit; else w3 |= bit;
+                    }
+                }
+            }
+            if (pos + 16 <= a.n_hist_max) {
+                *reinterpret_cast<uint4*>(a.keep_mask + pos) = make_uint4(w0, w1, w2, w3);
+            } else {
+#pragma unroll
+                for (int b = 0; b < 16; ++b) {
+                    const uint32_t w = b < 4 ? w0 : (b < 8 ? w1 : (b < 12 ? w2 : w3));
+                    if (pos + b < n_hist) a.keep_mask[pos + b] = (w >> ((b & 3) * 8)) & 0xff;
+                }
+            }
+        }
+    }
+}
+
 }  // namespace
 
 extern "C" omni_status omnitide_select_units(omnitide_ctx* ctx, void* stream, const omni_unit* units,
@@ -271,5 +471,30 @@ extern "C" omni_status omnitide_select_units(omnitide_ctx* ctx, void* stream, co
         OMNI_CUDA(ctx, cudaFuncSetAttribute(select_units_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     select_units_kernel<<<1, SEL_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(a);
     OMNI_CHECK_LAUNCH(ctx, "select_units_kernel");
+    return OMNI_OK;
+}
+
+extern "C" omni_status omnitide_plan_structural(omnitide_ctx* ctx, void* stream, const omni_unit* units,
+                                                const int32_t* n_units_dev, int32_t n_units_max,
+                                                const omni_structural_params* params, uint8_t* unit_keep_out,
+                                                int32_t* unit_kept_len_out, uint8_t* keep_mask_out, int32_t n_hist_max,
+                                                int32_t* n_kept_out, omni_unit* units_out, int32_t* n_units_out) {
+    if (!ctx) return OMNI_ERR_INVALID_ARG;
+    if (!units || !params || !unit_keep_out || !n_kept_out || !units_out || !n_units_out)
+        OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "plan_structural: null pointer");
+    if (n_units_max <= 0 || n_units_max > ctx->g.u_cap) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "plan_structural: n_units_max %d outside (0, u_cap]", n_units_max);
+    if (n_units_max > SEL_MAX_UNITS) OMNI_FAIL(ctx, OMNI_ERR_UNSUPPORTED, "plan_structural: more than %d units", SEL_MAX_UNITS);
+    if (n_hist_max < 0 || n_hist_max > ctx->g.s_cap) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "plan_structural: n_hist_max outside [0, s_cap]");
+    if (keep_mask_out && !omni_aligned16(keep_mask_out)) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "plan_structural: keep_mask_out must be 16-byte aligned");
+    if (units == units_out) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "plan_structural: units_out must not alias units");
+    PlanArgs a;
+    a.units = units; a.n_units_dev = n_units_dev; a.n_units_max = n_units_max; a.p = *params;
+    a.unit_keep = unit_keep_out; a.unit_kept_len = unit_kept_len_out; a.keep_mask = keep_mask_out; a.n_hist_max = n_hist_max;
+    a.n_kept_out = n_kept_out; a.units_out = units_out; a.n_units_out = n_units_out; a.status = ctx->status_dev;
+    const size_t smem = ((size_t)8 * n_units_max + 4) * sizeof(int);
+    if (smem > 48 * 1024)
+        OMNI_CUDA(ctx, cudaFuncSetAttribute(plan_structural_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    plan_structural_kernel<<<1, SEL_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(a);
+    OMNI_CHECK_LAUNCH(ctx, "plan_structural_kernel");
     return OMNI_OK;
 }

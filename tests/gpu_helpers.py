@@ -100,7 +100,7 @@ def bytes_of(t):
 
 
 def gpu_compact_units(ctx, k, v, units_np, unit_keep_np, page, units_out_np=None, in_place=False, s_span_max=None,
-                      u_max=None, want_slot_map=True):
+                      u_max=None, want_slot_map=True, kept_len_np=None):
     """omnipage_compact_units on a history unit table and one keep code per unit."""
     U = len(units_np)
     S = int(units_np[:, 1].sum()) if U else 0
@@ -120,10 +120,34 @@ def gpu_compact_units(ctx, k, v, units_np, unit_keep_np, page, units_out_np=None
     if units_out_np is not None and len(units_out_np):
         dk = ob.units_to_device(units_out_np, umax)
         nk = i32(len(units_out_np))
-    ctx.compact_units(k, v, kd, vd, du, i32(U), umax, keep, smax, page, dk, nk, slot_map, info, page_class)
+    klen = None
+    if kept_len_np is not None:
+        klen = torch.full((umax + 16,), 10 ** 6, dtype=torch.int32, device="cuda")      # stale entries beyond n_units are ignored
+        klen[:U] = torch.from_numpy(np.asarray(kept_len_np, dtype=np.int32)).cuda()
+    ctx.compact_units(k, v, kd, vd, du, i32(U), umax, keep, smax, page, dk, nk, slot_map, info, page_class, unit_kept_len=klen)
     torch.cuda.synchronize()
     status = ctx.poll_status()
     out = ob.info_to_dict(info)
     out.update(k=kd, v=vd, slot_map=slot_map[:S].cpu().numpy() if want_slot_map else None,
                page_class=page_class[:n_pages].cpu().numpy(), status=status)
     return out
+
+
+def gpu_plan_structural(ctx, units_np, H_, L_, R, sink, Tb, want_mask=True, use_dev_count=True):
+    U = len(units_np)
+    n = int(units_np[:, 1].sum())
+    du = ob.units_to_device(units_np, U + 3)
+    unit_keep = torch.full((U + 19,), 9, dtype=torch.uint8, device="cuda")
+    kept_len = torch.full((U + 19,), -9, dtype=torch.int32, device="cuda")
+    keep_mask = torch.full((n + 32,), 9, dtype=torch.uint8, device="cuda") if want_mask else None
+    n_kept, n_units_out = i32(-1), i32(-1)
+    units_out = torch.zeros((U + 3, 6), dtype=torch.int32, device="cuda")
+    ctx.plan_structural(du, i32(U) if use_dev_count else None, U if not use_dev_count else U + 3,
+                        ob.structural_params(H_, L_, R, sink, Tb), unit_keep, kept_len, keep_mask, n, n_kept, units_out,
+                        n_units_out)
+    torch.cuda.synchronize()
+    nu = int(n_units_out.item())
+    return dict(unit_keep=unit_keep[:U].cpu().numpy(), unit_kept_len=kept_len[:U].cpu().numpy(),
+                keep_mask=keep_mask[:n].cpu().numpy() if want_mask else None, n_kept=int(n_kept.item()),
+                units_out=units_out[:max(nu, 0)].cpu().numpy(), status=ctx.poll_status(),
+                unit_keep_dev=unit_keep, kept_len_dev=kept_len, units_out_dev=units_out, n_units_out_dev=n_units_out)

@@ -44,6 +44,7 @@ def test_struct_layouts_match_the_header():
     from paper_2609_34653_b200 import binding
     assert ctypes.sizeof(binding.Geometry) == 28
     assert ctypes.sizeof(binding.SelectParams) == 20
+    assert ctypes.sizeof(binding.StructuralParams) == 28
     assert ctypes.sizeof(binding.CompactInfo) == 32
 
 

@@ -499,3 +499,58 @@ def test_budget_covers_history_is_full_attention(H, ob):
     assert res["info"]["rows_moved"] == 0 and res["info"]["n_kept"] == w.n_hist
     o_ref, _ = oc.chunk_attention(w.q, w.k_hist, w.v_hist, w.k_chunk, w.v_chunk)
     _check_attention(res["o"], None, o_ref, None)
+
+
+# ------------------------------------------------------- structural (score-free) retention plan
+def test_plan_structural_exact(H, ob):
+    """omnitide_plan_structural equals the oracle's plan on random streams: codes, kept lengths, mask, table."""
+    from tests.test_oracle_pins import _random_stream, _toy_stream
+    rng = np.random.default_rng(616)
+    ctx = ob.Context(4, 1, 64, "fp32", 4096, 64, 16)
+    cases = [(_toy_stream(), 40, 45, 2, (2, 1, 0), 4), (_toy_stream(), 40, 30, 2, (2, 1, 0), 4),
+             (_toy_stream(), 74, 10, 1, (0, 0, 0), 0), (_toy_stream(), 40, 5, 2, (2, 1, 0), 4)]
+    for _ in range(120):
+        u = _random_stream(rng, int(rng.integers(1, 10)), with_prefix=rng.random() < 0.8)
+        n = int(u[:, 1].sum())
+        Hw = int(rng.integers(0, n + 10))
+        cases.append((u, Hw, int(rng.integers(0, Hw + 1)), int(rng.integers(0, 4)),
+                      (int(rng.integers(0, 12)), int(rng.integers(0, 12)), 0), int(rng.integers(0, 60))))
+    for i, (u, Hw, Lw, R, sink, Tb) in enumerate(cases):
+        exp = oc.plan_structural(u, Hw, Lw, R, sink, Tb)
+        got = H.gpu_plan_structural(ctx, u, Hw, Lw, R, sink, Tb, use_dev_count=(i % 2 == 0))
+        assert got["status"] == 0
+        assert np.array_equal(got["unit_keep"], exp["unit_keep"]), i
+        assert np.array_equal(got["unit_kept_len"], exp["unit_kept_len"]), i
+        assert np.array_equal(got["keep_mask"], exp["keep_mask"]), i
+        assert got["n_kept"] == exp["n_kept"] and np.array_equal(got["units_out"], exp["units_out"]), i
+    # a malformed table is flagged and yields an empty plan
+    bad = _toy_stream()
+    bad[3, 0] += 1
+    got = H.gpu_plan_structural(ctx, bad, 0, 0, 1, (1, 1, 0), 0)
+    assert got["status"] & 2 and got["n_kept"] == 0
+    ctx.close()
+
+
+def test_structural_plan_then_compaction_bit_exact(H, ob):
+    """The plan's sink prefixes through the unit-granular compaction equal the oracle's pack of the plan's mask."""
+    rng = np.random.default_rng(717)
+    w = wl.layer_8b(n_hist=6000, budget=2000)
+    u = w.units
+    n = w.n_hist
+    exp_plan = oc.plan_structural(u, 3000, 2500, 2, (24, 8, 0), 64)
+    assert (exp_plan["unit_keep"] == 1).any(), "the case must contain sink prefixes"
+    ctx = H.make_ctx(w)
+    plan = H.gpu_plan_structural(ctx, u, 3000, 2500, 2, (24, 8, 0), 64)
+    assert np.array_equal(plan["unit_kept_len"], exp_plan["unit_kept_len"])
+    k, v = ob.to_device(w.k_hist, w.dtype), ob.to_device(w.v_hist, w.dtype)
+    raw_k, raw_v = H.bytes_of(k).reshape(n, -1), H.bytes_of(v).reshape(n, -1)
+    exp = oc.compact_pack(raw_k, raw_v, exp_plan["keep_mask"], w.page_size, exp_plan["units_out"])
+    got = H.gpu_compact_units(ctx, k, v, u, plan["unit_keep"], w.page_size, units_out_np=plan["units_out"],
+                              kept_len_np=plan["unit_kept_len"])
+    m = exp["n_kept"]
+    assert (got["n_kept"], got["span_pages"], got["rows_moved"]) == (m, exp["span_pages"], exp["rows_moved"])
+    assert got["part_begin"] == exp["part_begin"].tolist()
+    assert np.array_equal(got["slot_map"], exp["slot_map"])
+    assert np.array_equal(H.bytes_of(got["k"][:m]).reshape(m, -1), exp["k"])
+    assert np.array_equal(H.bytes_of(got["v"][:m]).reshape(m, -1), exp["v"])
+    ctx.close()
