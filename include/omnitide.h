@@ -296,6 +296,22 @@ omni_status omnitide_chunk_step(omnitide_ctx* ctx, void* stream,
                                 void* o_out, int32_t out_dtype, omni_compact_info* info_out);
 
 /*
+ * The pass as the paper runs it (no scoring): omnitide_plan_structural -> omnipage_compact_units with the planned
+ * prefix lengths -> omnitide_chunk_attention -> omnipage_append.  Arguments as omnitide_chunk_step, with the
+ * structural parameters in place of the modality weights and the selection parameters.
+ */
+omni_status omnitide_chunk_step_structural(omnitide_ctx* ctx, void* stream,
+                                           const void* q, const void* k_chunk, const void* v_chunk, int32_t t,
+                                           const omni_unit* chunk_units, int32_t n_chunk_units,
+                                           const void* k_cache, const void* v_cache,
+                                           const int32_t* n_hist_dev, int32_t n_hist_max,
+                                           const omni_unit* units, const int32_t* n_units_dev, int32_t n_units_max,
+                                           const omni_structural_params* params /*[host]*/, int32_t page_size, float scale,
+                                           void* k_cache_out, void* v_cache_out, omni_unit* units_out,
+                                           int32_t* n_hist_out, int32_t* n_units_out,
+                                           void* o_out, int32_t out_dtype, omni_compact_info* info_out);
+
+/*
  * The same pass for a caller whose chunk lives in host memory: q/k_chunk/v_chunk/chunk_units are
  * HOST pointers (pinned memory recommended) copied to context staging buffers on `stream`, and the
  * attention output is copied back to o_host (out_dtype elements).  The call returns after the

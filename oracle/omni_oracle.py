@@ -428,3 +428,17 @@ def stream_step(q, k_cache, v_cache, units, k_chunk, v_chunk, chunk_units, w_mod
     v_new = np.concatenate([cp["v"], np.asarray(v_chunk)], axis=0)
     return dict(score=score, mass=mass, select=sel, compact=cp, o=o, lse=lse,
                 units=units_new, k_cache=k_new, v_cache=v_new)
+
+
+def stream_step_structural(q, k_cache, v_cache, units, k_chunk, v_chunk, chunk_units, high_watermark, low_watermark,
+                           n_recent_events, sink_prefix, text_budget, page_size, scale=None):
+    """The pass as the paper runs it: plan from metadata -> compact -> append -> attend (no scoring)."""
+    units = np.asarray(units)
+    n_hist = int(units[:, U_LEN].sum())
+    plan = plan_structural(units, high_watermark, low_watermark, n_recent_events, sink_prefix, text_budget)
+    cp = compact_pack(k_cache[:n_hist], v_cache[:n_hist], plan["keep_mask"], page_size, plan["units_out"])
+    o, lse = chunk_attention(q, cp["k"], cp["v"], k_chunk, v_chunk, scale)
+    units_new = append_chunk(plan["units_out"], cp["n_kept"], chunk_units)
+    k_new = np.concatenate([cp["k"], np.asarray(k_chunk)], axis=0)
+    v_new = np.concatenate([cp["v"], np.asarray(v_chunk)], axis=0)
+    return dict(plan=plan, compact=cp, o=o, lse=lse, units=units_new, k_cache=k_new, v_cache=v_new)

@@ -43,7 +43,7 @@ class CompactInfo(C.Structure):
 EXPORTS = [
     "omnitide_create", "omnitide_destroy", "omnitide_poll_status", "omnitide_last_error",
     "omnitide_score_units", "omnitide_select_units", "omnitide_plan_structural", "omnipage_compact", "omnipage_compact_units", "omnipage_compact_units_batched", "omnipage_append",
-    "omnitide_chunk_attention", "omnitide_chunk_step", "omnitide_chunk_step_host",
+    "omnitide_chunk_attention", "omnitide_chunk_step", "omnitide_chunk_step_host", "omnitide_chunk_step_structural",
     "omnitide_set_option", "omnitide_launch_count", "omnitide_score_units_noalloc",
 ]
 NOALLOC_MAX_UNITS = 1024
@@ -78,6 +78,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     step = [vp, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp, i32, vp, vp, i32, C.POINTER(f32),
             C.POINTER(SelectParams), i32, f32, vp, vp, vp, vp, vp, vp, i32, vp]
     lib.omnitide_chunk_step.argtypes = step
+    lib.omnitide_chunk_step_structural.argtypes = [vp, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp, i32, vp, vp, i32,
+                                                   C.POINTER(StructuralParams), i32, f32, vp, vp, vp, vp, vp, vp, i32, vp]
     lib.omnitide_chunk_step_host.argtypes = step
     for name in EXPORTS:
         fn = getattr(lib, name)
@@ -239,6 +241,16 @@ class Context:
                        n_units_max, w, C.byref(params), page_size, float(scale), _ptr(k_cache_out), _ptr(v_cache_out),
                        _ptr(units_out), _ptr(n_hist_out), _ptr(n_units_out), hp(o_out), out_dtype, _ptr(info_out)),
                     name)
+
+    def chunk_step_structural(self, q, k_chunk, v_chunk, t, chunk_units, n_chunk_units, k_cache, v_cache, n_hist_dev,
+                              n_hist_max, units, n_units_dev, n_units_max, params, page_size, scale, k_cache_out,
+                              v_cache_out, units_out, n_hist_out, n_units_out, o_out, out_dtype, info_out=None):
+        self._check(self.lib.omnitide_chunk_step_structural(
+            self._ctx, _stream(), _ptr(q), _ptr(k_chunk), _ptr(v_chunk), t, _ptr(chunk_units), n_chunk_units,
+            _ptr(k_cache), _ptr(v_cache), _ptr(n_hist_dev), n_hist_max, _ptr(units), _ptr(n_units_dev), n_units_max,
+            C.byref(params), page_size, float(scale), _ptr(k_cache_out), _ptr(v_cache_out), _ptr(units_out),
+            _ptr(n_hist_out), _ptr(n_units_out), _ptr(o_out), out_dtype, _ptr(info_out)),
+            "omnitide_chunk_step_structural")
 
     def chunk_step(self, *a, info_out=None):
         self._step(self.lib.omnitide_chunk_step, "omnitide_chunk_step", _ptr, *a, info_out)

@@ -17,7 +17,7 @@ cudaError_t alloc(T** p, size_t n) {
 
 void free_all(omnitide_ctx* c) {
     void* ptrs[] = {c->status_dev, c->score_part, c->score_tile_mass, c->score_mass64, c->inplace_k, c->inplace_v,
-                    c->ws_scores, c->ws_unit_keep, c->ws_keep_mask, c->ws_slot_map, c->ws_counts, c->ws_info, c->st_q,
+                    c->ws_scores, c->ws_unit_keep, c->ws_kept_len, c->ws_keep_mask, c->ws_slot_map, c->ws_counts, c->ws_info, c->st_q,
                     c->st_k, c->st_v, c->st_o, c->st_units, c->attn_part_o, c->attn_part_ml, c->cp_words};
     for (void* p : ptrs)
         if (p) cudaFree(p);
@@ -62,6 +62,7 @@ extern "C" omni_status omnitide_create(omnitide_ctx** ctx_out, const omni_geomet
     ok = ok && cudaMemset(c->cp_words, 0, ((size_t)c->sm_count + 1) * sizeof(unsigned long long)) == cudaSuccess;
     ok &= alloc(&c->ws_scores, (size_t)g->u_cap) == cudaSuccess;
     ok &= alloc(&c->ws_unit_keep, (size_t)g->u_cap + 16) == cudaSuccess;
+    ok &= alloc(&c->ws_kept_len, (size_t)g->u_cap) == cudaSuccess;
     ok &= alloc(&c->ws_keep_mask, (size_t)g->s_cap + 16) == cudaSuccess;
     ok &= alloc(&c->ws_slot_map, (size_t)g->s_cap + 16) == cudaSuccess;
     ok &= alloc(&c->ws_counts, 4) == cudaSuccess;
@@ -210,6 +211,38 @@ extern "C" omni_status omnitide_chunk_step(omnitide_ctx* ctx, void* stream, cons
     return chunk_step_impl(nullptr, ctx, stream, q, k_chunk, v_chunk, t, chunk_units, n_chunk_units, k_cache, v_cache,
                            n_hist_dev, n_hist_max, units, n_units_dev, n_units_max, w_modality, params, page_size, scale,
                            k_cache_out, v_cache_out, units_out, n_hist_out, n_units_out, o_out, out_dtype, info_out);
+}
+
+extern "C" omni_status omnitide_chunk_step_structural(omnitide_ctx* ctx, void* stream, const void* q, const void* k_chunk,
+                                                      const void* v_chunk, int32_t t, const omni_unit* chunk_units,
+                                                      int32_t n_chunk_units, const void* k_cache, const void* v_cache,
+                                                      const int32_t* n_hist_dev, int32_t n_hist_max, const omni_unit* units,
+                                                      const int32_t* n_units_dev, int32_t n_units_max,
+                                                      const omni_structural_params* params, int32_t page_size, float scale,
+                                                      void* k_cache_out, void* v_cache_out, omni_unit* units_out,
+                                                      int32_t* n_hist_out, int32_t* n_units_out, void* o_out,
+                                                      int32_t out_dtype, omni_compact_info* info_out) {
+    if (!ctx) return OMNI_ERR_INVALID_ARG;
+    if (!k_cache_out || !v_cache_out || k_cache_out == k_cache || v_cache_out == v_cache)
+        OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "chunk_step_structural: output caches must be distinct buffers");
+    if (!units_out || !n_hist_out || !n_units_out || !params)
+        OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "chunk_step_structural: null pointer");
+    int32_t* n_kept = ctx->ws_counts;
+    int32_t* n_units_kept = ctx->ws_counts + 1;
+    omni_compact_info* info = info_out ? info_out : ctx->ws_info;
+    // plan from metadata alone (no scoring pass), pack the planned runs, attend, append
+    omni_status s = omnitide_plan_structural(ctx, stream, units, n_units_dev, n_units_max, params, ctx->ws_unit_keep,
+                                             ctx->ws_kept_len, nullptr, n_hist_max, n_kept, units_out, n_units_kept);
+    if (s) return s;
+    s = omnipage_compact_units(ctx, stream, k_cache, v_cache, k_cache_out, v_cache_out, units, n_units_dev, n_units_max,
+                               ctx->ws_unit_keep, ctx->ws_kept_len, n_hist_max, page_size, units_out, n_units_kept, nullptr,
+                               info, nullptr);
+    if (s) return s;
+    s = omnitide_chunk_attention(ctx, stream, q, t, k_cache_out, v_cache_out, n_kept, n_hist_max, k_chunk, v_chunk, scale,
+                                 o_out, out_dtype, nullptr);
+    if (s) return s;
+    return omnipage_append(ctx, stream, k_cache_out, v_cache_out, n_kept, k_chunk, v_chunk, t, units_out, n_units_kept,
+                           chunk_units, n_chunk_units, n_hist_out, n_units_out);
 }
 
 extern "C" omni_status omnitide_chunk_step_host(omnitide_ctx* ctx, void* stream, const void* q_host,

@@ -30,6 +30,7 @@ struct omnitide_ctx {
     // work buffers of omnitide_chunk_step
     float* ws_scores;             // [u_cap]
     uint8_t* ws_unit_keep;        // [u_cap]
+    int32_t* ws_kept_len;         // [u_cap] tokens kept at the start of every unit (structural plan)
     uint8_t* ws_keep_mask;        // [s_cap]
     int32_t* ws_slot_map;         // [s_cap]
     int32_t* ws_counts;           // {n_kept, n_units_kept}

@@ -201,3 +201,64 @@ def test_stream_loop_short(H, ob, P):
         n_hist_a, n_hist_b, n_units_a, n_units_b = n_hist_b, n_hist_a, n_units_b, n_units_a
     assert evicted, "the schedule never exceeded the budget: the test did not exercise eviction"
     ctx.close()
+
+
+def test_stream_loop_structural_short(H, ob, P):
+    """The score-free pass (structural plan -> unit-granular compaction with sink prefixes -> attention -> append)
+    carried on the device over nine chunks of the config-4 schedule, with a text span added to every other chunk so
+    that the text budget matters; every step against the oracle advanced from the same state: unit table, counts
+    and cache bytes exactly, attention within tolerance."""
+    sched = wl.loop_schedule(n_chunks=9)
+    Hw, Lw, R, sink, Tb, page = 4000, 3000, 2, (48, 6, 0), 40, 64
+    h_q, h_kv, d = 32, 8, 128
+    s_cap, u_cap, t_cap = 12288, 96, 2432
+    ctx = ob.Context(h_q, h_kv, d, "bf16", s_cap, u_cap, t_cap)
+    rng = np.random.Generator(np.random.PCG64(4343))
+    draw = lambda shape: wl.round_to_bf16(rng.standard_normal(shape, dtype=np.float32))
+    units = wl.loop_prefix_units()
+    k_cache, v_cache = draw((16, h_kv, d)), draw((16, h_kv, d))
+    dev = lambda a: ob.to_device(a, "bf16")
+    k_a = torch.zeros((s_cap, h_kv, d), dtype=torch.bfloat16, device="cuda")
+    v_a = torch.zeros_like(k_a)
+    k_b, v_b = torch.full_like(k_a, float("nan")), torch.full_like(v_a, float("nan"))
+    k_a[:16], v_a[:16] = dev(k_cache), dev(v_cache)
+    units_a = ob.units_to_device(units, u_cap)
+    units_b = torch.zeros_like(units_a)
+    n_hist_a, n_units_a = H.i32(16), H.i32(len(units))
+    n_hist_b, n_units_b = H.i32(-1), H.i32(-1)
+    params = ob.structural_params(Hw, Lw, R, sink, Tb)
+    saw_sink = saw_drop = False
+    for c, cu in enumerate(sched):
+        if c % 2 == 1:                                       # a text query behind the audio of every other chunk
+            tx = wl.make_units([(int(rng.integers(16, 40)), wl.MOD_TEXT, c + 1)], group_of_first=None)
+            tx[0, 0] = int(cu[:, 1].sum())
+            cu = np.concatenate([cu, tx], axis=0)
+        T = int(cu[:, 1].sum())
+        n, U = len(k_cache), len(units)
+        q, k_chunk, v_chunk = draw((T, h_q, d)), draw((T, h_kv, d)), draw((T, h_kv, d))
+        o = torch.full((T, h_q, d), float("nan"), dtype=torch.float32, device="cuda")
+        info = torch.zeros((8,), dtype=torch.int32, device="cuda")
+        ctx.chunk_step_structural(dev(q), dev(k_chunk), dev(v_chunk), T, ob.units_to_device(cu), len(cu), k_a, v_a, n_hist_a, n,
+                                  units_a, n_units_a, U, params, page, 0.0, k_b, v_b, units_b, n_hist_b, n_units_b, o,
+                                  ob.DTYPE_FP32, info_out=info)
+        torch.cuda.synchronize()
+        assert ctx.poll_status() == 0
+        st = oc.stream_step_structural(q, k_cache, v_cache, units, k_chunk, v_chunk, cu, Hw, Lw, R, sink, Tb, page)
+        n_new = len(st["k_cache"])
+        assert int(n_hist_b.item()) == n_new and int(n_units_b.item()) == len(st["units"])
+        assert np.array_equal(units_b[:len(st["units"])].cpu().numpy(), st["units"])
+        got, cp = ob.info_to_dict(info), st["compact"]
+        assert (got["n_kept"], got["span_pages"], got["rows_moved"]) == (cp["n_kept"], cp["span_pages"], cp["rows_moved"])
+        assert got["part_begin"] == cp["part_begin"].tolist()
+        for gpu_c, ref_c in ((k_b, st["k_cache"]), (v_b, st["v_cache"])):
+            bits = H.bytes_of(gpu_c[:n_new]).reshape(n_new, -1).view(np.uint16).reshape(n_new, h_kv, d)
+            assert np.array_equal(bits, wl.bf16_bits(ref_c))
+        P._check_attention(o.cpu().numpy(), None, st["o"], None)
+        saw_sink |= bool((st["plan"]["unit_keep"] == 1).any())
+        saw_drop |= bool((st["plan"]["unit_keep"] == 0).any())
+        k_cache, v_cache, units = st["k_cache"], st["v_cache"], st["units"]
+        k_a, k_b, v_a, v_b = k_b, k_a, v_b, v_a
+        units_a, units_b = units_b, units_a
+        n_hist_a, n_hist_b, n_units_a, n_units_b = n_hist_b, n_hist_a, n_units_b, n_units_a
+    assert saw_sink and saw_drop, "the schedule must exercise sink prefixes and dropped spans"
+    ctx.close()
