@@ -137,7 +137,7 @@ def whole_job(per_replica_value, world):
     return per_replica_value * world
 
 
-def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=64):
+def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=64, structural=False):
     """The 36-layer stream loop (frames of {640, 1280, 2304} tokens plus 2 s of audio at 10-25 tok/s per
     chunk): per chunk and per layer one omnitide_chunk_step on a device-resident cache.  Returns the
     mean milliseconds per chunk over the chunks whose history already exceeds the budget (CUDA events
@@ -162,6 +162,9 @@ def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=6
                            n_units=[torch.tensor([1], dtype=torch.int32, device="cuda"), torch.zeros(1, dtype=torch.int32, device="cuda")],
                            info=torch.zeros(8, dtype=torch.int32, device="cuda")))
     params = ob.select_params(budget, 1, (-1, -1, -1))
+    # the paper's score-free plan: start above the budget, trim to 72 % of it (its 2500 / 1800 watermark ratio),
+    # two newest events whole, sink prefixes of 32 image and 8 audio tokens, 256 tokens of older text
+    sparams = ob.structural_params(budget, int(budget * 0.72), 2, (32, 8, 0), 256)
     w_mod = (1.0, 2.0, 2.0)
     hist_bound, units_bound = 16, 1
     o = torch.empty((t_cap, h_q, d), dtype=torch.float32, device="cuda")
@@ -179,9 +182,14 @@ def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=6
         e0.record()
         for l, L in enumerate(layers):
             q, kc, vc = ins[l]
-            ctx.chunk_step(q, kc, vc, T, cu_dev, len(cu), L["k"][a], L["v"][a], L["n_hist"][a], hist_bound, L["units"][a],
-                           L["n_units"][a], units_bound, w_mod, params, page, 0.0, L["k"][b], L["v"][b], L["units"][b],
-                           L["n_hist"][b], L["n_units"][b], o, ob.DTYPE_FP32, info_out=L["info"])
+            if structural:
+                ctx.chunk_step_structural(q, kc, vc, T, cu_dev, len(cu), L["k"][a], L["v"][a], L["n_hist"][a], hist_bound,
+                                          L["units"][a], L["n_units"][a], units_bound, sparams, page, 0.0, L["k"][b], L["v"][b],
+                                          L["units"][b], L["n_hist"][b], L["n_units"][b], o, ob.DTYPE_FP32, info_out=L["info"])
+            else:
+                ctx.chunk_step(q, kc, vc, T, cu_dev, len(cu), L["k"][a], L["v"][a], L["n_hist"][a], hist_bound, L["units"][a],
+                               L["n_units"][a], units_bound, w_mod, params, page, 0.0, L["k"][b], L["v"][b], L["units"][b],
+                               L["n_hist"][b], L["n_units"][b], o, ob.DTYPE_FP32, info_out=L["info"])
         e1.record()
         torch.cuda.synchronize()
         assert ctx.poll_status() == 0, "device status word not clean inside the stream loop"
@@ -193,7 +201,9 @@ def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=6
         units_bound = int(max(int(L["n_units"][b].item()) for L in layers))
     launches = ctx.launch_count()
     ctx.close()
-    steady = [r for r in rows if r["evicting"]] or rows[-max(1, len(rows) // 2):]
+    # steady state: every chunk from the first retention round on (with watermarks most chunks have no round)
+    first = next((i for i, r in enumerate(rows) if r["evicting"]), len(rows) // 2)
+    steady = rows[first:] or rows[-1:]
     return {"ms_per_chunk": float(np.mean([r["ms"] for r in steady])), "layers": n_layers, "chunks": len(rows),
             "chunks_timed": len(steady), "budget": budget, "page": page,
             "mean_chunk_tokens": float(np.mean([r["t"] for r in steady])),
@@ -201,8 +211,9 @@ def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=6
             "kept_rows_mean": float(np.mean([r["kept"] for r in steady])),
             "span_slots_mean": float(np.mean([r["span"] for r in steady])),
             "span_over_kept": float(np.mean([r["span"] / max(r["kept"], 1.0) for r in steady])),
-            "gpu_launches": int(launches),
-            "note": "36 layer steps per chunk timed with CUDA events; chunks counted once the history exceeds the budget"}
+            "retention_rounds": int(sum(1 for r in steady if r["evicting"])),
+            "gpu_launches": int(launches), "selection": "structural (score-free)" if structural else "scored",
+            "note": "36 layer steps per chunk timed with CUDA events; chunks counted from the first retention round on"}
 
 
 def run_reference(args, rank, world):
@@ -253,7 +264,7 @@ def main():
                     help="time omnipage_compact (token keep mask + slot map) instead of the unit-granular entry point")
     ap.add_argument("--batch-layers", type=int, default=36,
                     help="layers packed by one launch of the cross-layer batched compaction (0: skip it)")
-    ap.add_argument("--loop-chunks", type=int, default=24, help="chunks of the 36-layer stream loop (0: skip it)")
+    ap.add_argument("--loop-chunks", type=int, default=40, help="chunks of the 36-layer stream loop (0: skip it)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -513,6 +524,9 @@ def main():
         loop = run_stream_loop(ob, torch, args.loop_chunks, rank)
         loop["ms_per_chunk"] = max_over_ranks([loop["ms_per_chunk"]], world, "cuda")[0]
         line["stream_loop"] = loop
+        loop_s = run_stream_loop(ob, torch, args.loop_chunks, rank, structural=True)
+        loop_s["ms_per_chunk"] = max_over_ranks([loop_s["ms_per_chunk"]], world, "cuda")[0]
+        line["stream_loop_structural"] = loop_s
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import omni_oracle as oc
         import threadpoolctl
