@@ -38,6 +38,14 @@ What follows the paper and what does not
                        boundary span are parameters the paper leaves open;
                        pinned by a hand-worked example, an independent
                        token-level replay and invariants.
+* rope_reindex      -- the position shift the runtime applies to cached keys after
+                       logical deletion (Section 5.2): a kept token's position
+                       drops by the number of deleted tokens before it and its
+                       key is re-rotated by that amount.  The paper names RoPE
+                       only; the pairing (half-split), the base and the number
+                       of rotated dimensions are parameters.  Pinned against
+                       the complex-number definition of RoPE and by group
+                       properties (composition, inverse, norm).
 * score_units       -- the paper's OmniPick collects no attention scores at
                        run time; the statistic scored here is the one its
                        design study measures offline (attention weight from
@@ -405,6 +413,39 @@ def chunk_attention(q, k_hist, v_hist, k_chunk, v_chunk, scale=None, rows=None):
         o[:, h, :] = (p[:, :Nh] @ vh[:, g, :] + p[:, Nh:] @ vc[:, g, :]) / z
         lse[:, h] = (m + np.log(z))[:, 0]
     return o, lse
+
+
+# ---------------------------------------------------------------------------
+# R -- RoPE position re-index of moved keys
+# ---------------------------------------------------------------------------
+def rope_reindex(k_rows, delta, theta_base=10000.0, n_dims=None):
+    """Rotate key rows by a position shift (Section 5.2: "the runtime applies the corresponding RoPE
+    adjustment to cached keys").
+
+    k_rows [n, Hkv, D]; delta [n] integer position shifts (new position - old position).  Half-split
+    pairing: dimension i pairs with i + n_dims/2, i < n_dims/2, angle delta * theta_base**(-2i/n_dims);
+    dimensions >= n_dims are left alone.  float64 arithmetic; returns float64 [n, Hkv, D].
+    """
+    k = _f64(k_rows).copy()
+    n, hkv, d = k.shape
+    nd = d if n_dims is None else int(n_dims)
+    half = nd // 2
+    inv_freq = float(theta_base) ** (-2.0 * np.arange(half, dtype=np.float64) / nd)
+    ang = np.asarray(delta, dtype=np.float64)[:, None] * inv_freq[None, :]            # [n, half]
+    c, s_ = np.cos(ang)[:, None, :], np.sin(ang)[:, None, :]
+    x, y = k[:, :, :half].copy(), k[:, :, half:nd].copy()
+    k[:, :, :half] = x * c - y * s_
+    k[:, :, half:nd] = x * s_ + y * c
+    return k
+
+
+def compact_pack_rope(k_cache, v_cache, keep_mask, theta_base=10000.0, n_dims=None):
+    """Eager pack with the keys re-rotated to their new positions (position == slot index before and
+    after): returns (k [n, Hkv, D] float64 before storage rounding, v rows unchanged, delta [n])."""
+    keep = np.asarray(keep_mask).astype(bool)
+    src = np.nonzero(keep)[0]
+    delta = np.arange(len(src)) - src
+    return rope_reindex(np.asarray(k_cache)[src], delta, theta_base, n_dims), np.asarray(v_cache)[src], delta
 
 
 # ---------------------------------------------------------------------------

@@ -33,19 +33,6 @@ __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
 
 __device__ __forceinline__ int nonzero_bytes(uint32_t w) { return __popc(__vcmpne4(w, 0u)) >> 3; }
 
-// Loads the 16 mask bytes at [pos, pos+16) with positions >= s read as zero.
-__device__ __forceinline__ uint4 load_mask16(const uint8_t* mask, int pos, int s) {
-    uint4 v = make_uint4(0, 0, 0, 0);
-    if (pos + 16 <= s) {
-        v = *reinterpret_cast<const uint4*>(mask + pos);
-    } else if (pos < s) {
-        uint32_t w[4] = {0, 0, 0, 0};
-        for (int b = 0; b < s - pos; ++b) w[b >> 2] |= (mask[pos + b] ? 1u : 0u) << ((b & 3) * 8);
-        v = make_uint4(w[0], w[1], w[2], w[3]);
-    }
-    return v;
-}
-
 __device__ __forceinline__ int warp_excl_scan(int x, int lane, int& total) {
     int incl = x;
 #pragma unroll

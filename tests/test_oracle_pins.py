@@ -578,3 +578,43 @@ def test_plan_structural_matches_token_level_replay_and_invariants():
             for i in range(len(u)):
                 if u[i, 4] != 0 and int(u[i, 3]) not in rec and not (u[i, 5] & 1) and u[i, 2] in (0, 1):
                     assert kept[i] in (0, min(int(lens[i]), sink[int(u[i, 2])]))
+
+
+# ------------------------------------------------------------------ RoPE position re-index
+def _rope_textbook(x, pos, base, nd):
+    """RoPE from its complex-number definition: (x_i + j x_{i+nd/2}) * exp(j pos theta_i)."""
+    half = nd // 2
+    z = x[..., :half] + 1j * x[..., half:nd]
+    theta = base ** (-2.0 * np.arange(half) / nd)
+    z = z * np.exp(1j * np.asarray(pos, dtype=np.float64)[:, None, None] * theta[None, None, :])
+    out = np.array(x, dtype=np.float64, copy=True)
+    out[..., :half], out[..., half:nd] = z.real, z.imag
+    return out
+
+
+def test_rope_reindex_against_definition_and_group_properties():
+    rng = np.random.default_rng(818)
+    n, hkv, d = 37, 2, 16
+    x = rng.standard_normal((n, hkv, d))
+    pos = rng.integers(0, 5000, size=n)
+    delta = -rng.integers(0, 3000, size=n)
+    for nd in (16, 8):
+        keyed = _rope_textbook(x, pos, 10000.0, nd)                      # keys as cached at their old positions
+        moved = oc.rope_reindex(keyed, delta, 10000.0, nd)
+        assert np.allclose(moved, _rope_textbook(x, pos + delta, 10000.0, nd), rtol=0, atol=1e-9)   # == keys at the new positions
+        assert np.array_equal(moved[..., nd:], keyed[..., nd:])         # dimensions beyond n_dims untouched
+        # zero shift is the identity, a shift and its inverse compose to the identity, norms are preserved
+        assert np.array_equal(oc.rope_reindex(keyed, np.zeros(n, dtype=int), 10000.0, nd), keyed)
+        assert np.allclose(oc.rope_reindex(moved, -delta, 10000.0, nd), keyed, rtol=0, atol=1e-9)
+        assert np.allclose(np.linalg.norm(moved, axis=-1), np.linalg.norm(keyed, axis=-1))
+    # the dot product of a query and a key depends on their distance only: shifting both leaves it unchanged
+    q = _rope_textbook(rng.standard_normal((n, hkv, d)), pos + 7, 500000.0, d)
+    k = _rope_textbook(x, pos, 500000.0, d)
+    before = (q * k).sum(-1)
+    after = (oc.rope_reindex(q, delta, 500000.0) * oc.rope_reindex(k, delta, 500000.0)).sum(-1)
+    assert np.allclose(before, after, atol=1e-9)
+    # packed form: delta = new slot - old slot
+    mask = rng.random(n) < 0.5
+    kk, vv, dl = oc.compact_pack_rope(x, x + 1, mask, 10000.0)
+    assert np.array_equal(dl, np.arange(mask.sum()) - np.nonzero(mask)[0]) and np.array_equal(vv, (x + 1)[mask])
+    assert np.allclose(kk, oc.rope_reindex(x[mask], dl, 10000.0))
