@@ -482,6 +482,25 @@ def main():
         "frac": dec_bytes / (dec_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "ms": dec_ms, "bytes": dec_bytes,
         "note": f"omnitide_chunk_attention with t = 1 over {kept} retained rows (K and V read once per KV group), merge kernel included"}
 
+    # ---- the unit-granular pack with the RoPE re-index of the moved keys fused in
+    revs = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(d_reps)]
+    for i in range(3 + d_reps):
+        s_ = sets[i % R]
+        if i >= 3:
+            revs[i - 3][0].record()
+        ctx.compact_units_rope(s_["k_in"], s_["v_in"], s_["k_out"], s_["v_out"], units_in, n_units_dev, U, unit_keep, N,
+                               w.page_size, units_out, n_units_kept, None, info, None, 1000000.0, w.d)
+        if i >= 3:
+            revs[i - 3][1].record()
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0, "device status word not clean after the RoPE-fused compaction"
+    rope_ms = max_over_ranks([float(np.mean([a_.elapsed_time(b_) for a_, b_ in revs]))], world, "cuda")[0]
+    line["kernels"]["compact_rope"] = {
+        "bound": "hbm", "achieved": work["compact_bytes"] / (rope_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+        "frac": work["compact_bytes"] / (rope_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "ms": rope_ms,
+        "entry": "omnipage_compact_units_rope",
+        "note": "same bytes as compact; every moved K row is re-rotated to its new position in shared memory"}
+
     # ---- cross-layer batched compaction: the same unit decision applied to the K/V caches of 36 layers in one launch
     batched = None
     if args.batch_layers > 0:

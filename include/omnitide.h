@@ -91,6 +91,12 @@ typedef struct {
     int32_t text_budget;        /* tokens of older text spans kept, oldest first */
 } omni_structural_params;
 
+/* RoPE of the cached keys (Section 5.2 names RoPE only; the rest are the model's parameters). */
+typedef struct {
+    float theta_base;   /* frequency base, e.g. 10000 or 1000000 */
+    int32_t n_dims;     /* rotated dimensions per head: even, <= d; dimension i pairs with i + n_dims / 2 */
+} omni_rope_params;
+
 /* Integer results of one compaction, written to device memory. */
 typedef struct {
     int32_t n_kept;         /* rows retained */
@@ -226,6 +232,23 @@ omni_status omnipage_compact_units(omnitide_ctx* ctx, void* stream,
                                    int32_t s_span_max, int32_t page_size,
                                    const omni_unit* units_kept, const int32_t* n_units_kept_dev,
                                    int32_t* slot_map_out, omni_compact_info* info_out, uint8_t* page_class_out);
+
+/*
+ * (next row: RoPE position re-index fused into the gather; Section 5.2 "the runtime applies the corresponding RoPE
+ * adjustment to cached keys")  omnipage_compact_units with every moved K row re-rotated to its new position while it
+ * passes through shared memory.  Positions are slot indices (the cache is dense before and after the pack), so the
+ * shift of a row is (destination slot - source slot) <= 0; angle = shift * theta_base^(-2i / n_dims) for the pair
+ * (i, i + n_dims/2) of every head; angles in double, rotation in fp32, result rounded to bf16 (nearest even).
+ * V rows and all integer outputs are those of omnipage_compact_units.  bf16 caches only.
+ */
+omni_status omnipage_compact_units_rope(omnitide_ctx* ctx, void* stream,
+                                        const void* k_src, const void* v_src, void* k_dst, void* v_dst,
+                                        const omni_unit* units, const int32_t* n_units_dev, int32_t n_units_max,
+                                        const uint8_t* unit_keep, const int32_t* unit_kept_len,
+                                        int32_t s_span_max, int32_t page_size,
+                                        const omni_unit* units_kept, const int32_t* n_units_kept_dev,
+                                        int32_t* slot_map_out, omni_compact_info* info_out, uint8_t* page_class_out,
+                                        const omni_rope_params* rope /*[host]*/);
 
 /*
  * (next row: cross-layer batching) The unit-granular pack applied to n_layers caches in ONE launch with one shared

@@ -35,6 +35,10 @@ class StructuralParams(C.Structure):
                 ("sink_prefix", C.c_int32 * 3), ("text_budget", C.c_int32)]
 
 
+class RopeParams(C.Structure):
+    _fields_ = [("theta_base", C.c_float), ("n_dims", C.c_int32)]
+
+
 class CompactInfo(C.Structure):
     _fields_ = [("n_kept", C.c_int32), ("span_pages", C.c_int32), ("rows_moved", C.c_int32),
                 ("part_begin", C.c_int32 * 4), ("reserved", C.c_int32)]
@@ -42,7 +46,7 @@ class CompactInfo(C.Structure):
 
 EXPORTS = [
     "omnitide_create", "omnitide_destroy", "omnitide_poll_status", "omnitide_last_error",
-    "omnitide_score_units", "omnitide_select_units", "omnitide_plan_structural", "omnipage_compact", "omnipage_compact_units", "omnipage_compact_units_batched", "omnipage_append",
+    "omnitide_score_units", "omnitide_select_units", "omnitide_plan_structural", "omnipage_compact", "omnipage_compact_units", "omnipage_compact_units_rope", "omnipage_compact_units_batched", "omnipage_append",
     "omnitide_chunk_attention", "omnitide_chunk_step", "omnitide_chunk_step_host", "omnitide_chunk_step_structural",
     "omnitide_set_option", "omnitide_launch_count", "omnitide_score_units_noalloc",
 ]
@@ -69,6 +73,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.omnipage_compact.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, i32, vp, vp, vp]
     lib.omnitide_plan_structural.argtypes = [vp, vp, vp, vp, i32, C.POINTER(StructuralParams), vp, vp, vp, i32, vp, vp, vp]
     lib.omnipage_compact_units.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, i32, i32, vp, vp, vp, vp, vp]
+    lib.omnipage_compact_units_rope.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, i32, i32, vp, vp, vp, vp, vp,
+                                                C.POINTER(RopeParams)]
     lib.omnipage_compact_units_batched.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, vp, i32, vp, vp, i32, i32, vp, vp, vp,
                                                    vp, vp]
     lib.omnipage_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, i32, vp, vp]
@@ -207,6 +213,16 @@ class Context:
                                                     _ptr(n_units_kept_dev), _ptr(slot_map_out), _ptr(info_out),
                                                     _ptr(page_class_out)),
                     "omnipage_compact_units")
+
+    def compact_units_rope(self, k_src, v_src, k_dst, v_dst, units, n_units_dev, n_units_max, unit_keep, s_span_max,
+                           page_size, units_kept, n_units_kept_dev, slot_map_out, info_out, page_class_out, theta_base,
+                           n_dims, unit_kept_len=None):
+        rp = RopeParams(float(theta_base), int(n_dims))
+        self._check(self.lib.omnipage_compact_units_rope(
+            self._ctx, _stream(), _ptr(k_src), _ptr(v_src), _ptr(k_dst), _ptr(v_dst), _ptr(units), _ptr(n_units_dev),
+            n_units_max, _ptr(unit_keep), _ptr(unit_kept_len), s_span_max, page_size, _ptr(units_kept),
+            _ptr(n_units_kept_dev), _ptr(slot_map_out), _ptr(info_out), _ptr(page_class_out), C.byref(rp)),
+            "omnipage_compact_units_rope")
 
     def compact_units_batched(self, k_src_ptrs, v_src_ptrs, k_dst_ptrs, v_dst_ptrs, n_layers, units, n_units_dev,
                               n_units_max, unit_keep, s_span_max, page_size, units_kept, n_units_kept_dev, slot_map_out,

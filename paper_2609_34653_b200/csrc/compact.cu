@@ -13,6 +13,7 @@
 #include "tc_ptx.cuh"
 
 #include <algorithm>
+#include <cmath>
 
 namespace {
 
@@ -509,10 +510,90 @@ struct CompactUnitsArgs {
     const omni_unit* units_kept; const int32_t* n_units_kept_dev;
     int32_t* slot_map; omni_compact_info* info; uint8_t* page_class; int32_t* status;
     int rows_cap; int n_slots;
+    // RoPE re-index of the moved keys (rope_dims == 0: off): bf16 rows of heads of rope_head_dim elements
+    int rope_dims; int rope_head_dim; double rope_log2_base;
     // batched form: n_layers caches share the one source -> destination map (device arrays of n_layers pointers)
     int n_layers;
     const char* const* k_src_l; const char* const* v_src_l; char* const* k_dst_l; char* const* v_dst_l;
 };
+
+// The same row mover with the keys re-rotated to their new positions (Section 5.2: a kept token's position drops by
+// the number of deleted tokens before it and the runtime applies the matching RoPE adjustment to its cached key).
+// Positions are slot indices, so the shift of row r is (d0 + r) - src_list[r].  The whole warp takes part: lane 0
+// drives the bulk copies, and once a K row has landed in shared memory every lane rotates the pairs
+// (i, i + rope_dims / 2) of its dimensions i = lane, lane + 32, ... in all heads, in place, before the row is stored.
+// Angles are formed and reduced to one turn in double (a shift of 1e5 positions times a float frequency would lose
+// the phase), the rotation itself runs in fp32 and the result is rounded to bf16 (nearest even).
+__device__ __forceinline__ void move_rows_rope(const CompactUnitsArgs& a, const int* src_list, const int d0, const int n_rows,
+                                               char* rowbuf, uint64_t (*cbar)[CP_MAX_SLOTS], int* abort_flag_p) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const int n_copies = 2 * n_rows;
+    const int mcp = n_copies > wid ? (n_copies - wid + CP_WARPS - 1) / CP_WARPS : 0;
+    char* gbuf0 = rowbuf + (size_t)(wid * a.n_slots) * a.row_bytes;
+    const uint32_t buf0 = tc::smem_u32(gbuf0);
+    const int half = a.rope_dims >> 1, n_heads = (a.row_bytes >> 1) / a.rope_head_dim;
+    double inv_freq[4];                                      // rope_dims <= 256: at most four frequencies per lane
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int i = lane + 32 * j;
+        inv_freq[j] = i < half ? exp2(-(2.0 * i / a.rope_dims) * a.rope_log2_base) : 0.0;
+    }
+    auto src_of = [&](int q) {
+        const int i = wid + q * CP_WARPS;
+        return ((i & 1) ? a.v_src : a.k_src) + (size_t)src_list[i >> 1] * a.row_bytes;
+    };
+    auto issue_load = [&](int q) {
+        const int slot = q % a.n_slots;
+        const uint32_t bar = tc::smem_u32(&cbar[wid][slot]);
+        tc::mbar_expect_tx(bar, a.row_bytes);
+        bulk_load(buf0 + slot * a.row_bytes, src_of(q), a.row_bytes, bar);
+    };
+    if (lane == 0)
+        for (int q = 0; q < mcp && q < a.n_slots; ++q) issue_load(q);
+    bool ok = true;
+    for (int q = 0; q < mcp && ok; ++q) {
+        const int slot = q % a.n_slots;
+        ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&cbar[wid][slot]), (q / a.n_slots) & 1, abort_flag_p));
+        if (!ok) break;
+        const int i_copy = wid + q * CP_WARPS, row = i_copy >> 1;
+        const int delta = (d0 + row) - src_list[row];
+        if (!(i_copy & 1) && delta != 0) {
+            __nv_bfloat16* r = reinterpret_cast<__nv_bfloat16*>(gbuf0 + (size_t)slot * a.row_bytes);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int i = lane + 32 * j;
+                if (i < half) {
+                    // the phase is reduced to one turn in double (three operations), then the fast fp32 sine and
+                    // cosine (absolute error about 2^-21, far below the bf16 step of the result) do the rest
+                    const double turns = (double)delta * inv_freq[j] * 0.15915494309189535;
+                    float c, sn;
+                    __sincosf((float)((turns - rint(turns)) * 6.283185307179586), &sn, &c);
+                    for (int h = 0; h < n_heads; ++h) {
+                        __nv_bfloat16* px = r + h * a.rope_head_dim + i;
+                        const float x = __bfloat162float(px[0]), y = __bfloat162float(px[half]);
+                        px[0] = __float2bfloat16_rn(x * c - y * sn);
+                        px[half] = __float2bfloat16_rn(x * sn + y * c);
+                    }
+                }
+            }
+            tc::fence_proxy_async_smem();                    // the bulk store reads what the lanes just wrote
+        }
+        __syncwarp();
+        if (lane == 0) {
+            const char* dst_base = (i_copy & 1) ? a.v_dst : a.k_dst;
+            bulk_store(const_cast<char*>(dst_base) + (size_t)(d0 + row) * a.row_bytes, buf0 + slot * a.row_bytes, a.row_bytes);
+            if (q >= 1 && q - 1 + a.n_slots < mcp) {
+                asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                issue_load(q - 1 + a.n_slots);
+            }
+        }
+        __syncwarp();
+    }
+    if (lane == 0) {
+        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        if (!ok) atomicOr(a.status, OMNI_DEV_TIMEOUT);
+    }
+}
 
 template <bool BATCHED>
 __global__ void __launch_bounds__(CP_THREADS, 1) compact_units_kernel(const CompactUnitsArgs a) {
@@ -659,7 +740,8 @@ __global__ void __launch_bounds__(CP_THREADS, 1) compact_units_kernel(const Comp
     if (!BATCHED) {
         if (a.k_dst == nullptr) return;
         __syncthreads();                                    // the source list is complete
-        move_rows(a, src_list, d0, n_rows, rowbuf, cbar, &abort_flag);
+        if (a.rope_dims > 0) move_rows_rope(a, src_list, d0, n_rows, rowbuf, cbar, &abort_flag);
+        else move_rows(a, src_list, d0, n_rows, rowbuf, cbar, &abort_flag);
         return;
     }
     // ---- batched form: copies are numbered layer-major, (layer, destination row, K or V), and every CTA takes an
@@ -854,7 +936,7 @@ extern "C" omni_status omnipage_compact(omnitide_ctx* ctx, void* stream, const v
     return OMNI_OK;
 }
 
-extern "C" omni_status omnipage_compact_units(omnitide_ctx* ctx, void* stream, const void* k_src, const void* v_src,
+static omni_status compact_units_impl(const omni_rope_params* rope, omnitide_ctx* ctx, void* stream, const void* k_src, const void* v_src,
                                               void* k_dst, void* v_dst, const omni_unit* units,
                                               const int32_t* n_units_dev, int32_t n_units_max, const uint8_t* unit_keep,
                                               const int32_t* unit_kept_len, int32_t s_span_max, int32_t page_size,
@@ -894,6 +976,14 @@ extern "C" omni_status omnipage_compact_units(omnitide_ctx* ctx, void* stream, c
     a.slot_map = slot_map_out; a.info = info_out; a.page_class = page_class_out; a.status = ctx->status_dev;
     const int grid = ctx->sm_count;
     a.n_layers = 1; a.k_src_l = a.v_src_l = nullptr; a.k_dst_l = a.v_dst_l = nullptr;
+    a.rope_dims = 0; a.rope_head_dim = ctx->g.d; a.rope_log2_base = 0.0;
+    if (rope) {
+        if (ctx->g.dtype != OMNI_DTYPE_BF16) OMNI_FAIL(ctx, OMNI_ERR_UNSUPPORTED, "compact_units_rope: bf16 caches only");
+        if (rope->n_dims <= 0 || (rope->n_dims & 1) || rope->n_dims > ctx->g.d || rope->n_dims > 256 || !(rope->theta_base > 1.0f))
+            OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "compact_units_rope: n_dims must be even, in (0, min(d, 256)], theta_base > 1");
+        a.rope_dims = rope->n_dims;
+        a.rope_log2_base = std::log2((double)rope->theta_base);
+    }
     a.rows_cap = (((s_span_max + grid - 1) / grid + 1) + 3) & ~3;
     const size_t smem_lists = ((size_t)3 * n_units_max + 8 + a.rows_cap) * sizeof(int);
     const size_t smem_lists_al = (smem_lists + 127) & ~(size_t)127;
@@ -905,6 +995,7 @@ extern "C" omni_status omnipage_compact_units(omnitide_ctx* ctx, void* stream, c
         a.n_slots = (int)std::min<size_t>(CP_MAX_SLOTS, per_warp / ctx->row_bytes);
         if (a.n_slots < 2) a.n_slots = 0;
     }
+    if (rope && a.n_slots == 0 && k_src) OMNI_FAIL(ctx, OMNI_ERR_UNSUPPORTED, "compact_units_rope: rows of 512 bytes to 12 KB only");
     const size_t smem = smem_lists_al + (size_t)a.n_slots * CP_WARPS * ctx->row_bytes;
     if (smem > 48 * 1024)
         OMNI_CUDA(ctx, cudaFuncSetAttribute(compact_units_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -918,6 +1009,33 @@ extern "C" omni_status omnipage_compact_units(omnitide_ctx* ctx, void* stream, c
         OMNI_CHECK_LAUNCH(ctx, "copy_rows_kernel");
     }
     return OMNI_OK;
+}
+
+extern "C" omni_status omnipage_compact_units(omnitide_ctx* ctx, void* stream, const void* k_src, const void* v_src,
+                                              void* k_dst, void* v_dst, const omni_unit* units,
+                                              const int32_t* n_units_dev, int32_t n_units_max, const uint8_t* unit_keep,
+                                              const int32_t* unit_kept_len, int32_t s_span_max, int32_t page_size,
+                                              const omni_unit* units_kept,
+                                              const int32_t* n_units_kept_dev, int32_t* slot_map_out,
+                                              omni_compact_info* info_out, uint8_t* page_class_out) {
+    return compact_units_impl(nullptr, ctx, stream, k_src, v_src, k_dst, v_dst, units, n_units_dev, n_units_max, unit_keep,
+                              unit_kept_len, s_span_max, page_size, units_kept, n_units_kept_dev, slot_map_out, info_out,
+                              page_class_out);
+}
+
+extern "C" omni_status omnipage_compact_units_rope(omnitide_ctx* ctx, void* stream, const void* k_src, const void* v_src,
+                                                   void* k_dst, void* v_dst, const omni_unit* units,
+                                                   const int32_t* n_units_dev, int32_t n_units_max,
+                                                   const uint8_t* unit_keep, const int32_t* unit_kept_len,
+                                                   int32_t s_span_max, int32_t page_size, const omni_unit* units_kept,
+                                                   const int32_t* n_units_kept_dev, int32_t* slot_map_out,
+                                                   omni_compact_info* info_out, uint8_t* page_class_out,
+                                                   const omni_rope_params* rope) {
+    if (!ctx) return OMNI_ERR_INVALID_ARG;
+    if (!rope) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "compact_units_rope: null rope parameters");
+    return compact_units_impl(rope, ctx, stream, k_src, v_src, k_dst, v_dst, units, n_units_dev, n_units_max, unit_keep,
+                              unit_kept_len, s_span_max, page_size, units_kept, n_units_kept_dev, slot_map_out, info_out,
+                              page_class_out);
 }
 
 extern "C" omni_status omnipage_compact_units_batched(omnitide_ctx* ctx, void* stream, const void* const* k_src,
@@ -948,6 +1066,7 @@ extern "C" omni_status omnipage_compact_units_batched(omnitide_ctx* ctx, void* s
     a.units_kept = units_kept; a.n_units_kept_dev = n_units_kept_dev;
     a.slot_map = slot_map_out; a.info = info_out; a.page_class = page_class_out; a.status = ctx->status_dev;
     a.n_layers = n_layers;
+    a.rope_dims = 0; a.rope_head_dim = ctx->g.d; a.rope_log2_base = 0.0;
     a.k_src_l = reinterpret_cast<const char* const*>(k_src); a.v_src_l = reinterpret_cast<const char* const*>(v_src);
     a.k_dst_l = reinterpret_cast<char* const*>(k_dst); a.v_dst_l = reinterpret_cast<char* const*>(v_dst);
     const int grid = ctx->sm_count;

@@ -554,3 +554,41 @@ def test_structural_plan_then_compaction_bit_exact(H, ob):
     assert np.array_equal(H.bytes_of(got["k"][:m]).reshape(m, -1), exp["k"])
     assert np.array_equal(H.bytes_of(got["v"][:m]).reshape(m, -1), exp["v"])
     ctx.close()
+
+
+# ------------------------------------------------------------- RoPE re-index fused into the pack
+@pytest.mark.parametrize("n_dims,base", [(128, 10000.0), (64, 1000000.0)])
+def test_compact_units_rope(H, ob, n_dims, base):
+    """Keys re-rotated to their new positions while they are packed: within one bf16 step of the float64 oracle on
+    every element and bit-identical on all but a sliver (fp32 rotation vs float64); V rows and integers exact."""
+    rng = np.random.default_rng(919)
+    w = wl.layer_8b(n_hist=9000, budget=3000)
+    u, n = w.units, w.n_hist
+    keep_u = np.where(rng.random(len(u)) < 0.4, 2, 0).astype(np.uint8)
+    keep_u[0] = 2
+    mask = np.repeat(keep_u != 0, u[:, 1]).astype(np.uint8)
+    ctx = H.make_ctx(w)
+    k, v = ob.to_device(w.k_hist, "bf16"), ob.to_device(w.v_hist, "bf16")
+    kd, vd = torch.zeros_like(k), torch.zeros_like(v)
+    du = ob.units_to_device(u)
+    keep = torch.from_numpy(keep_u).cuda()
+    info = torch.zeros((8,), dtype=torch.int32, device="cuda")
+    ctx.compact_units_rope(k, v, kd, vd, du, H.i32(len(u)), len(u), keep, n, w.page_size, None, None, None, info, None, base,
+                           n_dims)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    k_ref, v_ref, delta = oc.compact_pack_rope(w.k_hist, w.v_hist, mask, base, n_dims)
+    m = len(delta)
+    assert ob.info_to_dict(info)["n_kept"] == m and (delta < 0).any()
+    assert np.array_equal(H.bytes_of(vd[:m]).reshape(m, -1), H.bytes_of(v[torch.from_numpy(np.nonzero(mask)[0]).cuda()]).reshape(m, -1))
+    got = kd[:m].float().cpu().numpy().astype(np.float64)
+    ref16 = wl.round_to_bf16(k_ref.astype(np.float32)).astype(np.float64)
+    # one bf16 step at the value's binade, plus the fp32 rounding of the two products when they cancel
+    # (x cos - y sin near zero: absolute error up to about 2^-22 of the operands, whatever the result's size)
+    step = np.abs(ref16) * 2.0 ** -7 + np.abs(w.k_hist).max() * 2.0 ** -21
+    assert (np.abs(got - ref16) <= step).all()
+    assert (got != ref16).mean() < 2e-3, (got != ref16).mean()
+    # rows that do not move (the leading kept run) are copied bit for bit
+    lead = int(np.argmin(mask)) if not mask.all() else m
+    assert np.array_equal(H.bytes_of(kd[:lead]), H.bytes_of(k[:lead]))
+    ctx.close()
