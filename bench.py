@@ -137,7 +137,7 @@ def whole_job(per_replica_value, world):
     return per_replica_value * world
 
 
-def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=64, structural=False):
+def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=64, structural=False, score_window=0):
     """The 36-layer stream loop (frames of {640, 1280, 2304} tokens plus 2 s of audio at 10-25 tok/s per
     chunk): per chunk and per layer one omnitide_chunk_step on a device-resident cache.  Returns the
     mean milliseconds per chunk over the chunks whose history already exceeds the budget (CUDA events
@@ -148,6 +148,8 @@ def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=6
     h_q, h_kv, d, t_cap, u_cap = 32, 8, 128, 2432, 96
     s_cap = ((budget + 2 * t_cap + 255) // 256) * 256
     ctx = ob.Context(h_q, h_kv, d, "bf16", s_cap, u_cap, t_cap)
+    if score_window:
+        ctx.set_option(ob.OPT_SCORE_WINDOW, score_window)
     gen = torch.Generator(device="cuda").manual_seed(4000 + rank)
     randn = lambda *shape: torch.randn(*shape, generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
     prefix = wl.loop_prefix_units()
@@ -212,7 +214,8 @@ def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=6
             "span_slots_mean": float(np.mean([r["span"] for r in steady])),
             "span_over_kept": float(np.mean([r["span"] / max(r["kept"], 1.0) for r in steady])),
             "retention_rounds": int(sum(1 for r in steady if r["evicting"])),
-            "gpu_launches": int(launches), "selection": "structural (score-free)" if structural else "scored",
+            "gpu_launches": int(launches), "selection": "structural (score-free)" if structural else
+            (f"scored by the last {score_window} queries of the chunk" if score_window else "scored by every query of the chunk"),
             "note": "36 layer steps per chunk timed with CUDA events; chunks counted from the first retention round on"}
 
 
@@ -546,6 +549,9 @@ def main():
         loop_s = run_stream_loop(ob, torch, args.loop_chunks, rank, structural=True)
         loop_s["ms_per_chunk"] = max_over_ranks([loop_s["ms_per_chunk"]], world, "cuda")[0]
         line["stream_loop_structural"] = loop_s
+        loop_w = run_stream_loop(ob, torch, args.loop_chunks, rank, score_window=128)
+        loop_w["ms_per_chunk"] = max_over_ranks([loop_w["ms_per_chunk"]], world, "cuda")[0]
+        line["stream_loop_window128"] = loop_w
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import omni_oracle as oc
         import threadpoolctl

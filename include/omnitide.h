@@ -383,8 +383,11 @@ omni_status omnitide_score_units_noalloc(void* stream, int32_t h_q, int32_t h_kv
                                          float* scores_out, float* mass_out);
 
 /* Options.  OMNI_OPT_FORCE_CUDA_CORES != 0 routes scoring and attention through the fp32 CUDA-core
- * kernels even where the tensor-core kernels apply (a second implementation for cross-checks). */
-enum { OMNI_OPT_FORCE_CUDA_CORES = 1 };
+ * kernels even where the tensor-core kernels apply (a second implementation for cross-checks).
+ * OMNI_OPT_SCORE_WINDOW = W > 0 makes omnitide_chunk_step (and its host form) score the history with the last W
+ * queries of the chunk only, a trailing observation window as in the score-based methods the paper cites (Section 3);
+ * 0 (default) scores with every query.  A caller of omnitide_score_units gets the same by passing that row range. */
+enum { OMNI_OPT_FORCE_CUDA_CORES = 1, OMNI_OPT_SCORE_WINDOW = 2 };
 omni_status omnitide_set_option(omnitide_ctx* ctx, int32_t option, int32_t value);
 
 /* Number of kernels this library has launched on this context since creation (for accounting). */

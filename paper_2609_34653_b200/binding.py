@@ -19,6 +19,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_CAPACITY = rang
 DEV_TIMEOUT, DEV_BAD_UNITS, DEV_BAD_COUNT = 1, 2, 4
 DTYPE_BF16, DTYPE_FP32 = 0, 1
 OPT_FORCE_CUDA_CORES = 1
+OPT_SCORE_WINDOW = 2
 _STATUS_NAMES = {1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "CUDA_ERROR", 4: "TIMEOUT", 5: "CAPACITY"}
 
 

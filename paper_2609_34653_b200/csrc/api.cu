@@ -118,6 +118,11 @@ extern "C" int64_t omnitide_launch_count(const omnitide_ctx* ctx) { return ctx ?
 extern "C" omni_status omnitide_set_option(omnitide_ctx* ctx, int32_t option, int32_t value) {
     if (!ctx) return OMNI_ERR_INVALID_ARG;
     if (option == OMNI_OPT_FORCE_CUDA_CORES) { ctx->force_cuda_cores = value != 0; return OMNI_OK; }
+    if (option == OMNI_OPT_SCORE_WINDOW) {
+        if (value < 0) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "score window must be >= 0");
+        ctx->score_window = value;
+        return OMNI_OK;
+    }
     OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "unknown option %d", option);
 }
 
@@ -179,7 +184,14 @@ static omni_status chunk_step_impl(cudaEvent_t chunk_kv_ready, omnitide_ctx* ctx
     int32_t* n_units_kept = ctx->ws_counts + 1;
     omni_compact_info* info = info_out ? info_out : ctx->ws_info;
     omni_status s;
-    s = omnitide_score_units(ctx, stream, q, t, k_cache, n_hist_dev, n_hist_max, units, n_units_dev, n_units_max,
+    // observation window: only the last `score_window` queries of the chunk score the history (0: all of them)
+    const void* q_score = q;
+    int32_t t_score = t;
+    if (ctx->score_window > 0 && ctx->score_window < t) {
+        t_score = ctx->score_window;
+        q_score = static_cast<const char*>(q) + (size_t)(t - t_score) * ctx->g.h_q * ctx->g.d * ctx->es;
+    }
+    s = omnitide_score_units(ctx, stream, q_score, t_score, k_cache, n_hist_dev, n_hist_max, units, n_units_dev, n_units_max,
                              w_modality, scale, ctx->ws_scores, nullptr);
     if (s) return s;
     // the keep decision stays per unit between the two steps: no token mask, no slot map inside the pass

@@ -48,6 +48,7 @@ struct omnitide_ctx {
     void* encode_tiled;           // cuTensorMapEncodeTiled, resolved through the runtime
     int64_t launches;
     bool force_cuda_cores;        // OMNI_OPT_FORCE_CUDA_CORES
+    int score_window;             // OMNI_OPT_SCORE_WINDOW: trailing queries that score in omnitide_chunk_step (0: all)
     char err[256];
 };
 

@@ -592,3 +592,45 @@ def test_compact_units_rope(H, ob, n_dims, base):
     lead = int(np.argmin(mask)) if not mask.all() else m
     assert np.array_equal(H.bytes_of(kd[:lead]), H.bytes_of(k[:lead]))
     ctx.close()
+
+
+def test_chunk_step_with_observation_window(H, ob, cfg2):
+    """OMNI_OPT_SCORE_WINDOW: the pass scores with the last W queries only; the scores equal the oracle's on
+    that row range and the selection follows the oracle's rule on them."""
+    w = cfg2
+    W = 128
+    N, T, U = w.n_hist, w.t, len(w.units)
+    ctx = ob.Context(w.h_q, w.h_kv, w.d, w.dtype, N + T + 64, U + 8, T)
+    ctx.set_option(ob.OPT_SCORE_WINDOW, W)
+    kc_in = torch.zeros((N + T + 64, w.h_kv, w.d), dtype=torch.bfloat16, device="cuda")
+    vc_in = torch.zeros_like(kc_in)
+    kc_in[:N], vc_in[:N] = ob.to_device(w.k_hist, "bf16"), ob.to_device(w.v_hist, "bf16")
+    kc_out, vc_out = torch.zeros_like(kc_in), torch.zeros_like(vc_in)
+    units_out = torch.zeros((U + 8, 6), dtype=torch.int32, device="cuda")
+    n_hist_out, n_units_out = H.i32(-1), H.i32(-1)
+    o = torch.zeros((T, w.h_q, w.d), dtype=torch.float32, device="cuda")
+    q = ob.to_device(w.q, "bf16")
+    ctx.chunk_step(q, ob.to_device(w.k_chunk, "bf16"), ob.to_device(w.v_chunk, "bf16"), T, ob.units_to_device(w.chunk_units),
+                   len(w.chunk_units), kc_in, vc_in, H.i32(N), N, ob.units_to_device(w.units, U + 8), H.i32(U), U,
+                   w.w_modality, ob.select_params(w.budget, w.n_recent_events, w.modality_cap), w.page_size, 0.0, kc_out,
+                   vc_out, units_out, n_hist_out, n_units_out, o, ob.DTYPE_FP32)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    # the scores of the window, through the scoring entry point on the same row range, against the oracle
+    win = dataclasses_replace_q(w, W)
+    s_gpu, m_gpu = H.gpu_score(ctx, win)
+    s_ref, m_ref = oc.score_units(win.q, w.k_hist, w.units, w.w_modality)
+    _check_scores(s_gpu, m_gpu, s_ref, m_ref)
+    sel = oc.select_units(w.units, s_gpu, w.budget, w.n_recent_events, w.modality_cap)
+    nu = int(n_units_out.item()) - len(w.chunk_units)
+    assert np.array_equal(units_out[:nu].cpu().numpy(), sel["units_out"])
+    assert int(n_hist_out.item()) == sel["n_kept"] + T
+    # and the window changes the decision input: scores of all queries differ from scores of the window
+    s_all, _ = oc.score_units(w.q, w.k_hist, w.units, w.w_modality)
+    assert np.abs(s_all - s_ref).max() > 1e-3
+    ctx.close()
+
+
+def dataclasses_replace_q(w, W):
+    import dataclasses
+    return dataclasses.replace(w, q=np.ascontiguousarray(w.q[-W:]))
