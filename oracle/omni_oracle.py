@@ -38,6 +38,16 @@ What follows the paper and what does not
                        boundary span are parameters the paper leaves open;
                        pinned by a hand-worked example, an independent
                        token-level replay and invariants.
+* migrate_suffix    -- OmniPage's ordered-suffix migration, the mode the paper uses
+                       on CUDA (Section 6.2 "Checking layout improvement"): scan
+                       backward for the smallest suffix whose packing shortens
+                       the page-rounded span by at least a configured number of
+                       pages, pack only that suffix in order, leave the rest in
+                       place; no migration if no suffix qualifies.  Page
+                       alignment of the suffix start and the default threshold
+                       are readings.  Pinned by brute force over every suffix
+                       start and by invariants.  Attention over the resulting
+                       layout with holes is attention over the live rows.
 * rope_reindex      -- the position shift the runtime applies to cached keys after
                        logical deletion (Section 5.2): a kept token's position
                        drops by the number of deleted tokens before it and its
@@ -413,6 +423,61 @@ def chunk_attention(q, k_hist, v_hist, k_chunk, v_chunk, scale=None, rows=None):
         o[:, h, :] = (p[:, :Nh] @ vh[:, g, :] + p[:, Nh:] @ vc[:, g, :]) / z
         lse[:, h] = (m + np.log(z))[:, 0]
     return o, lse
+
+
+# ---------------------------------------------------------------------------
+# M -- selective migration, ordered-suffix mode
+# ---------------------------------------------------------------------------
+def migrate_suffix(k_cache, v_cache, keep_mask, page_size, min_pages_saved=1):
+    """Pack only a suffix of the cache (Section 6.2, ordered-suffix mode).
+
+    keep_mask [S] marks the live slots of the span [0, S).  Among the page-aligned suffix starts
+    p = 0, P, 2P, ... the LARGEST one (the smallest suffix, found by scanning backward from the end)
+    is taken whose packing shortens the page-rounded span by at least `min_pages_saved` pages:
+        new_span(p) = p + #live slots in [p, S);   saved(p) = ceil(S / P) - ceil(new_span(p) / P).
+    The live rows of [p, S) are packed, in order, to slots p, p+1, ...; every slot before p keeps its
+    content and its hole pattern.  If no suffix qualifies nothing moves.  As-if semantics: all reads
+    precede all writes.
+    Returns dict(start (p, or -1 when nothing moves), k, v (caches of S rows after the move; rows at
+    and beyond new_span are unspecified and returned unchanged), keep_mask (the new one), new_span,
+    pages_saved, rows_moved, slot_map [S] (new slot of every live row, -1 for dead ones)).
+    """
+    keep = np.asarray(keep_mask).astype(bool)
+    S, P = len(keep), int(page_size)
+    pages = lambda n: (n + P - 1) // P
+    start = -1
+    for p in range(((S - 1) // P) * P if S else -P, -1, -P):            # backward from the last page
+        live = int(keep[p:].sum())
+        if pages(S) - pages(p + live) >= min_pages_saved:
+            start = p
+            break
+    k = np.array(k_cache, copy=True) if k_cache is not None else None
+    v = np.array(v_cache, copy=True) if v_cache is not None else None
+    new_mask = keep.copy()
+    slot_map = np.where(keep, np.arange(S), -1).astype(np.int32)
+    if start < 0:
+        return dict(start=-1, k=k, v=v, keep_mask=new_mask.astype(np.uint8), new_span=S, pages_saved=0, rows_moved=0,
+                    slot_map=slot_map)
+    src = start + np.nonzero(keep[start:])[0]
+    dst = start + np.arange(len(src))
+    if k is not None:
+        k[dst] = np.asarray(k_cache)[src]
+        v[dst] = np.asarray(v_cache)[src]
+    new_mask[start:] = False
+    new_mask[dst] = True
+    slot_map[src] = dst
+    new_span = start + len(src)
+    return dict(start=start, k=k, v=v, keep_mask=new_mask.astype(np.uint8), new_span=new_span,
+                pages_saved=pages(S) - pages(new_span), rows_moved=int((src != dst).sum()), slot_map=slot_map)
+
+
+def chunk_attention_masked(q, k_cache, v_cache, keep_mask, k_chunk, v_chunk, scale=None, rows=None):
+    """Attention over a history with holes: only the live slots are visible (Section 6, "Fragmentation
+    after logical eviction": masked entries are not attended to).  By definition this is dense
+    attention over the live rows in order."""
+    live = np.asarray(keep_mask).astype(bool)
+    n = len(live)
+    return chunk_attention(q, np.asarray(k_cache)[:n][live], np.asarray(v_cache)[:n][live], k_chunk, v_chunk, scale, rows)
 
 
 # ---------------------------------------------------------------------------

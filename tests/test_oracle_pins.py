@@ -618,3 +618,64 @@ def test_rope_reindex_against_definition_and_group_properties():
     kk, vv, dl = oc.compact_pack_rope(x, x + 1, mask, 10000.0)
     assert np.array_equal(dl, np.arange(mask.sum()) - np.nonzero(mask)[0]) and np.array_equal(vv, (x + 1)[mask])
     assert np.allclose(kk, oc.rope_reindex(x[mask], dl, 10000.0))
+
+
+# ------------------------------------------------------------------ ordered-suffix migration
+def test_migrate_suffix_brute_force_and_invariants():
+    rng = np.random.default_rng(929)
+    for trial in range(400):
+        P = int(rng.choice([4, 8, 16]))
+        S = int(rng.integers(1, 200))
+        dens = rng.random()
+        keep = (rng.random(S) < dens).astype(np.uint8)
+        if rng.random() < 0.3:                                   # a dense head and a sparse tail, the case the mode is for
+            keep[:S // 2] = 1
+        theta = int(rng.integers(1, 4))
+        k = rng.integers(0, 1 << 30, size=(S, 3))
+        v = rng.integers(0, 1 << 30, size=(S, 3))
+        r = oc.migrate_suffix(k, v, keep, P, theta)
+        pages = lambda n: -(-n // P)
+        # brute force over every page-aligned start: the chosen one is the largest that saves >= theta pages
+        ok = [p for p in range(0, S, P) if pages(S) - pages(p + int(keep[p:].sum())) >= theta]
+        assert r["start"] == (max(ok) if ok else -1)
+        if not ok:
+            assert r["rows_moved"] == 0 and np.array_equal(r["keep_mask"], keep) and np.array_equal(r["k"], k)
+            continue
+        p = r["start"]
+        assert p % P == 0 and r["pages_saved"] >= theta and r["new_span"] == p + int(keep[p:].sum())
+        # everything before the suffix is untouched: contents and holes
+        assert np.array_equal(r["k"][:p], k[:p]) and np.array_equal(r["keep_mask"][:p], keep[:p])
+        # the suffix is packed in order: the live rows after the move are the live rows before it, same order
+        live_before = np.nonzero(keep)[0]
+        live_after = np.nonzero(r["keep_mask"])[0]
+        assert np.array_equal(r["k"][live_after], k[live_before]) and np.array_equal(r["v"][live_after], v[live_before])
+        assert np.array_equal(r["slot_map"][live_before], live_after) and (r["slot_map"][keep == 0] == -1).all()
+        assert r["keep_mask"][p:r["new_span"]].all() and not r["keep_mask"][r["new_span"]:].any()
+        assert r["rows_moved"] == int((live_before != live_after).sum())
+    # worked by hand: 12 slots, pages of 4, live slots {0, 2, 3, 6, 8, 11}.  Packing [8, 12) gives span 10 (3 pages, none
+    # saved); packing [4, 12) gives span 7 (2 pages, one saved): the scan stops there; nothing saves two pages.
+    keep = np.array([1, 0, 1, 1, 0, 0, 1, 0, 1, 0, 0, 1], dtype=np.uint8)
+    r = oc.migrate_suffix(np.arange(12), np.arange(12) + 100, keep, 4, 1)
+    assert r["start"] == 4 and r["new_span"] == 7 and r["pages_saved"] == 1 and r["rows_moved"] == 3
+    assert r["k"][:7].tolist() == [0, 1, 2, 3, 6, 8, 11] and r["keep_mask"].tolist() == [1, 0, 1, 1, 1, 1, 1, 0, 0, 0, 0, 0]
+    assert oc.migrate_suffix(np.arange(12), np.arange(12) + 100, keep, 4, 2)["start"] == -1
+
+
+def test_attention_masked_is_attention_over_live_rows():
+    w = wl.tiny()
+    rng = np.random.default_rng(939)
+    keep = (rng.random(w.n_hist) < 0.6).astype(np.uint8)
+    o, lse = oc.chunk_attention_masked(w.q, w.k_hist, w.v_hist, keep, w.k_chunk, w.v_chunk)
+    # brute force for a few outputs: explicit -inf on the dead slots of the FULL history
+    for i, h in [(0, 0), (17, 3), (255, 1)]:
+        keys = np.concatenate([w.k_hist[:, 0], w.k_chunk[:i + 1, 0]]).astype(np.float64)
+        vals = np.concatenate([w.v_hist[:, 0], w.v_chunk[:i + 1, 0]]).astype(np.float64)
+        s = keys @ w.q[i, h].astype(np.float64) / math.sqrt(w.d)
+        s[:w.n_hist][keep == 0] = -np.inf
+        p = np.exp(s - s.max())
+        assert np.allclose(o[i, h], (p @ vals) / p.sum(), atol=1e-12)
+    # a suffix migration does not change what attention sees
+    m = oc.migrate_suffix(w.k_hist, w.v_hist, keep, 16, 1)
+    assert m["start"] >= 0
+    o2, _ = oc.chunk_attention_masked(w.q, m["k"], m["v"], m["keep_mask"], w.k_chunk, w.v_chunk)
+    assert np.allclose(o, o2, atol=1e-12)
