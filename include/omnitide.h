@@ -319,6 +319,22 @@ omni_status omnitide_chunk_step(omnitide_ctx* ctx, void* stream,
                                 void* o_out, int32_t out_dtype, omni_compact_info* info_out);
 
 /*
+ * (next row: layouts with holes)  omnitide_chunk_attention over a history in which only the slots marked in
+ * hist_keep_mask are live (Section 6, "Fragmentation after logical eviction": logical deletion leaves masked holes
+ * between surviving entries; Section 6.1: a tile is skipped only when all its entries are masked).  The span
+ * [0, *s_span_dev) of k_hist / v_hist is presented; 128-key blocks with no live slot are skipped (no load, no MMA),
+ * the other blocks have their dead columns masked.  Equals attention over the live rows in order.
+ *   hist_keep_mask [dev] s_span_max bytes readable up to a multiple of 16 (nonzero = live), 16-byte aligned;
+ *   dead slots inside the span must hold finite values (evicted entries do); slots beyond the span may hold anything.
+ */
+omni_status omnitide_chunk_attention_masked(omnitide_ctx* ctx, void* stream,
+                                            const void* q, int32_t t,
+                                            const void* k_hist, const void* v_hist, const uint8_t* hist_keep_mask,
+                                            const int32_t* s_span_dev, int32_t s_span_max,
+                                            const void* k_chunk, const void* v_chunk, float scale,
+                                            void* o_out, int32_t out_dtype, float* lse_out);
+
+/*
  * The pass as the paper runs it (no scoring): omnitide_plan_structural -> omnipage_compact_units with the planned
  * prefix lengths -> omnitide_chunk_attention -> omnipage_append.  Arguments as omnitide_chunk_step, with the
  * structural parameters in place of the modality weights and the selection parameters.

@@ -48,7 +48,7 @@ class CompactInfo(C.Structure):
 EXPORTS = [
     "omnitide_create", "omnitide_destroy", "omnitide_poll_status", "omnitide_last_error",
     "omnitide_score_units", "omnitide_select_units", "omnitide_plan_structural", "omnipage_compact", "omnipage_compact_units", "omnipage_compact_units_rope", "omnipage_compact_units_batched", "omnipage_append",
-    "omnitide_chunk_attention", "omnitide_chunk_step", "omnitide_chunk_step_host", "omnitide_chunk_step_structural",
+    "omnitide_chunk_attention", "omnitide_chunk_attention_masked", "omnitide_chunk_step", "omnitide_chunk_step_host", "omnitide_chunk_step_structural",
     "omnitide_set_option", "omnitide_launch_count", "omnitide_score_units_noalloc",
 ]
 NOALLOC_MAX_UNITS = 1024
@@ -80,6 +80,7 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
                                                    vp, vp]
     lib.omnipage_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, i32, vp, vp]
     lib.omnitide_chunk_attention.argtypes = [vp, vp, vp, i32, vp, vp, vp, i32, vp, vp, f32, vp, i32, vp]
+    lib.omnitide_chunk_attention_masked.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, i32, vp, vp, f32, vp, i32, vp]
     lib.omnitide_score_units_noalloc.argtypes = [vp, i32, i32, i32, i32, vp, i32, vp, i32, vp, i32, C.POINTER(f32), f32,
                                                  vp, vp]
     step = [vp, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp, i32, vp, vp, i32, C.POINTER(f32),
@@ -248,6 +249,14 @@ class Context:
                                                       _ptr(n_hist_dev), n_hist_max, _ptr(k_chunk), _ptr(v_chunk),
                                                       float(scale), _ptr(o_out), out_dtype, _ptr(lse_out)),
                     "omnitide_chunk_attention")
+
+    def chunk_attention_masked(self, q, t, k_hist, v_hist, hist_keep_mask, s_span_dev, s_span_max, k_chunk, v_chunk, scale,
+                               o_out, out_dtype, lse_out=None):
+        self._check(self.lib.omnitide_chunk_attention_masked(self._ctx, _stream(), _ptr(q), t, _ptr(k_hist), _ptr(v_hist),
+                                                             _ptr(hist_keep_mask), _ptr(s_span_dev), s_span_max,
+                                                             _ptr(k_chunk), _ptr(v_chunk), float(scale), _ptr(o_out),
+                                                             out_dtype, _ptr(lse_out)),
+                    "omnitide_chunk_attention_masked")
 
     def _step(self, fn, name, hp, q, k_chunk, v_chunk, t, chunk_units, n_chunk_units, k_cache, v_cache, n_hist_dev,
               n_hist_max, units, n_units_dev, n_units_max, w_modality, params, page_size, scale, k_cache_out,

@@ -18,7 +18,8 @@ cudaError_t alloc(T** p, size_t n) {
 void free_all(omnitide_ctx* c) {
     void* ptrs[] = {c->status_dev, c->score_part, c->score_tile_mass, c->score_mass64, c->inplace_k, c->inplace_v,
                     c->ws_scores, c->ws_unit_keep, c->ws_kept_len, c->ws_keep_mask, c->ws_slot_map, c->ws_counts, c->ws_info, c->st_q,
-                    c->st_k, c->st_v, c->st_o, c->st_units, c->attn_part_o, c->attn_part_ml, c->cp_words};
+                    c->st_k, c->st_v, c->st_o, c->st_units, c->attn_part_o, c->attn_part_ml, c->cp_words, c->attn_live_idx, c->attn_live_mask,
+                    c->attn_n_live};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
@@ -58,6 +59,9 @@ extern "C" omni_status omnitide_create(omnitide_ctx** ctx_out, const omni_geomet
     ok &= cudaStreamCreateWithFlags(&c->aux_stream, cudaStreamNonBlocking) == cudaSuccess;
     ok &= cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
     ok &= cudaEventCreateWithFlags(&c->ev_kv, cudaEventDisableTiming) == cudaSuccess;
+    ok &= alloc(&c->attn_live_idx, (size_t)g->s_cap / 128 + 2) == cudaSuccess;
+    ok &= alloc(&c->attn_live_mask, (size_t)g->s_cap / 128 + 2) == cudaSuccess;
+    ok &= alloc(&c->attn_n_live, (size_t)1) == cudaSuccess;
     ok &= alloc(&c->cp_words, (size_t)c->sm_count + 1) == cudaSuccess;
     ok = ok && cudaMemset(c->cp_words, 0, ((size_t)c->sm_count + 1) * sizeof(unsigned long long)) == cudaSuccess;
     ok &= alloc(&c->ws_scores, (size_t)g->u_cap) == cudaSuccess;
@@ -145,7 +149,7 @@ extern "C" omni_status omnitide_score_units(omnitide_ctx* ctx, void* stream, con
                              scale, scores_out, mass_out);
 }
 
-extern "C" omni_status omnitide_chunk_attention(omnitide_ctx* ctx, void* stream, const void* q, int32_t t,
+static omni_status chunk_attention_impl(const uint8_t* hist_mask, omnitide_ctx* ctx, void* stream, const void* q, int32_t t,
                                                 const void* k_hist, const void* v_hist, const int32_t* n_hist_dev,
                                                 int32_t n_hist_max, const void* k_chunk, const void* v_chunk, float scale,
                                                 void* o_out, int32_t out_dtype, float* lse_out) {
@@ -156,15 +160,34 @@ extern "C" omni_status omnitide_chunk_attention(omnitide_ctx* ctx, void* stream,
     if (n_hist_max < 0 || n_hist_max > ctx->g.s_cap) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "attention: n_hist_max outside [0, s_cap]");
     if (out_dtype != OMNI_DTYPE_BF16 && out_dtype != OMNI_DTYPE_FP32) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "attention: bad out_dtype");
     if (!omni_aligned16(q) || !omni_aligned16(k_hist) || !omni_aligned16(v_hist) || !omni_aligned16(k_chunk) ||
-        !omni_aligned16(v_chunk) || !omni_aligned16(o_out))
+        !omni_aligned16(v_chunk) || !omni_aligned16(o_out) || !omni_aligned16(hist_mask))
         OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "attention: pointers must be 16-byte aligned");
     if (scale <= 0.f) scale = 1.0f / sqrtf((float)ctx->g.d);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (tc_geometry(ctx))
         return omni_attention_tc(ctx, st, q, t, k_hist, v_hist, n_hist_dev, n_hist_max, k_chunk, v_chunk, scale, o_out,
-                                 out_dtype, lse_out);
+                                 out_dtype, lse_out, hist_mask);
     return omni_attention_simple(ctx, st, q, t, k_hist, v_hist, n_hist_dev, n_hist_max, k_chunk, v_chunk, scale, o_out,
-                                 out_dtype, lse_out);
+                                 out_dtype, lse_out, hist_mask);
+}
+
+extern "C" omni_status omnitide_chunk_attention(omnitide_ctx* ctx, void* stream, const void* q, int32_t t,
+                                                const void* k_hist, const void* v_hist, const int32_t* n_hist_dev,
+                                                int32_t n_hist_max, const void* k_chunk, const void* v_chunk, float scale,
+                                                void* o_out, int32_t out_dtype, float* lse_out) {
+    return chunk_attention_impl(nullptr, ctx, stream, q, t, k_hist, v_hist, n_hist_dev, n_hist_max, k_chunk, v_chunk, scale,
+                                o_out, out_dtype, lse_out);
+}
+
+extern "C" omni_status omnitide_chunk_attention_masked(omnitide_ctx* ctx, void* stream, const void* q, int32_t t,
+                                                       const void* k_hist, const void* v_hist, const uint8_t* hist_keep_mask,
+                                                       const int32_t* s_span_dev, int32_t s_span_max, const void* k_chunk,
+                                                       const void* v_chunk, float scale, void* o_out, int32_t out_dtype,
+                                                       float* lse_out) {
+    if (!ctx) return OMNI_ERR_INVALID_ARG;
+    if (!hist_keep_mask && s_span_max > 0) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "attention_masked: null keep mask");
+    return chunk_attention_impl(hist_keep_mask, ctx, stream, q, t, k_hist, v_hist, s_span_dev, s_span_max, k_chunk, v_chunk,
+                                scale, o_out, out_dtype, lse_out);
 }
 
 static omni_status chunk_step_impl(cudaEvent_t chunk_kv_ready, omnitide_ctx* ctx, void* stream, const void* q, const void* k_chunk,

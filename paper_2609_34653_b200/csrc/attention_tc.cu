@@ -75,6 +75,9 @@ struct AttnParams {
     void* o_out; int out_dtype; float* lse_out;
     int32_t* status;
     int n_tiles;          // query tiles of 128 rows
+    // history with holes (all three null: dense history): the 128-key blocks that hold a live slot, their live bits,
+    // and how many there are; written by attn_block_scan_kernel before this launch
+    const int32_t* live_idx; const uint4* live_mask; const int32_t* n_live;
     int pack_shift;       // >= 0: GQA-packed single tile, row r = (token r >> pack_shift, head of the group r & (G-1)); -1: off
     float* part_o;        // [cta][2 slots][128 rows][128] un-normalised partial outputs
     float2* part_ml;      // [cta][2 slots][128 rows] (running max, sum)
@@ -170,9 +173,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (threadIdx.x == 0 && blockIdx.x == 0) atomicOr(p.status, OMNI_DEV_BAD_COUNT);
         n_hist = max(0, min(n_hist, p.n_hist_max));
     }
-    const int nhb = (n_hist + BK - 1) / BK;
-    const int hist_tail = n_hist - (nhb - 1) * BK;           // valid keys in the last history block (if nhb > 0)
-    const bool tail_partial = nhb > 0 && hist_tail < BK;
+    // with holes only the live blocks are visited: block j of the history is block live_idx[j] of the cache
+    const bool masked = p.live_idx != nullptr;
+    const int nb_span = (n_hist + BK - 1) / BK;
+    const int nhb = masked ? max(0, min(*p.n_live, nb_span)) : nb_span;
+    const int hist_tail = n_hist - (nb_span - 1) * BK;       // slots of the span in its last block (if nb_span > 0)
+    // rows of the last visited block beyond the span may hold anything: they are masked in S and zeroed in V
+    const bool tail_partial = nhb > 0 && hist_tail < BK && (!masked || p.live_idx[nhb - 1] == nb_span - 1);
 
     PartIter it;
     // GQA-packed mode (few queries, e.g. decode): one tile holds all query heads of a KV group, items are KV heads
@@ -239,7 +246,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 tc::mbar_expect_tx(full, TILE_BYTES);
                 const bool hist = j < nhb;
                 const CUtensorMap* map = hist ? (is_v ? &tm_vh : &tm_kh) : (is_v ? &tm_vc : &tm_kc);
-                const int row = (hist ? j : j - nhb) * BK;
+                const int row = (hist ? (masked ? __ldg(p.live_idx + j) : j) : j - nhb) * BK;
                 const uint32_t dst = kv_smem + stage * TILE_BYTES;
                 tc::tma_load_2d(dst, map, kvh * HD, row, full);
                 tc::tma_load_2d(dst + HALF_BYTES, map, kvh * HD + 64, row, full);
@@ -380,6 +387,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const int buf = g & 1;                                     // P buffer of this block
                 const uint32_t s_tmem = tmem + w * HK + lane_addr;
                 const uint32_t p_tmem = tmem + 128 + buf * 64 + w * 32 + lane_addr;
+                // live bits of this warpgroup's 64 keys (all ones for a dense history and for chunk blocks); the load is
+                // issued before the wait for S so that its latency is hidden
+                unsigned long long live = ~0ull;
+                if (masked && j < nhb) live = __ldg(reinterpret_cast<const unsigned long long*>(p.live_mask + j) + w);
                 ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&bars->s_full), g & 1, abort_flag));
                 tc::tcgen05_fence_after();
                 if ((warp & 3) == 0) TRACE(w, 0);
@@ -400,6 +411,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     for (int i = 0; i < 32; ++i) {
                         if (i >= n_valid) sa[i] = 0xff800000u;           // -inf
                         if (32 + i >= n_valid) sb[i] = 0xff800000u;
+                    }
+                }
+                if (live != ~0ull) {                         // holes inside the block (warp-uniform: one mask per block)
+                    const uint32_t lo = (uint32_t)live, hi = (uint32_t)(live >> 32);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        if (!((lo >> i) & 1u)) sa[i] = 0xff800000u;
+                        if (!((hi >> i) & 1u)) sb[i] = 0xff800000u;
                     }
                 }
                 // row maximum of the 64 logits: three-input maxima, four independent chains
@@ -586,6 +605,66 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
 }
 
+// History with holes: which 128-key blocks hold a live slot, and their live bits.  One CTA; thread b takes block b
+// (and b + 1024, ...); the live blocks are numbered by a block-wide scan.  Slots at and beyond the span count as dead.
+__global__ void __launch_bounds__(1024) attn_block_scan_kernel(const uint8_t* __restrict__ mask, const int32_t* n_hist_dev,
+                                                               int n_hist_max, int32_t* live_idx, uint4* live_mask,
+                                                               int32_t* n_live, int32_t* status) {
+    __shared__ int warp_tot[32];
+    __shared__ int s_base;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    int n_hist = n_hist_dev ? *n_hist_dev : n_hist_max;
+    if (n_hist < 0 || n_hist > n_hist_max) {
+        if (tid == 0) atomicOr(status, OMNI_DEV_BAD_COUNT);
+        n_hist = max(0, min(n_hist, n_hist_max));
+    }
+    const int nb = (n_hist + BK - 1) / BK;
+    if (tid == 0) s_base = 0;
+    __syncthreads();
+    for (int b0 = 0; b0 < nb; b0 += 1024) {
+        const int b = b0 + tid;
+        uint32_t bits[4] = {0u, 0u, 0u, 0u};
+        if (b < nb) {
+#pragma unroll
+            for (int v = 0; v < 8; ++v) {
+                const int pos = b * BK + v * 16;
+                if (pos < n_hist) {
+                    const uint4 m = __ldg(reinterpret_cast<const uint4*>(mask + pos));
+                    const uint32_t w4[4] = {m.x, m.y, m.z, m.w};
+                    uint32_t sixteen = 0u;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const uint32_t nz = __vcmpne4(w4[k], 0u);        // 0xff per live byte
+                        const uint32_t nib = ((nz >> 7) & 1u) | ((nz >> 14) & 2u) | ((nz >> 21) & 4u) | ((nz >> 28) & 8u);
+                        sixteen |= nib << (4 * k);
+                    }
+                    const int valid = n_hist - pos;                      // < 16 only in the last vector of the span
+                    if (valid < 16) sixteen &= (1u << valid) - 1u;
+                    bits[v >> 1] |= sixteen << ((v & 1) * 16);
+                }
+            }
+        }
+        const bool live = (bits[0] | bits[1] | bits[2] | bits[3]) != 0u;
+        const unsigned ballot = __ballot_sync(0xffffffffu, live);
+        if (lane == 0) warp_tot[wid] = __popc(ballot);
+        __syncthreads();
+        int before = s_base + __popc(ballot & ((1u << lane) - 1u));
+        for (int w = 0; w < wid; ++w) before += warp_tot[w];
+        if (live) {
+            live_idx[before] = b;
+            live_mask[before] = make_uint4(bits[0], bits[1], bits[2], bits[3]);
+        }
+        __syncthreads();
+        if (tid == 0) {
+            int tot = 0;
+            for (int w = 0; w < 32; ++w) tot += warp_tot[w];
+            s_base += tot;
+        }
+        __syncthreads();
+    }
+    if (tid == 0) *n_live = s_base;
+}
+
 // Merge the partial outputs of every item that was cut between CTAs.  Grid (share boundaries, 4 groups of 32 rows);
 // a warp owns 4 rows and a lane 4 of a row's 128 columns.  Shared memory: one int per CTA of the main kernel.
 constexpr int MERGE_BATCH = 4;
@@ -605,6 +684,7 @@ __global__ void __launch_bounds__(256) attention_merge_kernel(const AttnParams p
     n_hist = max(0, min(n_hist, p.n_hist_max));
     Sched s;
     s.nhb = (n_hist + BK - 1) / BK; s.n_tiles = p.n_tiles; s.h_q = p.pack_shift >= 0 ? p.h_kv : p.h_q;
+    if (p.live_idx) s.nhb = max(0, min(*p.n_live, s.nhb));
     const long long total = s.total();
     // share boundaries, one per thread (the divisions run in parallel), kept behind the slot list
     long long* s_begin = reinterpret_cast<long long*>(s_slot + ((n_cta + 2) & ~1));         // [n_cta + 1]
@@ -689,7 +769,8 @@ __global__ void __launch_bounds__(256) attention_merge_kernel(const AttnParams p
 
 omni_status omni_attention_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q, int t, const void* k_hist,
                               const void* v_hist, const int32_t* n_hist_dev, int n_hist_max, const void* k_chunk,
-                              const void* v_chunk, float scale, void* o_out, int out_dtype, float* lse_out) {
+                              const void* v_chunk, float scale, void* o_out, int out_dtype, float* lse_out,
+                              const uint8_t* hist_mask) {
     const omni_geometry& g = ctx->g;
     CUtensorMap tm_q, tm_kh, tm_vh, tm_kc, tm_vc;
     const uint64_t q_inner = (uint64_t)g.h_q * HD, kv_inner = (uint64_t)g.h_kv * HD;
@@ -712,6 +793,13 @@ omni_status omni_attention_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q,
     p.scale = scale; p.scale_log2 = scale * 1.4426950408889634f;
     p.o_out = o_out; p.out_dtype = out_dtype; p.lse_out = lse_out; p.status = ctx->status_dev;
     p.pack_shift = pack_shift;
+    p.live_idx = nullptr; p.live_mask = nullptr; p.n_live = nullptr;
+    if (hist_mask && n_hist_max > 0) {
+        attn_block_scan_kernel<<<1, 1024, 0, st>>>(hist_mask, n_hist_dev, n_hist_max, ctx->attn_live_idx, ctx->attn_live_mask,
+                                                   ctx->attn_n_live, ctx->status_dev);
+        OMNI_CHECK_LAUNCH(ctx, "attn_block_scan_kernel");
+        p.live_idx = ctx->attn_live_idx; p.live_mask = ctx->attn_live_mask; p.n_live = ctx->attn_n_live;
+    }
     p.n_tiles = pack_shift >= 0 ? 1 : (t + BQ - 1) / BQ;
     const int n_items_heads = pack_shift >= 0 ? g.h_kv : g.h_q;
     // one CTA per SM, fewer when the whole job is small (at least 4 block steps per CTA)

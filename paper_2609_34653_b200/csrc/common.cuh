@@ -43,6 +43,9 @@ struct omnitide_ctx {
     float* attn_part_o;           // allocated on first use
     float* attn_part_ml;
     size_t attn_part_cap;
+    int32_t* attn_live_idx;       // [s_cap / 128 + 2] blocks of the history that hold a live slot (masked attention)
+    uint4* attn_live_mask;        // [s_cap / 128 + 2] their 128 live bits
+    int32_t* attn_n_live;
     bool attn_attr_set;           // the attention kernel's shared-memory limit has been raised on this device
     // -----------------------------------------------------------------------------------
     void* encode_tiled;           // cuTensorMapEncodeTiled, resolved through the runtime
@@ -78,14 +81,16 @@ static inline bool omni_aligned16(const void* p) { return (reinterpret_cast<uint
 // internal entry points implemented per file
 omni_status omni_attention_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q, int t, const void* k_hist,
                               const void* v_hist, const int32_t* n_hist_dev, int n_hist_max, const void* k_chunk,
-                              const void* v_chunk, float scale, void* o_out, int out_dtype, float* lse_out);
+                              const void* v_chunk, float scale, void* o_out, int out_dtype, float* lse_out,
+                              const uint8_t* hist_mask);
 omni_status omni_score_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q, int t, const void* k_cache,
                           const int32_t* n_hist_dev, int n_hist_max, const omni_unit* units,
                           const int32_t* n_units_dev, int n_units_max, const float* w, float scale,
                           float* scores_out, float* mass_out);
 omni_status omni_attention_simple(omnitide_ctx* ctx, cudaStream_t st, const void* q, int t, const void* k_hist,
                                   const void* v_hist, const int32_t* n_hist_dev, int n_hist_max, const void* k_chunk,
-                                  const void* v_chunk, float scale, void* o_out, int out_dtype, float* lse_out);
+                                  const void* v_chunk, float scale, void* o_out, int out_dtype, float* lse_out,
+                                  const uint8_t* hist_mask);
 omni_status omni_score_simple(omnitide_ctx* ctx, cudaStream_t st, const void* q, int t, const void* k_cache,
                               const int32_t* n_hist_dev, int n_hist_max, const omni_unit* units,
                               const int32_t* n_units_dev, int n_units_max, const float* w, float scale,

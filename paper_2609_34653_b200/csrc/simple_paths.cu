@@ -24,7 +24,8 @@ template <typename T>
 __global__ void __launch_bounds__(SP_WARPS * 32) attention_rows_kernel(
     const T* __restrict__ q, int t, int h_q, int h_kv, int d, const T* __restrict__ k_hist,
     const T* __restrict__ v_hist, const int32_t* n_hist_dev, int n_hist_max, const T* __restrict__ k_chunk,
-    const T* __restrict__ v_chunk, float scale, void* o_out, int out_dtype, float* lse_out, int32_t* status) {
+    const T* __restrict__ v_chunk, float scale, void* o_out, int out_dtype, float* lse_out, int32_t* status,
+    const uint8_t* __restrict__ hist_mask) {
     const int lane = threadIdx.x & 31;
     const long long row = (long long)blockIdx.x * SP_WARPS + (threadIdx.x >> 5);
     if (row >= (long long)t * h_q) return;
@@ -46,6 +47,7 @@ __global__ void __launch_bounds__(SP_WARPS * 32) attention_rows_kernel(
     const size_t kv_stride = (size_t)h_kv * d;
     const int n_keys = n_hist + i + 1;
     for (int j = 0; j < n_keys; ++j) {
+        if (hist_mask && j < n_hist && hist_mask[j] == 0) continue;      // a hole of the history: not visible
         const T* kr = j < n_hist ? k_hist + (size_t)j * kv_stride + (size_t)g * d
                                  : k_chunk + (size_t)(j - n_hist) * kv_stride + (size_t)g * d;
         const T* vr = j < n_hist ? v_hist + (size_t)j * kv_stride + (size_t)g * d
@@ -168,19 +170,20 @@ __global__ void score_finalize64_kernel(const double* mass64, const omni_unit* u
 
 omni_status omni_attention_simple(omnitide_ctx* ctx, cudaStream_t st, const void* q, int t, const void* k_hist,
                                   const void* v_hist, const int32_t* n_hist_dev, int n_hist_max, const void* k_chunk,
-                                  const void* v_chunk, float scale, void* o_out, int out_dtype, float* lse_out) {
+                                  const void* v_chunk, float scale, void* o_out, int out_dtype, float* lse_out,
+                                  const uint8_t* hist_mask) {
     const omni_geometry& g = ctx->g;
     const long long rows = (long long)t * g.h_q;
     const int grid = (int)((rows + SP_WARPS - 1) / SP_WARPS);
     if (g.dtype == OMNI_DTYPE_FP32)
         attention_rows_kernel<float><<<grid, SP_WARPS * 32, 0, st>>>(
             (const float*)q, t, g.h_q, g.h_kv, g.d, (const float*)k_hist, (const float*)v_hist, n_hist_dev, n_hist_max,
-            (const float*)k_chunk, (const float*)v_chunk, scale, o_out, out_dtype, lse_out, ctx->status_dev);
+            (const float*)k_chunk, (const float*)v_chunk, scale, o_out, out_dtype, lse_out, ctx->status_dev, hist_mask);
     else
         attention_rows_kernel<__nv_bfloat16><<<grid, SP_WARPS * 32, 0, st>>>(
             (const __nv_bfloat16*)q, t, g.h_q, g.h_kv, g.d, (const __nv_bfloat16*)k_hist, (const __nv_bfloat16*)v_hist,
             n_hist_dev, n_hist_max, (const __nv_bfloat16*)k_chunk, (const __nv_bfloat16*)v_chunk, scale, o_out,
-            out_dtype, lse_out, ctx->status_dev);
+            out_dtype, lse_out, ctx->status_dev, hist_mask);
     OMNI_CHECK_LAUNCH(ctx, "attention_rows_kernel");
     return OMNI_OK;
 }

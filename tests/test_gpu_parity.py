@@ -634,3 +634,72 @@ def test_chunk_step_with_observation_window(H, ob, cfg2):
 def dataclasses_replace_q(w, W):
     import dataclasses
     return dataclasses.replace(w, q=np.ascontiguousarray(w.q[-W:]))
+
+
+# ------------------------------------------------------------------ attention over a history with holes
+@pytest.mark.parametrize("t,n_hist,h_q,h_kv,pattern", [
+    (128, 1000, 8, 2, "random50"),      # holes in every block
+    (200, 3000, 8, 2, "blocks"),        # whole blocks dead (skipped), others partly live
+    (77, 517, 4, 1, "random10"),        # sparse, ragged tail
+    (64, 2048, 4, 2, "all_dead"),       # the history contributes nothing
+    (64, 1300, 4, 2, "all_live"),       # equals the dense call
+    (1, 4000, 32, 8, "random50"),       # decode over holes (GQA-packed tile)
+    (690, 16384, 32, 8, "sinks"),       # config-2 sizes: kept units whole, others reduced to short prefixes
+])
+def test_attention_masked_tensor_core(H, ob, t, n_hist, h_q, h_kv, pattern):
+    rng = np.random.default_rng(t + n_hist)
+    units = wl.make_units([(n_hist, 0, 0)], group_of_first=None)
+    chunk_units = wl.make_units([(t, 0, 1)], group_of_first=None)
+    q, kh, vh, kc, vc = wl.random_layer_inputs(rng, units, chunk_units, h_q, h_kv, 128, "bf16")
+    if pattern.startswith("random"):
+        keep = (rng.random(n_hist) < int(pattern[6:]) / 100.0).astype(np.uint8)
+    elif pattern == "blocks":
+        keep = np.repeat((rng.random((n_hist + 127) // 128) < 0.5), 128)[:n_hist].astype(np.uint8)
+        keep &= (rng.random(n_hist) < 0.8).astype(np.uint8)
+        keep[128:256] = 0
+    elif pattern == "all_dead":
+        keep = np.zeros(n_hist, np.uint8)
+    elif pattern == "all_live":
+        keep = np.ones(n_hist, np.uint8)
+    else:                                                    # 'sinks'
+        keep = np.zeros(n_hist, np.uint8)
+        for s0 in range(0, n_hist, 690):
+            keep[s0:s0 + (690 if rng.random() < 0.2 else 24)] = 1
+    w = wl.Workload("m", h_q, h_kv, 128, "bf16", units, chunk_units, 1, 64, 1, q=q, k_hist=kh, v_hist=vh, k_chunk=kc, v_chunk=vc)
+    ctx = ob.Context(h_q, h_kv, 128, "bf16", n_hist + 300, 8, t)
+    pad = 200
+    khd = torch.full((n_hist + pad, h_kv, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    vhd = torch.full((n_hist + pad, h_kv, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    khd[:n_hist], vhd[:n_hist] = ob.to_device(kh, "bf16"), ob.to_device(vh, "bf16")
+    mask = torch.full((n_hist + pad + 16,), 1, dtype=torch.uint8, device="cuda")        # stale ones beyond the span
+    mask[:n_hist] = torch.from_numpy(keep).cuda()
+    o = torch.full((t, h_q, 128), float("nan"), dtype=torch.float32, device="cuda")
+    lse = torch.full((t, h_q), float("nan"), dtype=torch.float32, device="cuda")
+    ctx.chunk_attention_masked(ob.to_device(q, "bf16"), t, khd, vhd, mask, H.i32(n_hist), n_hist + pad, ob.to_device(kc, "bf16"),
+                               ob.to_device(vc, "bf16"), 0.0, o, ob.DTYPE_FP32, lse)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    o_ref, lse_ref = oc.chunk_attention_masked(q, kh, vh, keep, kc, vc)
+    _check_attention(o.cpu().numpy(), lse.cpu().numpy(), o_ref, lse_ref)
+    if pattern == "all_live":
+        o2, _ = H.gpu_attention(ctx, w, khd, vhd, n_hist, n_hist_max=n_hist + pad)
+        assert np.array_equal(o2, o.cpu().numpy())
+    ctx.close()
+
+
+def test_attention_masked_cuda_cores(H, ob):
+    w = wl.tiny()
+    rng = np.random.default_rng(77)
+    keep = (rng.random(w.n_hist) < 0.4).astype(np.uint8)
+    ctx = H.make_ctx(w)
+    mask = torch.zeros((w.n_hist + 16,), dtype=torch.uint8, device="cuda")
+    mask[:w.n_hist] = torch.from_numpy(keep).cuda()
+    o = torch.zeros((w.t, w.h_q, w.d), dtype=torch.float32, device="cuda")
+    ctx.chunk_attention_masked(ob.to_device(w.q, "fp32"), w.t, ob.to_device(w.k_hist, "fp32"), ob.to_device(w.v_hist, "fp32"), mask,
+                               None, w.n_hist, ob.to_device(w.k_chunk, "fp32"), ob.to_device(w.v_chunk, "fp32"), 0.0, o,
+                               ob.DTYPE_FP32)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    o_ref, _ = oc.chunk_attention_masked(w.q, w.k_hist, w.v_hist, keep, w.k_chunk, w.v_chunk)
+    _check_attention(o.cpu().numpy(), None, o_ref, None)
+    ctx.close()
