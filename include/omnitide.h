@@ -234,6 +234,22 @@ omni_status omnipage_compact_units(omnitide_ctx* ctx, void* stream,
                                    int32_t* slot_map_out, omni_compact_info* info_out, uint8_t* page_class_out);
 
 /*
+ * (next row: selective migration, ordered-suffix mode; Section 6.2 "Checking layout improvement")  The mode the paper
+ * uses on CUDA, where attention traverses the physical span: scan backward from the end of the span for the smallest
+ * page-aligned suffix whose packing shortens the page-rounded span by at least min_pages_saved pages; pack only the
+ * live rows of that suffix, in order, to its start; every slot before it keeps its content and its holes.  If no
+ * suffix qualifies nothing moves.  In place (moves go through context scratch: reads of all sources precede all
+ * writes).  keep_mask [dev, in/out] and *s_span_dev [dev, in/out] describe the layout before and after; the result is
+ * what omnitide_chunk_attention_masked takes.  slot_map_out [dev, nullable] s_span_max int32: new slot of every live
+ * row, -1 for dead ones.  info_out [dev, nullable]: n_kept = live rows, span_pages = pages of the new span,
+ * rows_moved, part_begin = {suffix start or -1, new span, pages saved, old span}.  page_size a multiple of 16.
+ */
+omni_status omnipage_migrate_suffix(omnitide_ctx* ctx, void* stream, void* k_cache, void* v_cache,
+                                    uint8_t* keep_mask, int32_t* s_span_dev, int32_t s_span_max,
+                                    int32_t page_size, int32_t min_pages_saved,
+                                    int32_t* slot_map_out, omni_compact_info* info_out);
+
+/*
  * (next row: RoPE position re-index fused into the gather; Section 5.2 "the runtime applies the corresponding RoPE
  * adjustment to cached keys")  omnipage_compact_units with every moved K row re-rotated to its new position while it
  * passes through shared memory.  Positions are slot indices (the cache is dense before and after the pack), so the

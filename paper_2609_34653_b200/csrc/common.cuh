@@ -25,6 +25,7 @@ struct omnitide_ctx {
     void* inplace_k;              // staging for in-place compaction, allocated on first use
     void* inplace_v;
     size_t inplace_rows;
+    int32_t* mig_plan;            // [8] plan of the ordered-suffix migration, allocated on first use
     unsigned long long* cp_words; // [SMs] per-CTA count words of the compaction kernel, tagged with cp_epoch
     uint32_t cp_epoch;            // launches of the compaction kernel on this context so far
     // work buffers of omnitide_chunk_step

@@ -86,6 +86,9 @@ struct CompactArgs {
     int max_chunks;    // capacity of the chunk-prefix array
     int n_slots;       // row buffers per warp for the bulk-copy path (0: move rows with vector loads/stores)
     int part_groups;   // 512-byte mask groups per CTA
+    // ordered-suffix migration: the span that is packed starts at slot *span_off_dev (a multiple of 16; negative: nothing
+    // to pack); mask, sources and slot map are taken from there and slot-map values count from there too
+    const int32_t* span_off_dev;
     unsigned long long* words;   // [0]: arrival counter (low half, never reset); [1 + i]: (epoch << 32) | retained count of part i
     uint32_t epoch;
 };
@@ -283,7 +286,18 @@ __device__ __forceinline__ uint4 mask_at(const uint8_t* mask, int pos, int s) {
 // The mask is cut into gridDim.x parts of `part_groups` groups of 512 bytes; CTA i counts part i alone and
 // publishes the count in words[i] tagged with the epoch of this launch; every CTA then gathers all the
 // counts (the only cross-CTA step: all CTAs are resident, one per SM, and the wait is bounded).
-__global__ void __launch_bounds__(CP_THREADS, 1) compact_pack_kernel(const CompactArgs a) {
+__global__ void __launch_bounds__(CP_THREADS, 1) compact_pack_kernel(const CompactArgs a_in) {
+    CompactArgs a = a_in;
+    int span_off = 0;
+    if (a_in.span_off_dev) {
+        const int s_all = a_in.s_span_dev ? __ldg(a_in.s_span_dev) : a_in.s_span_max;
+        span_off = __ldg(a_in.span_off_dev);
+        if (span_off < 0 || span_off > s_all) span_off = max(0, min(s_all, a_in.s_span_max));   // nothing to pack: an empty span
+        a.mask += span_off;
+        if (a.k_src) { a.k_src += (size_t)span_off * a.row_bytes; a.v_src += (size_t)span_off * a.row_bytes; }
+        if (a.slot_map) a.slot_map += span_off;
+        a.s_span_max -= span_off;
+    }
     extern __shared__ __align__(128) int smem_i[];
     int* prefix = smem_i;                                   // [max_chunks]: part counts, then their exclusive scan
     int* src_list = smem_i + a.max_chunks;                  // [rows_cap]
@@ -303,7 +317,7 @@ __global__ void __launch_bounds__(CP_THREADS, 1) compact_pack_kernel(const Compa
     const int wg0 = wid * gpw, wg1 = min(a.part_groups, wg0 + gpw);   // this warp's groups of the part
     uint4 mv = make_uint4(0, 0, 0, 0);                                // its first group stays in registers
     if (wg0 < wg1 && my_base + wg0 * 512 + lane * 16 < a.s_span_max) mv = ld_mask(a.mask, (my_base + wg0 * 512) / 16 + lane);
-    int s = a.s_span_dev ? __ldg(a.s_span_dev) : a.s_span_max;
+    int s = a.s_span_dev ? __ldg(a.s_span_dev) - span_off : a.s_span_max;
     int nu = 0, u_len = 0, u_group = -1;
     if (a.units_kept) {
         nu = a.n_units_kept_dev ? __ldg(a.n_units_kept_dev) : a.n_units_max;
@@ -446,7 +460,7 @@ __global__ void __launch_bounds__(CP_THREADS, 1) compact_pack_kernel(const Compa
             const int base = my_base + g * 512;
             if (base >= s) break;
             const uint4 v = g == wg0 ? mv : mask_at(a.mask, base + lane * 16, s);
-            emit_slot_map(v, base, run, lane, s, a.slot_map);
+            emit_slot_map(v, base, run + span_off, lane, s, a.slot_map);
             run += __reduce_add_sync(0xffffffffu, count_kept(v));
         }
     }
@@ -842,6 +856,78 @@ __global__ void append_units_kernel(omni_unit* units, const int32_t* n_units_dev
 
 }  // namespace
 
+// ---------------------------------------------------------------------------------------------------
+// Ordered-suffix migration (Section 6.2): plan on one CTA, pack the chosen suffix with the mask kernel above
+// (through staging: a move may land on a source row of another move), then rewrite the mask of the suffix.
+// plan[0] = first slot of the suffix the pack kernel works on (the span itself when nothing qualifies: an empty
+// suffix), plan[1] = suffix start or -1, plan[2] = span after the move, plan[3] = span before, plan[4] = live slots.
+__global__ void __launch_bounds__(CP_THREADS, 1) suffix_plan_kernel(const uint8_t* __restrict__ mask, const int32_t* s_span_dev,
+                                                                    int s_span_max, int page, int theta, int32_t* plan,
+                                                                    int32_t* status) {
+    extern __shared__ int pg_cnt[];                          // [pages + 1]: live slots per page, reversed, then their scan
+    __shared__ int warp_tot[CP_WARPS + 1];
+    __shared__ int s_best;
+    const int tid = threadIdx.x;
+    int S = s_span_dev ? *s_span_dev : s_span_max;
+    if (S < 0 || S > s_span_max) {
+        if (tid == 0) atomicOr(status, OMNI_DEV_BAD_COUNT);
+        S = max(0, min(S, s_span_max));
+    }
+    const int n_pages = (S + page - 1) / page;
+    if (tid == 0) s_best = -1;
+    for (int pg = tid; pg < n_pages; pg += CP_THREADS) {
+        int cnt = 0;
+        const int hi = min(S, (pg + 1) * page);
+        for (int pos = pg * page; pos < hi; pos += 16) {
+            const uint4 v = clip_vec(ld_mask(mask, pos >> 4), hi - pos);
+            cnt += count_kept(v);
+        }
+        pg_cnt[n_pages - 1 - pg] = cnt;                      // reversed: a prefix sum becomes a suffix sum
+    }
+    __syncthreads();
+    const int total_live = block_excl_scan(pg_cnt, n_pages, warp_tot);   // pg_cnt[j] = live slots in the last j pages
+    // suffix that starts at page i holds pg_cnt[n_pages - i] live slots
+    for (int i = tid; i < n_pages; i += CP_THREADS) {
+        const int live = pg_cnt[n_pages - i];
+        const int new_span = i * page + live;
+        if (n_pages - (new_span + page - 1) / page >= theta) atomicMax(&s_best, i);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        const int i = s_best;
+        plan[0] = i >= 0 ? i * page : S;
+        plan[1] = i >= 0 ? i * page : -1;
+        plan[2] = i >= 0 ? i * page + pg_cnt[n_pages - i] : S;
+        plan[3] = S;
+        plan[4] = total_live;
+    }
+}
+
+__global__ void __launch_bounds__(256) suffix_finish_kernel(uint8_t* mask, int32_t* s_span_dev, int page, const int32_t* plan,
+                                                            const omni_compact_info* pack_info, int32_t* slot_map,
+                                                            omni_compact_info* info) {
+    const int start = plan[1], new_span = plan[2], S = plan[3];
+    const int gtid = blockIdx.x * blockDim.x + threadIdx.x, gsz = gridDim.x * blockDim.x;
+    const int keep_from = start >= 0 ? start : S;            // slots before it keep their place and their holes
+    if (slot_map)
+        for (int sl = gtid; sl < keep_from; sl += gsz) slot_map[sl] = mask[sl] ? sl : -1;
+    if (start >= 0)
+        for (int sl = start + gtid; sl < S; sl += gsz) mask[sl] = sl < new_span ? 1 : 0;
+    if (gtid == 0) {
+        if (start >= 0 && s_span_dev) *s_span_dev = new_span;
+        if (info) {
+            info->n_kept = plan[4];
+            info->span_pages = (new_span + page - 1) / page;
+            info->rows_moved = start >= 0 ? pack_info->rows_moved : 0;
+            info->part_begin[0] = start;
+            info->part_begin[1] = new_span;
+            info->part_begin[2] = (S + page - 1) / page - (new_span + page - 1) / page;
+            info->part_begin[3] = S;
+            info->reserved = 0;
+        }
+    }
+}
+
 // Staging rows of the in-place mode, allocated on the first in-place call on a context (synchronous).
 static omni_status omni_inplace_staging(omnitide_ctx* ctx) {
     if (ctx->inplace_rows >= (size_t)ctx->g.s_cap) return OMNI_OK;
@@ -855,7 +941,7 @@ static omni_status omni_inplace_staging(omnitide_ctx* ctx) {
     return OMNI_OK;
 }
 
-extern "C" omni_status omnipage_compact(omnitide_ctx* ctx, void* stream, const void* k_src, const void* v_src,
+static omni_status compact_pack_impl(const int32_t* span_off_dev, omnitide_ctx* ctx, void* stream, const void* k_src, const void* v_src,
                                         void* k_dst, void* v_dst, const uint8_t* keep_mask,
                                         const int32_t* s_span_dev, int32_t s_span_max, int32_t page_size, int32_t mode,
                                         const omni_unit* units_kept, const int32_t* n_units_kept_dev,
@@ -901,6 +987,7 @@ extern "C" omni_status omnipage_compact(omnitide_ctx* ctx, void* stream, const v
     a.part_groups = std::max(1, (n_grp + grid - 1) / grid);
     ++ctx->cp_epoch;                                         // wraps together with the 32-bit arrival counter
     a.words = ctx->cp_words;
+    a.span_off_dev = span_off_dev;
     a.epoch = ctx->cp_epoch;
     const size_t smem_lists = (size_t)(a.max_chunks + a.rows_cap) * sizeof(int);
     const size_t budget = 200 * 1024;
@@ -929,7 +1016,7 @@ extern "C" omni_status omnipage_compact(omnitide_ctx* ctx, void* stream, const v
         if (!info_out) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "compact: in-place mode needs info_out");
         copy_rows_kernel<<<ctx->sm_count * 4, 256, 0, st>>>(
             static_cast<const char*>(kd), static_cast<const char*>(vd), static_cast<char*>(k_dst),
-            static_cast<char*>(v_dst), &info_out->n_kept, s_span_max, nullptr, ctx->g.s_cap, (int)ctx->row_bytes,
+            static_cast<char*>(v_dst), &info_out->n_kept, s_span_max, span_off_dev, ctx->g.s_cap, (int)ctx->row_bytes,
             ctx->status_dev);
         OMNI_CHECK_LAUNCH(ctx, "copy_rows_kernel");
     }
@@ -1008,6 +1095,47 @@ static omni_status compact_units_impl(const omni_rope_params* rope, omnitide_ctx
             ctx->status_dev);
         OMNI_CHECK_LAUNCH(ctx, "copy_rows_kernel");
     }
+    return OMNI_OK;
+}
+
+extern "C" omni_status omnipage_compact(omnitide_ctx* ctx, void* stream, const void* k_src, const void* v_src,
+                                        void* k_dst, void* v_dst, const uint8_t* keep_mask,
+                                        const int32_t* s_span_dev, int32_t s_span_max, int32_t page_size, int32_t mode,
+                                        const omni_unit* units_kept, const int32_t* n_units_kept_dev,
+                                        int32_t n_units_max, int32_t* slot_map_out, omni_compact_info* info_out,
+                                        uint8_t* page_class_out) {
+    return compact_pack_impl(nullptr, ctx, stream, k_src, v_src, k_dst, v_dst, keep_mask, s_span_dev, s_span_max, page_size,
+                             mode, units_kept, n_units_kept_dev, n_units_max, slot_map_out, info_out, page_class_out);
+}
+
+extern "C" omni_status omnipage_migrate_suffix(omnitide_ctx* ctx, void* stream, void* k_cache, void* v_cache,
+                                               uint8_t* keep_mask, int32_t* s_span_dev, int32_t s_span_max,
+                                               int32_t page_size, int32_t min_pages_saved, int32_t* slot_map_out,
+                                               omni_compact_info* info_out) {
+    if (!ctx) return OMNI_ERR_INVALID_ARG;
+    if (!k_cache || !v_cache || !keep_mask || !s_span_dev || s_span_max <= 0)
+        OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "migrate_suffix: null pointer or empty span");
+    if (page_size <= 0 || (page_size & 15)) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "migrate_suffix: page size must be a multiple of 16");
+    if (min_pages_saved < 1) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "migrate_suffix: the threshold is at least one page");
+    if (s_span_max > ctx->g.s_cap) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "migrate_suffix: s_span_max %d > s_cap %d", s_span_max, ctx->g.s_cap);
+    if (!omni_aligned16(keep_mask)) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "migrate_suffix: the mask must be 16-byte aligned");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!ctx->mig_plan) OMNI_CUDA(ctx, cudaMalloc(&ctx->mig_plan, 8 * sizeof(int32_t)));
+    const size_t plan_smem = ((size_t)(s_span_max + page_size - 1) / page_size + 2) * sizeof(int);
+    if (plan_smem > 200 * 1024) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "migrate_suffix: too many pages for one launch");
+    if (plan_smem > 48 * 1024)
+        OMNI_CUDA(ctx, cudaFuncSetAttribute(suffix_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan_smem));
+    suffix_plan_kernel<<<1, CP_THREADS, plan_smem, st>>>(keep_mask, s_span_dev, s_span_max, page_size, min_pages_saved,
+                                                         ctx->mig_plan, ctx->status_dev);
+    OMNI_CHECK_LAUNCH(ctx, "suffix_plan_kernel");
+    // the pack of the suffix, in place through staging; its slot map counts from the start of the suffix on
+    const omni_status ps = compact_pack_impl(ctx->mig_plan, ctx, stream, k_cache, v_cache, k_cache, v_cache, keep_mask,
+                                             s_span_dev, s_span_max, page_size, OMNI_COMPACT_PACK, nullptr, nullptr, 1,
+                                             slot_map_out, ctx->ws_info, nullptr);
+    if (ps) return ps;
+    suffix_finish_kernel<<<std::min(ctx->sm_count, 64), 256, 0, st>>>(keep_mask, s_span_dev, page_size, ctx->mig_plan,
+                                                                       ctx->ws_info, slot_map_out, info_out);
+    OMNI_CHECK_LAUNCH(ctx, "suffix_finish_kernel");
     return OMNI_OK;
 }
 

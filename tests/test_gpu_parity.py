@@ -703,3 +703,95 @@ def test_attention_masked_cuda_cores(H, ob):
     o_ref, _ = oc.chunk_attention_masked(w.q, w.k_hist, w.v_hist, keep, w.k_chunk, w.v_chunk)
     _check_attention(o.cpu().numpy(), None, o_ref, None)
     ctx.close()
+
+
+# ------------------------------------------------------------------ ordered-suffix migration
+@pytest.mark.parametrize("S,page,theta,pattern,seed", [
+    (1000, 16, 1, "tail_sparse", 0),
+    (5000, 64, 2, "tail_sparse", 1),
+    (16384, 64, 4, "sinks", 2),
+    (3000, 256, 1, "random", 3),
+    (2048, 64, 1, "dense", 4),          # nothing qualifies: nothing moves
+    (80000, 64, 8, "sinks", 5),
+    (777, 16, 3, "random", 6),
+])
+def test_migrate_suffix_bit_exact(H, ob, S, page, theta, pattern, seed):
+    """omnipage_migrate_suffix equals the oracle: chosen suffix, new mask and span, slot map, and every row of the
+    cache up to the new span, bit for bit; then attention over the migrated layout is unchanged."""
+    rng = np.random.default_rng(300 + seed)
+    if pattern == "tail_sparse":
+        keep = np.ones(S, np.uint8)
+        keep[S // 2:] = (rng.random(S - S // 2) < 0.3).astype(np.uint8)
+    elif pattern == "sinks":
+        keep = np.zeros(S, np.uint8)
+        for s0 in range(0, S, 690):
+            keep[s0:s0 + (690 if rng.random() < 0.3 else 24)] = 1
+        keep[:16] = 1
+    elif pattern == "random":
+        keep = (rng.random(S) < 0.5).astype(np.uint8)
+    else:
+        keep = np.ones(S, np.uint8)
+    rowshape = (2, 128)
+    raw = rng.integers(0, 256, size=(2, S, rowshape[0] * rowshape[1] * 2), dtype=np.uint8)
+    k = torch.from_numpy(raw[0]).cuda().view(torch.bfloat16).view(S, *rowshape).contiguous()
+    v = torch.from_numpy(raw[1]).cuda().view(torch.bfloat16).view(S, *rowshape).contiguous()
+    exp = oc.migrate_suffix(raw[0], raw[1], keep, page, theta)
+    ctx = ob.Context(8, 2, 128, "bf16", S + 64, 8, 16)
+    mask = torch.zeros((S + 48,), dtype=torch.uint8, device="cuda")
+    mask[:S] = torch.from_numpy(keep).cuda()
+    mask[S:S + 40] = 1                                        # stale bytes beyond the span
+    span = H.i32(S)
+    slot_map = torch.full((S + 48,), -5, dtype=torch.int32, device="cuda")
+    info = torch.full((8,), -5, dtype=torch.int32, device="cuda")
+    ctx.migrate_suffix(k, v, mask, span, S + 40, page, theta, slot_map, info)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    got = ob.info_to_dict(info)
+    ns = exp["new_span"]
+    assert got["part_begin"] == [exp["start"], ns, exp["pages_saved"], S]
+    assert got["n_kept"] == int(keep.sum()) and got["rows_moved"] == exp["rows_moved"] and int(span.item()) == ns
+    assert np.array_equal(mask[:S].cpu().numpy(), exp["keep_mask"])
+    assert np.array_equal(slot_map[:S].cpu().numpy(), exp["slot_map"])
+    assert np.array_equal(H.bytes_of(k[:ns]).reshape(ns, -1), exp["k"][:ns])
+    assert np.array_equal(H.bytes_of(v[:ns]).reshape(ns, -1), exp["v"][:ns])
+    if pattern == "dense":
+        assert exp["start"] == -1 and got["rows_moved"] == 0
+    else:
+        assert exp["start"] >= 0
+    ctx.close()
+
+
+def test_native_suffix_eager_layouts_attend_alike(H, ob, cfg2):
+    """The three layouts of the paper's ablation (native holes, ordered-suffix migration, eager pack) present the same
+    live rows: attention over each of them matches the oracle, and the spans shrink in that order."""
+    w = cfg2
+    rng = np.random.default_rng(31)
+    N, T = w.n_hist, w.t
+    plan = oc.plan_structural(w.units, 0, 6000, 2, (24, 8, 0), 64)
+    keep = plan["keep_mask"]
+    o_ref, _ = oc.chunk_attention_masked(w.q, w.k_hist, w.v_hist, keep, w.k_chunk, w.v_chunk)
+    ctx = H.make_ctx(w)
+    q, kc, vc = (ob.to_device(a, "bf16") for a in (w.q, w.k_chunk, w.v_chunk))
+    k, v = ob.to_device(w.k_hist, "bf16").clone(), ob.to_device(w.v_hist, "bf16").clone()
+    mask = torch.zeros((N + 16,), dtype=torch.uint8, device="cuda")
+    mask[:N] = torch.from_numpy(keep).cuda()
+    span = H.i32(N)
+    o = torch.zeros((T, w.h_q, w.d), dtype=torch.float32, device="cuda")
+    # native: holes left in place
+    ctx.chunk_attention_masked(q, T, k, v, mask, span, N, kc, vc, 0.0, o, ob.DTYPE_FP32)
+    torch.cuda.synchronize()
+    _check_attention(o.cpu().numpy(), None, o_ref, None)
+    # ordered suffix
+    info = torch.zeros((8,), dtype=torch.int32, device="cuda")
+    ctx.migrate_suffix(k, v, mask, span, N, w.page_size, 4, None, info)
+    ctx.chunk_attention_masked(q, T, k, v, mask, span, N, kc, vc, 0.0, o, ob.DTYPE_FP32)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    _check_attention(o.cpu().numpy(), None, o_ref, None)
+    span_suffix = int(span.item())
+    # eager
+    got = H.gpu_compact(ctx, ob.to_device(w.k_hist, "bf16"), ob.to_device(w.v_hist, "bf16"), keep, w.page_size)
+    o3, _ = H.gpu_attention(ctx, w, got["k"], got["v"], got["n_kept"], n_hist_max=N, want_lse=False)
+    _check_attention(o3, None, o_ref, None)
+    assert got["n_kept"] <= span_suffix < N
+    ctx.close()
