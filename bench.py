@@ -265,6 +265,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--mask-compaction", action="store_true",
                     help="time omnipage_compact (token keep mask + slot map) instead of the unit-granular entry point")
+    ap.add_argument("--no-ablation", dest="ablation", action="store_false",
+                    help="skip the native / ordered-suffix / eager layout ablation")
     ap.add_argument("--batch-layers", type=int, default=36,
                     help="layers packed by one launch of the cross-layer batched compaction (0: skip it)")
     ap.add_argument("--loop-chunks", type=int, default=40, help="chunks of the 36-layer stream loop (0: skip it)")
@@ -503,6 +505,61 @@ def main():
         "frac": work["compact_bytes"] / (rope_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "ms": rope_ms,
         "entry": "omnipage_compact_units_rope",
         "note": "same bytes as compact; every moved K row is re-rotated to its new position in shared memory"}
+
+    # ---- the paper's three-way layout ablation on this workload, with its own structural plan (sink prefixes):
+    # native (holes left in place), ordered-suffix migration, eager pack; each followed by the chunk attention
+    abl = None
+    if args.ablation:
+        sp = ob.structural_params(0, w.budget, 2, (32, 8, 0), 256)
+        a_keep = torch.zeros(u_cap + 16, dtype=torch.uint8, device="cuda")
+        a_klen = torch.zeros(u_cap + 16, dtype=torch.int32, device="cuda")
+        a_mask = torch.zeros(s_cap + 16, dtype=torch.uint8, device="cuda")
+        a_mask0 = torch.zeros_like(a_mask)
+        a_units = torch.zeros((u_cap, 6), dtype=torch.int32, device="cuda")
+        a_nk, a_nu = cnt(0), cnt(0)
+        ctx.plan_structural(units_in, n_units_dev, U, sp, a_keep, a_klen, a_mask0, N, a_nk, a_units, a_nu)
+        span_dev = cnt(N)
+        a_info = torch.zeros(8, dtype=torch.int32, device="cuda")
+        ev = lambda: torch.cuda.Event(enable_timing=True)
+        reps = max(5, min(args.steps, 20))
+        res = {"native": [], "suffix_migrate": [], "suffix_attention": [], "eager_pack": [], "eager_attention": []}
+        spans = {}
+        for i in range(2 + reps):
+            s_ = sets[i % R]
+            k_w, v_w = s_["k_out"], s_["v_out"]              # scratch copies the suffix mode may rewrite in place
+            k_w.copy_(s_["k_in"]); v_w.copy_(s_["v_in"])
+            a_mask.copy_(a_mask0); span_dev.fill_(N)
+            e = [ev() for _ in range(8)]
+            e[0].record()
+            ctx.chunk_attention_masked(s_["q"], T, k_w, v_w, a_mask, span_dev, N, s_["kc"], s_["vc"], 0.0, s_["o"], ob.DTYPE_FP32)
+            e[1].record()
+            ctx.migrate_suffix(k_w, v_w, a_mask, span_dev, N, w.page_size, 8, None, a_info)
+            e[2].record()
+            ctx.chunk_attention_masked(s_["q"], T, k_w, v_w, a_mask, span_dev, N, s_["kc"], s_["vc"], 0.0, s_["o"], ob.DTYPE_FP32)
+            e[3].record()
+            torch.cuda.synchronize()
+            spans["suffix"] = int(span_dev.item())
+            e[4].record()
+            ctx.compact_units(s_["k_in"], s_["v_in"], k_w, v_w, units_in, n_units_dev, U, a_keep, N, w.page_size, a_units, a_nu,
+                              None, info, None, unit_kept_len=a_klen)
+            e[5].record()
+            ctx.chunk_attention(s_["q"], T, k_w, v_w, a_nk, N, s_["kc"], s_["vc"], 0.0, s_["o"], ob.DTYPE_FP32)
+            e[6].record()
+            torch.cuda.synchronize()
+            if i >= 2:
+                for name, (x, y) in zip(res, ((0, 1), (1, 2), (2, 3), (4, 5), (5, 6))):
+                    res[name].append(e[x].elapsed_time(e[y]))
+        assert ctx.poll_status() == 0, "device status word not clean after the layout ablation"
+        live = int(a_nk.item())
+        abl = {k_: float(np.mean(v_)) for k_, v_ in res.items()}
+        abl = {"live_rows": live, "span_native": N, "span_suffix": spans["suffix"],
+               "span_eager": ((live + w.page_size - 1) // w.page_size) * w.page_size,
+               "native_ms": abl["native"], "suffix_ms": abl["suffix_migrate"] + abl["suffix_attention"],
+               "suffix_migrate_ms": abl["suffix_migrate"], "suffix_attention_ms": abl["suffix_attention"],
+               "eager_ms": abl["eager_pack"] + abl["eager_attention"], "eager_pack_ms": abl["eager_pack"],
+               "eager_attention_ms": abl["eager_attention"],
+               "note": "maintenance + chunk attention per layout after one structural retention round (suffix threshold 8 pages)"}
+        line["layout_ablation"] = abl
 
     # ---- cross-layer batched compaction: the same unit decision applied to the K/V caches of 36 layers in one launch
     batched = None
