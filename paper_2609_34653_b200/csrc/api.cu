@@ -19,7 +19,7 @@ void free_all(omnitide_ctx* c) {
     void* ptrs[] = {c->status_dev, c->score_part, c->score_tile_mass, c->score_mass64, c->inplace_k, c->inplace_v,
                     c->ws_scores, c->ws_unit_keep, c->ws_kept_len, c->ws_keep_mask, c->ws_slot_map, c->ws_counts, c->ws_info, c->st_q,
                     c->st_k, c->st_v, c->st_o, c->st_units, c->attn_part_o, c->attn_part_ml, c->cp_words, c->attn_live_idx, c->attn_live_mask,
-                    c->attn_n_live, c->mig_plan};
+                    c->attn_n_live, c->mig_plan, c->dec_counter};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
@@ -62,6 +62,8 @@ extern "C" omni_status omnitide_create(omnitide_ctx** ctx_out, const omni_geomet
     ok &= alloc(&c->attn_live_idx, (size_t)g->s_cap / 128 + 2) == cudaSuccess;
     ok &= alloc(&c->attn_live_mask, (size_t)g->s_cap / 128 + 2) == cudaSuccess;
     ok &= alloc(&c->attn_n_live, (size_t)1) == cudaSuccess;
+    ok &= alloc(&c->dec_counter, (size_t)g->h_kv) == cudaSuccess;
+    ok = ok && cudaMemset(c->dec_counter, 0, sizeof(int32_t) * (size_t)g->h_kv) == cudaSuccess;
     ok &= alloc(&c->cp_words, (size_t)c->sm_count + 1) == cudaSuccess;
     ok = ok && cudaMemset(c->cp_words, 0, ((size_t)c->sm_count + 1) * sizeof(unsigned long long)) == cudaSuccess;
     ok &= alloc(&c->ws_scores, (size_t)g->u_cap) == cudaSuccess;
@@ -164,9 +166,16 @@ static omni_status chunk_attention_impl(const uint8_t* hist_mask, omnitide_ctx* 
         OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "attention: pointers must be 16-byte aligned");
     if (scale <= 0.f) scale = 1.0f / sqrtf((float)ctx->g.d);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (tc_geometry(ctx))
+    if (tc_geometry(ctx)) {
+        // one query and a dense history: the split-KV decode kernel (HBM-bound, no tensor-core work to do)
+        if (t == 1 && !hist_mask) {
+            const omni_status ds = omni_attention_decode(ctx, st, q, k_hist, v_hist, n_hist_dev, n_hist_max, k_chunk, v_chunk,
+                                                         scale, o_out, out_dtype, lse_out);
+            if (ds != OMNI_ERR_UNSUPPORTED) return ds;
+        }
         return omni_attention_tc(ctx, st, q, t, k_hist, v_hist, n_hist_dev, n_hist_max, k_chunk, v_chunk, scale, o_out,
                                  out_dtype, lse_out, hist_mask);
+    }
     return omni_attention_simple(ctx, st, q, t, k_hist, v_hist, n_hist_dev, n_hist_max, k_chunk, v_chunk, scale, o_out,
                                  out_dtype, lse_out, hist_mask);
 }

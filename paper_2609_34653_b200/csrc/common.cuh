@@ -47,6 +47,7 @@ struct omnitide_ctx {
     int32_t* attn_live_idx;       // [s_cap / 128 + 2] blocks of the history that hold a live slot (masked attention)
     uint4* attn_live_mask;        // [s_cap / 128 + 2] their 128 live bits
     int32_t* attn_n_live;
+    int32_t* dec_counter;         // [h_kv] arrival counters of the decode kernel, zero between launches
     bool attn_attr_set;           // the attention kernel's shared-memory limit has been raised on this device
     // -----------------------------------------------------------------------------------
     void* encode_tiled;           // cuTensorMapEncodeTiled, resolved through the runtime
@@ -84,6 +85,9 @@ omni_status omni_attention_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q,
                               const void* v_hist, const int32_t* n_hist_dev, int n_hist_max, const void* k_chunk,
                               const void* v_chunk, float scale, void* o_out, int out_dtype, float* lse_out,
                               const uint8_t* hist_mask);
+omni_status omni_attention_decode(omnitide_ctx* ctx, cudaStream_t st, const void* q, const void* k_hist, const void* v_hist,
+                                  const int32_t* n_hist_dev, int n_hist_max, const void* k_chunk, const void* v_chunk,
+                                  float scale, void* o_out, int out_dtype, float* lse_out);
 omni_status omni_score_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q, int t, const void* k_cache,
                           const int32_t* n_hist_dev, int n_hist_max, const omni_unit* units,
                           const int32_t* n_units_dev, int n_units_max, const float* w, float scale,

@@ -795,3 +795,33 @@ def test_native_suffix_eager_layouts_attend_alike(H, ob, cfg2):
     _check_attention(o3, None, o_ref, None)
     assert got["n_kept"] <= span_suffix < N
     ctx.close()
+
+
+@pytest.mark.parametrize("h_q,h_kv", [(32, 8), (8, 1), (64, 8), (8, 8), (4, 2)])
+def test_decode_attention_many_lengths(H, ob, h_q, h_kv):
+    """One token against histories of many lengths (every alignment of the split and batch boundaries), for group
+    sizes 1, 2, 4 and 8, through the split-KV decode kernel; fp32 and bf16 outputs, log-sum-exp."""
+    rng = np.random.default_rng(h_q * 10 + h_kv)
+    n_max = 2600
+    units = wl.make_units([(n_max, 0, 0)], group_of_first=None)
+    chunk_units = wl.make_units([(1, 0, 1)], group_of_first=None)
+    q, kh, vh, kc, vc = wl.random_layer_inputs(rng, units, chunk_units, h_q, h_kv, 128, "bf16")
+    ctx = ob.Context(h_q, h_kv, 128, "bf16", n_max + 64, 8, 4)
+    khd, vhd = ob.to_device(kh, "bf16"), ob.to_device(vh, "bf16")
+    qd, kcd, vcd = ob.to_device(q, "bf16"), ob.to_device(kc, "bf16"), ob.to_device(vc, "bf16")
+    lengths = [0, 1, 2, 15, 16, 17, 63, 64, 65, 127, 128, 129, 500, 1023, 1024, 1025, 2048, 2599, 2600] + \
+        [int(x) for x in rng.integers(1, n_max, size=12)]
+    for n in lengths:
+        o = torch.full((1, h_q, 128), float("nan"), dtype=torch.float32, device="cuda")
+        lse = torch.full((1, h_q), float("nan"), dtype=torch.float32, device="cuda")
+        ctx.chunk_attention(qd, 1, khd, vhd, H.i32(n), n_max, kcd, vcd, 0.0, o, ob.DTYPE_FP32, lse)
+        torch.cuda.synchronize()
+        assert ctx.poll_status() == 0
+        o_ref, lse_ref = oc.chunk_attention(q, kh[:n], vh[:n], kc, vc)
+        _check_attention(o.cpu().numpy(), lse.cpu().numpy(), o_ref, lse_ref)
+    o16 = torch.zeros((1, h_q, 128), dtype=torch.bfloat16, device="cuda")
+    ctx.chunk_attention(qd, 1, khd, vhd, H.i32(777), n_max, kcd, vcd, 0.0, o16, ob.DTYPE_BF16)
+    ctx.chunk_attention(qd, 1, khd, vhd, H.i32(777), n_max, kcd, vcd, 0.0, o, ob.DTYPE_FP32)
+    torch.cuda.synchronize()
+    assert np.array_equal(o16.float().cpu().numpy(), wl.round_to_bf16(o.cpu().numpy()))
+    ctx.close()
