@@ -467,7 +467,7 @@ def main():
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                 "note": "attention FLOPs of the step over the whole host-buffer pass (copies + 5 stages)"},
     }
-    # ---- decode-phase attention: one new token against the compacted history (GQA-packed tile path), cache sets rotated
+    # ---- decode-phase attention: one new token against the compacted history (split-KV decode kernel), cache sets rotated
     d_reps = max(8, min(args.steps, 40))
     devs = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(d_reps)]
     o1 = torch.empty((1, w.h_q, w.d), dtype=torch.float32, device="cuda")
@@ -485,7 +485,7 @@ def main():
     line["kernels"]["decode_attention"] = {
         "bound": "hbm", "achieved": dec_bytes / (dec_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
         "frac": dec_bytes / (dec_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "ms": dec_ms, "bytes": dec_bytes,
-        "note": f"omnitide_chunk_attention with t = 1 over {kept} retained rows (K and V read once per KV group), merge kernel included"}
+        "note": f"omnitide_chunk_attention with t = 1 over {kept} retained rows: split-KV decode kernel, K and V read once per KV group, one launch"}
 
     # ---- the unit-granular pack with the RoPE re-index of the moved keys fused in
     revs = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(d_reps)]
