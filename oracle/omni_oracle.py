@@ -48,6 +48,21 @@ What follows the paper and what does not
                        are readings.  Pinned by brute force over every suffix
                        start and by invariants.  Attention over the resulting
                        layout with holes is attention over the live rows.
+* migrate_class     -- OmniPage's class-aware selective migration (Section 6.2
+                       "Packing scattered entries", "Checking layout
+                       improvement"; classes and promotion of Section 6.1):
+                       candidates (entries kept from partially evicted units,
+                       outside full pages) go, in physical order, to the earliest
+                       empty slot of a page that is empty or of their class; the
+                       plan is simulated and accepted only if the active pages
+                       or the active subblocks decrease; full pages are promoted
+                       to selected-history.  Readings: what "earlier empty slot"
+                       means while the plan is being simulated (vacated slots
+                       count), the mark that makes an entry a candidate, which
+                       full pages are promoted.  PARITY UNPINNED by the paper
+                       (it prints no example); pinned by hand-worked layouts,
+                       an independent set-based replay that checks every move
+                       is to the smallest admissible slot, and invariants.
 * rope_reindex      -- the position shift the runtime applies to cached keys after
                        logical deletion (Section 5.2): a kept token's position
                        drops by the number of deleted tokens before it and its
@@ -469,6 +484,103 @@ def migrate_suffix(k_cache, v_cache, keep_mask, page_size, min_pages_saved=1):
     new_span = start + len(src)
     return dict(start=start, k=k, v=v, keep_mask=new_mask.astype(np.uint8), new_span=new_span,
                 pages_saved=pages(S) - pages(new_span), rows_moved=int((src != dst).sum()), slot_map=slot_map)
+
+
+CLASS_MUST_KEEP, CLASS_SELECTED, CLASS_RECENT = 0, 1, 2      # allocation classes (Section 6.1)
+CLASS_CANDIDATE = 0x80                                       # slot_class bit 7: entry retained from a partially evicted unit
+PAGE_MIXED = 254
+
+
+def migrate_class(k_cache, v_cache, keep_mask, slot_class, page_size, subblock, promote=True):
+    """Class-aware selective migration (Section 6.2, "packing scattered entries" and "checking layout
+    improvement"; the allocation classes are those of Section 6.1).
+
+    keep_mask [S] marks the live slots after the logical deletion; slot_class [S] gives, for a live slot,
+    its allocation class in the low two bits (0 must-keep, 1 selected-history, 2 recent-context) and in
+    bit 7 whether the entry was retained from a partially evicted unit (a candidate).  Pages are P
+    consecutive slots, subblocks B consecutive slots (B divides P).
+
+    Plan.  Candidates are the live slots with bit 7 set whose page is not full when the plan starts (full
+    pages stay in place), visited in ascending physical order.  A candidate at slot s of class c goes to the
+    smallest slot d < s that is empty in the simulated layout at that moment (a hole of the starting layout not
+    yet filled, or a slot vacated by an earlier move of the plan) and whose page, in that simulated layout, is
+    empty or holds entries of class c only; if there is none it stays.  Entries that are not candidates never
+    move, and no entry moves twice.  A destination may be the source of an earlier move, so the copies are
+    as-if all sources were read before any destination is written.
+    Accept test.  The moves are simulated; a page (subblock) is active if it holds a live entry; the plan is
+    accepted iff the number of active pages or the number of active subblocks decreases.  A rejected plan
+    moves nothing.
+    Promotion (Section 6.1): after an accepted plan every full page whose entries are all of the classes
+    selected-history / recent-context becomes selected-history (its entries' class is rewritten to 1).
+
+    Returns dict(accepted, moves [(src, dst)], k, v, keep_mask, slot_class (of the new layout; dead slots 0),
+    page_class [n_pages] (class of a page's entries, PAGE_MIXED, PAGE_EMPTY), pages_before, pages_after,
+    subblocks_before, subblocks_after, n_candidates).
+    """
+    keep = np.asarray(keep_mask).astype(bool).copy()
+    cls = np.where(keep, np.asarray(slot_class).astype(np.uint8), 0).astype(np.uint8)
+    S, P, B = len(keep), int(page_size), int(subblock)
+    assert P % B == 0
+    n_pages = (S + P - 1) // P
+    page_of = np.arange(S) // P
+
+    def active(mask, size):
+        n = (S + size - 1) // size
+        return int(np.count_nonzero(np.bincount(np.arange(S)[mask] // size, minlength=n))) if S else 0
+
+    pages_before, sub_before = active(keep, P), active(keep, B)
+    # simulated layout
+    live = keep.copy()
+    c_now = cls.copy()
+    page_fill0 = np.bincount(page_of[keep], minlength=n_pages)
+    page_len = np.minimum(P, S - np.arange(n_pages) * P)            # the last page may be short
+    cnt = np.zeros((n_pages, 3), np.int64)                          # live entries per page and class
+    for c in range(3):
+        cnt[:, c] = np.bincount(page_of[keep & ((cls & 3) == c)], minlength=n_pages)
+    cand = [s for s in np.nonzero(keep & ((cls & CLASS_CANDIDATE) != 0))[0] if page_fill0[s // P] < page_len[s // P]]
+    moves = []
+    for s in cand:
+        c = int(cls[s] & 3)
+        others = cnt.sum(axis=1) - cnt[:, c]
+        ok_page = others == 0                                       # empty, or class c only
+        dst_ok = ~live[:s] & ok_page[page_of[:s]]
+        hit = np.nonzero(dst_ok)[0]
+        if len(hit) == 0:
+            continue
+        d = int(hit[0])
+        moves.append((int(s), d))
+        live[s], live[d] = False, True
+        c_now[d], c_now[s] = c_now[s], 0
+        cnt[s // P, c] -= 1
+        cnt[d // P, c] += 1
+    pages_after, sub_after = active(live, P), active(live, B)
+    accepted = bool(moves) and (pages_after < pages_before or sub_after < sub_before)
+    k = np.array(k_cache, copy=True) if k_cache is not None else None
+    v = np.array(v_cache, copy=True) if v_cache is not None else None
+    if not accepted:
+        live, c_now, moves_done = keep, cls, []
+        pages_after, sub_after = pages_before, sub_before
+    else:
+        moves_done = moves
+        if k is not None and moves:
+            src = np.array([m[0] for m in moves]); dst = np.array([m[1] for m in moves])
+            k[dst] = np.asarray(k_cache)[src]                       # sources are read from the starting layout
+            v[dst] = np.asarray(v_cache)[src]
+    c_out = c_now.copy()
+    page_class = np.full(n_pages, PAGE_EMPTY, np.uint8)
+    for p in range(n_pages):
+        sl = slice(p * P, min(S, (p + 1) * P))
+        m = live[sl]
+        if not m.any():
+            continue
+        kinds = np.unique(c_out[sl][m] & 3)
+        if accepted and promote and m.all() and len(m) == P and kinds.min() >= CLASS_SELECTED:
+            c_out[sl] = (c_out[sl] & ~np.uint8(3)) | np.uint8(CLASS_SELECTED)
+            kinds = np.array([CLASS_SELECTED])
+        page_class[p] = kinds[0] if len(kinds) == 1 else PAGE_MIXED
+    return dict(accepted=accepted, moves=moves_done, k=k, v=v, keep_mask=live.astype(np.uint8), slot_class=c_out,
+                page_class=page_class, pages_before=pages_before, pages_after=pages_after,
+                subblocks_before=sub_before, subblocks_after=sub_after, n_candidates=len(cand))
 
 
 def chunk_attention_masked(q, k_cache, v_cache, keep_mask, k_chunk, v_chunk, scale=None, rows=None):

@@ -679,3 +679,139 @@ def test_attention_masked_is_attention_over_live_rows():
     assert m["start"] >= 0
     o2, _ = oc.chunk_attention_masked(w.q, m["k"], m["v"], m["keep_mask"], w.k_chunk, w.v_chunk)
     assert np.allclose(o, o2, atol=1e-12)
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# class-aware selective migration (Section 6.2 "packing scattered entries" / "checking layout improvement")
+def _class_layout(spec):
+    """'M' must-keep, 's'/'r' selected / recent, 'S'/'R' the same as candidates, '.' a hole."""
+    code = {"M": 0, "s": 1, "r": 2, "S": 1 | 0x80, "R": 2 | 0x80}
+    spec = spec.replace(" ", "")
+    keep = np.array([ch != "." for ch in spec], dtype=np.uint8)
+    cls = np.array([code.get(ch, 0) for ch in spec], dtype=np.uint8)
+    return keep, cls
+
+
+def test_migrate_class_hand_worked():
+    # pages of 4, subblocks of 2.  Candidates in physical order: 4 (no earlier hole: stays), 7 -> 5, 9 -> 6,
+    # 15 -> 7 (the slot vacated by the first move; page 1 holds class selected only).  Pages 4 -> 3, subblocks 7 -> 5.
+    keep, cls = _class_layout("MMMM S..S .S.. r..S")
+    ids = np.arange(16)
+    r = oc.migrate_class(ids, ids + 100, keep, cls, 4, 2)
+    assert r["accepted"] and r["moves"] == [(7, 5), (9, 6), (15, 7)]
+    assert (r["pages_before"], r["pages_after"], r["subblocks_before"], r["subblocks_after"]) == (4, 3, 7, 5)
+    assert r["keep_mask"].tolist() == [1, 1, 1, 1, 1, 1, 1, 1, 0, 0, 0, 0, 1, 0, 0, 0]
+    assert r["k"][[4, 5, 6, 7, 12]].tolist() == [4, 7, 9, 15, 12] and r["v"][[5, 6, 7]].tolist() == [107, 109, 115]
+    assert r["page_class"].tolist() == [0, 1, oc.PAGE_EMPTY, 2] and r["n_candidates"] == 4
+    assert r["slot_class"][4:8].tolist() == [0x81] * 4                       # the moved entries keep class and mark
+
+    # destination pages must be empty or of the same class: the hole in the must-keep page (slot 2) and the holes
+    # of the page that holds a recent entry (5, 6) are closed to a selected-history candidate; page 2 is empty.
+    keep, cls = _class_layout("MM.M r..r .... ..S. ...S")
+    r = oc.migrate_class(ids.repeat(2)[:20], ids.repeat(2)[:20], keep, cls, 4, 2)
+    assert r["moves"] == [(14, 8), (19, 9)] and r["accepted"]
+    assert (r["pages_before"], r["pages_after"]) == (4, 3) and (r["subblocks_before"], r["subblocks_after"]) == (6, 5)
+    # a recent-context candidate may use the holes of the recent page, not the others
+    keep, cls = _class_layout("MM.M r..r .... ..R.")
+    assert oc.migrate_class(None, None, keep, cls, 4, 2)["moves"] == [(14, 5)]
+
+    # moving an entry between two pages that both stay active is not an improvement: rejected, nothing moves
+    keep, cls = _class_layout("S... sS..")
+    r = oc.migrate_class(np.arange(8), np.arange(8), keep, cls, 4, 2)
+    assert not r["accepted"] and r["moves"] == [] and np.array_equal(r["keep_mask"], keep)
+    assert np.array_equal(r["k"], np.arange(8)) and (r["pages_after"], r["subblocks_after"]) == (2, 2)
+    # ... but with the candidate alone in its subblock the subblock count drops: accepted although both pages stay
+    keep, cls = _class_layout("S... s..S")
+    r = oc.migrate_class(np.arange(8), np.arange(8), keep, cls, 4, 2)
+    assert r["accepted"] and r["moves"] == [(7, 1)] and (r["pages_after"], r["subblocks_after"]) == (2, 2)
+    assert (r["pages_before"], r["subblocks_before"]) == (2, 3)
+
+    # full pages stay in place: the candidates of page 1 do not move although page 0 has holes; the one of page 2 does
+    keep, cls = _class_layout("s... SSSS S...")
+    r = oc.migrate_class(None, None, keep, cls, 4, 2)
+    assert r["moves"] == [(8, 1)] and r["n_candidates"] == 1
+
+    # promotion: a page packed full of recent / selected entries becomes selected-history; a full page that holds
+    # must-keep entries does not; nothing is promoted when the plan is rejected
+    keep, cls = _class_layout("Rr.r .R.. MMMM")
+    r = oc.migrate_class(None, None, keep, cls, 4, 2)
+    assert r["moves"] == [(5, 2)] and r["accepted"]
+    assert r["slot_class"][:4].tolist() == [0x81, 1, 0x81, 1] and r["page_class"].tolist() == [1, oc.PAGE_EMPTY, 0]
+    r = oc.migrate_class(None, None, keep, cls, 4, 2, promote=False)
+    assert r["slot_class"][:4].tolist() == [0x82, 2, 0x82, 2] and r["page_class"].tolist() == [2, oc.PAGE_EMPTY, 0]
+    keep, cls = _class_layout("rrrr rR..")                                   # no hole before the candidate: no plan
+    r = oc.migrate_class(None, None, keep, cls, 4, 2)
+    assert not r["accepted"] and r["slot_class"][:4].tolist() == [2, 2, 2, 2] and r["page_class"].tolist() == [2, 2]
+
+
+def test_migrate_class_replay_minimality_and_invariants():
+    rng = np.random.default_rng(4711)
+    n_acc = n_rej = 0
+    for trial in range(300):
+        P = int(rng.choice([4, 8, 16])); B = int(rng.choice([b for b in (2, 4, 8, 16) if P % b == 0]))
+        S = int(rng.integers(1, 160))
+        keep = (rng.random(S) < rng.random()).astype(np.uint8)
+        # classes in runs (must-keep head, then selected / recent mixed by runs), candidates at random
+        cls = np.zeros(S, np.uint8)
+        pos = int(rng.integers(0, max(1, S // 4)))
+        while pos < S:
+            n = int(rng.integers(1, 3 * P)); cls[pos:pos + n] = rng.choice([1, 2]); pos += n
+        cls |= np.where(rng.random(S) < rng.random(), 0x80, 0).astype(np.uint8)
+        cls = np.where(keep == 1, cls, 0).astype(np.uint8)
+        ids = rng.permutation(S) + 1
+        r = oc.migrate_class(ids, -ids, keep, cls, P, B)
+        # independent replay with sets: every move went to the smallest empty compatible slot before its source
+        live = {s: (int(ids[s]), int(cls[s])) for s in range(S) if keep[s]}
+        full0 = {p for p in range(-(-S // P)) if all((s in live) for s in range(p * P, min(S, (p + 1) * P)))}
+        planned = []
+        for s in sorted(s for s in live if live[s][1] & 0x80 and s // P not in full0):
+            c = live[s][1] & 3
+            best = None
+            for d in range(s):
+                if d in live:
+                    continue
+                if all((live[x][1] & 3) == c for x in range(d // P * P, min(S, (d // P + 1) * P)) if x in live):
+                    best = d
+                    break
+            if best is not None:
+                live[best] = live.pop(s)
+                planned.append((s, best))
+        act = lambda slots, size: len({s // size for s in slots})
+        before = set(np.nonzero(keep)[0].tolist())
+        improves = bool(planned) and (act(live, P) < act(before, P) or act(live, B) < act(before, B))
+        assert r["accepted"] == improves
+        assert (r["pages_before"], r["subblocks_before"]) == (act(before, P), act(before, B))
+        if not improves:
+            n_rej += 1
+            assert r["moves"] == [] and np.array_equal(r["keep_mask"], keep) and np.array_equal(r["k"], ids)
+            assert np.array_equal(r["slot_class"], cls)
+            continue
+        n_acc += 1
+        assert r["moves"] == planned
+        assert (r["pages_after"], r["subblocks_after"]) == (act(live, P), act(live, B))
+        assert set(np.nonzero(r["keep_mask"])[0].tolist()) == set(live)
+        for s, (i, c) in live.items():
+            assert r["k"][s] == i and r["v"][s] == -i and (r["slot_class"][s] & 0x80) == (c & 0x80)
+            promoted = s // P * P + P <= S and all(x in live and (live[x][1] & 3) >= 1 for x in range(s // P * P, s // P * P + P))
+            assert (r["slot_class"][s] & 3) == (1 if promoted else (c & 3))
+        # the history is the same set of entries: nothing lost, nothing duplicated, non-candidates did not move
+        assert sorted(i for i, _ in live.values()) == sorted(int(ids[s]) for s in before)
+        moved_from = {s for s, _ in planned}
+        assert all(cls[s] & 0x80 for s in moved_from) and all(d < s for s, d in planned)
+    assert n_acc > 50 and n_rej > 20
+
+
+def test_migrate_class_leaves_attention_unchanged():
+    rng = np.random.default_rng(77)
+    S, P, B, hq, hkv, d, t = 96, 8, 4, 4, 2, 16, 5
+    keep = (rng.random(S) < 0.35).astype(np.uint8)
+    cls = np.where(keep == 1, rng.choice([1, 2], size=S) | np.where(rng.random(S) < 0.6, 0x80, 0), 0).astype(np.uint8)
+    k = rng.standard_normal((S, hkv, d)); v = rng.standard_normal((S, hkv, d))
+    q = rng.standard_normal((t, hq, d)); kc = rng.standard_normal((t, hkv, d)); vc = rng.standard_normal((t, hkv, d))
+    r = oc.migrate_class(k, v, keep, cls, P, B)
+    assert r["accepted"] and len(r["moves"]) > 5
+    a0 = oc.chunk_attention_masked(q, k, v, keep, kc, vc)
+    a1 = oc.chunk_attention_masked(q, r["k"], r["v"], r["keep_mask"], kc, vc)
+    out0 = a0[0] if isinstance(a0, tuple) else a0
+    out1 = a1[0] if isinstance(a1, tuple) else a1
+    assert np.allclose(out0, out1, rtol=0, atol=1e-12)
