@@ -266,7 +266,7 @@ def main():
     ap.add_argument("--mask-compaction", action="store_true",
                     help="time omnipage_compact (token keep mask + slot map) instead of the unit-granular entry point")
     ap.add_argument("--no-ablation", dest="ablation", action="store_false",
-                    help="skip the native / ordered-suffix / eager layout ablation")
+                    help="skip the native / class-aware / ordered-suffix / eager layout ablation")
     ap.add_argument("--batch-layers", type=int, default=36,
                     help="layers packed by one launch of the cross-layer batched compaction (0: skip it)")
     ap.add_argument("--loop-chunks", type=int, default=40, help="chunks of the 36-layer stream loop (0: skip it)")
@@ -520,9 +520,20 @@ def main():
         ctx.plan_structural(units_in, n_units_dev, U, sp, a_keep, a_klen, a_mask0, N, a_nk, a_units, a_nu)
         span_dev = cnt(N)
         a_info = torch.zeros(8, dtype=torch.int32, device="cuda")
+        # allocation classes of that plan: the sink prefixes of partially evicted units are the candidates
+        # (selected-history), units kept whole are recent-context
+        torch.cuda.synchronize()
+        u_host, klen_host = units_in[:U].cpu().numpy(), a_klen[:U].cpu().numpy()
+        cls_host = np.zeros(s_cap + 16, dtype=np.uint8)
+        for (st_, ln_), kl_ in zip(u_host[:, :2].tolist(), klen_host.tolist()):
+            cls_host[st_:st_ + kl_] = (1 | 0x80) if 0 < kl_ < ln_ else 2
+        a_cls0 = torch.from_numpy(cls_host).cuda()
+        a_cls = torch.zeros_like(a_cls0)
+        c_info = torch.zeros(8, dtype=torch.int32, device="cuda")
         ev = lambda: torch.cuda.Event(enable_timing=True)
         reps = max(5, min(args.steps, 20))
-        res = {"native": [], "suffix_migrate": [], "suffix_attention": [], "eager_pack": [], "eager_attention": []}
+        res = {"native": [], "suffix_migrate": [], "suffix_attention": [], "eager_pack": [], "eager_attention": [],
+               "class_migrate": [], "class_attention": []}
         spans = {}
         for i in range(2 + reps):
             s_ = sets[i % R]
@@ -546,9 +557,21 @@ def main():
             ctx.chunk_attention(s_["q"], T, k_w, v_w, a_nk, N, s_["kc"], s_["vc"], 0.0, s_["o"], ob.DTYPE_FP32)
             e[6].record()
             torch.cuda.synchronize()
+            # class-aware mode: fills earlier holes with the sink prefixes; the span stays, pages empty out
+            k_w.copy_(s_["k_in"]); v_w.copy_(s_["v_in"])
+            a_mask.copy_(a_mask0); a_cls.copy_(a_cls0); span_dev.fill_(N)
+            e2 = [ev() for _ in range(3)]
+            e2[0].record()
+            ctx.migrate_class(k_w, v_w, a_mask, a_cls, span_dev, N, w.page_size, max(1, w.page_size // 2), 1, None, None, c_info)
+            e2[1].record()
+            ctx.chunk_attention_masked(s_["q"], T, k_w, v_w, a_mask, span_dev, N, s_["kc"], s_["vc"], 0.0, s_["o"], ob.DTYPE_FP32)
+            e2[2].record()
+            torch.cuda.synchronize()
             if i >= 2:
                 for name, (x, y) in zip(res, ((0, 1), (1, 2), (2, 3), (4, 5), (5, 6))):
                     res[name].append(e[x].elapsed_time(e[y]))
+                res["class_migrate"].append(e2[0].elapsed_time(e2[1]))
+                res["class_attention"].append(e2[1].elapsed_time(e2[2]))
         assert ctx.poll_status() == 0, "device status word not clean after the layout ablation"
         live = int(a_nk.item())
         abl = {k_: float(np.mean(v_)) for k_, v_ in res.items()}
@@ -558,6 +581,10 @@ def main():
                "suffix_migrate_ms": abl["suffix_migrate"], "suffix_attention_ms": abl["suffix_attention"],
                "eager_ms": abl["eager_pack"] + abl["eager_attention"], "eager_pack_ms": abl["eager_pack"],
                "eager_attention_ms": abl["eager_attention"],
+               "class_ms": abl["class_migrate"] + abl["class_attention"], "class_migrate_ms": abl["class_migrate"],
+               "class_attention_ms": abl["class_attention"],
+               "class_info": dict(zip(("accepted", "n_moves", "n_candidates", "pages_before", "pages_after",
+                                       "subblocks_before", "subblocks_after"), c_info.cpu().tolist())),
                "note": "maintenance + chunk attention per layout after one structural retention round (suffix threshold 8 pages)"}
         line["layout_ablation"] = abl
 

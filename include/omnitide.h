@@ -106,6 +106,27 @@ typedef struct {
     int32_t reserved;
 } omni_compact_info;
 
+/* Allocation classes of Section 6.1, the low two bits of a slot_class byte; bit 7 marks an entry that was
+ * retained from a partially evicted unit (a candidate of the class-aware migration, Section 6.2). */
+enum {
+    OMNI_CLASS_MUST_KEEP = 0,
+    OMNI_CLASS_SELECTED = 1,
+    OMNI_CLASS_RECENT = 2,
+    OMNI_CLASS_CANDIDATE = 0x80
+};
+#define OMNI_PAGE_MIXED 254   /* page label: live entries of more than one class */
+#define OMNI_PAGE_EMPTY 255   /* page label: no live entry */
+
+/* Outcome of omnipage_migrate_class (32 bytes). */
+typedef struct omni_class_info {
+    int32_t accepted;          /* 1 if the plan reduced the active pages or the active subblocks and was carried out */
+    int32_t n_moves;           /* rows moved (0 when rejected) */
+    int32_t n_candidates;      /* candidates the planner visited */
+    int32_t pages_before, pages_after;          /* pages that hold a live entry */
+    int32_t subblocks_before, subblocks_after;  /* subblocks that hold a live entry */
+    int32_t reserved;
+} omni_class_info;
+
 typedef struct omnitide_ctx omnitide_ctx;
 
 /* Creates a context for one geometry on the current device and allocates its scratch memory.
@@ -248,6 +269,33 @@ omni_status omnipage_migrate_suffix(omnitide_ctx* ctx, void* stream, void* k_cac
                                     uint8_t* keep_mask, int32_t* s_span_dev, int32_t s_span_max,
                                     int32_t page_size, int32_t min_pages_saved,
                                     int32_t* slot_map_out, omni_compact_info* info_out);
+
+/*
+ * (next row: selective migration, class-aware mode; Section 6.2 "Packing scattered entries" and "Checking layout
+ * improvement", classes and promotion of Section 6.1)  Plans, checks and carries out the moves that fill earlier
+ * holes with the entries retained from partially evicted units.
+ *   keep_mask [dev, in/out] s_span_max bytes, 1 = live; slot_class [dev, in/out] s_span_max bytes, read where live:
+ *   class in bits 0-1 (OMNI_CLASS_*; the value 3 sets OMNI_DEV_BAD_UNITS and nothing moves), candidate mark in bit 7.
+ *   *s_span_dev [dev, nullable] / s_span_max [host]: the span; pages are page_size slots, subblocks `subblock` slots
+ *   (subblock divides page_size).
+ * Plan: the candidates (live, marked, in a page that is not full) are visited in ascending slot order; a candidate
+ * of class c at slot s goes to the smallest slot d < s that is empty in the layout as simulated so far (vacated
+ * slots count) and whose page is empty or holds class c only; if there is none it stays.  Nothing else moves.
+ * Accept test: the plan is carried out iff it lowers the number of pages, or of subblocks, that hold a live entry.
+ * If carried out: K/V rows move in place (all sources are read into context scratch before any destination is
+ * written), keep_mask and slot_class follow the entries (vacated slots become 0), and if `promote` is non-zero every
+ * page that is now full of selected-history / recent-context entries is relabelled selected-history.
+ *   moves_out [dev, nullable] 2 * s_span_max int32: the (source, destination) pairs in plan order, for the caller's
+ *   own per-slot metadata; page_class_out [dev, nullable] ceil(s_span_max / page_size) bytes: class of the page's
+ *   entries, OMNI_PAGE_MIXED or OMNI_PAGE_EMPTY (pages past the span are not written); info_out [dev] the counts.
+ * The layout (one bit per slot, eight bytes per page) must fit one CTA's shared memory, else OMNI_ERR_CAPACITY.
+ * The result is a layout for omnitide_chunk_attention_masked.
+ */
+omni_status omnipage_migrate_class(omnitide_ctx* ctx, void* stream, void* k_cache, void* v_cache,
+                                   uint8_t* keep_mask, uint8_t* slot_class, const int32_t* s_span_dev,
+                                   int32_t s_span_max, int32_t page_size, int32_t subblock, int32_t promote,
+                                   int32_t* moves_out, uint8_t* page_class_out, omni_class_info* info_out);
+
 
 /*
  * (next row: RoPE position re-index fused into the gather; Section 5.2 "the runtime applies the corresponding RoPE

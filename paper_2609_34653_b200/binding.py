@@ -45,9 +45,15 @@ class CompactInfo(C.Structure):
                 ("part_begin", C.c_int32 * 4), ("reserved", C.c_int32)]
 
 
+class ClassInfo(C.Structure):
+    _fields_ = [("accepted", C.c_int32), ("n_moves", C.c_int32), ("n_candidates", C.c_int32),
+                ("pages_before", C.c_int32), ("pages_after", C.c_int32),
+                ("subblocks_before", C.c_int32), ("subblocks_after", C.c_int32), ("reserved", C.c_int32)]
+
+
 EXPORTS = [
     "omnitide_create", "omnitide_destroy", "omnitide_poll_status", "omnitide_last_error",
-    "omnitide_score_units", "omnitide_select_units", "omnitide_plan_structural", "omnipage_compact", "omnipage_migrate_suffix", "omnipage_compact_units", "omnipage_compact_units_rope", "omnipage_compact_units_batched", "omnipage_append",
+    "omnitide_score_units", "omnitide_select_units", "omnitide_plan_structural", "omnipage_compact", "omnipage_migrate_suffix", "omnipage_migrate_class", "omnipage_compact_units", "omnipage_compact_units_rope", "omnipage_compact_units_batched", "omnipage_append",
     "omnitide_chunk_attention", "omnitide_chunk_attention_masked", "omnitide_chunk_step", "omnitide_chunk_step_host", "omnitide_chunk_step_structural",
     "omnitide_set_option", "omnitide_launch_count", "omnitide_score_units_noalloc",
 ]
@@ -74,6 +80,7 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.omnipage_compact.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, i32, vp, vp, vp]
     lib.omnitide_plan_structural.argtypes = [vp, vp, vp, vp, i32, C.POINTER(StructuralParams), vp, vp, vp, i32, vp, vp, vp]
     lib.omnipage_migrate_suffix.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp]
+    lib.omnipage_migrate_class.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp]
     lib.omnipage_compact_units.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, i32, i32, vp, vp, vp, vp, vp]
     lib.omnipage_compact_units_rope.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, i32, i32, vp, vp, vp, vp, vp,
                                                 C.POINTER(RopeParams)]
@@ -213,6 +220,13 @@ class Context:
         self._check(self.lib.omnipage_migrate_suffix(self._ctx, _stream(), _ptr(k_cache), _ptr(v_cache), _ptr(keep_mask),
                                                      _ptr(s_span_dev), s_span_max, page_size, min_pages_saved,
                                                      _ptr(slot_map_out), _ptr(info_out)), "omnipage_migrate_suffix")
+
+    def migrate_class(self, k_cache, v_cache, keep_mask, slot_class, s_span_dev, s_span_max, page_size, subblock,
+                      promote, moves_out, page_class_out, info_out):
+        self._check(self.lib.omnipage_migrate_class(self._ctx, _stream(), _ptr(k_cache), _ptr(v_cache), _ptr(keep_mask),
+                                                    _ptr(slot_class), _ptr(s_span_dev), s_span_max, page_size, subblock,
+                                                    int(bool(promote)), _ptr(moves_out), _ptr(page_class_out),
+                                                    _ptr(info_out)), "omnipage_migrate_class")
 
     def compact_units(self, k_src, v_src, k_dst, v_dst, units, n_units_dev, n_units_max, unit_keep, s_span_max,
                       page_size, units_kept, n_units_kept_dev, slot_map_out, info_out, page_class_out, unit_kept_len=None):

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libomnitide.so")
-SOURCES = ["api.cu", "compact.cu", "select.cu", "simple_paths.cu", "attention_tc.cu", "score_tc.cu", "decode.cu"]
+SOURCES = ["api.cu", "compact.cu", "select.cu", "simple_paths.cu", "attention_tc.cu", "score_tc.cu", "decode.cu", "migrate_class.cu"]
 
 
 def _newest_source_mtime() -> float:

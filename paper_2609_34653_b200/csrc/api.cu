@@ -19,7 +19,7 @@ void free_all(omnitide_ctx* c) {
     void* ptrs[] = {c->status_dev, c->score_part, c->score_tile_mass, c->score_mass64, c->inplace_k, c->inplace_v,
                     c->ws_scores, c->ws_unit_keep, c->ws_kept_len, c->ws_keep_mask, c->ws_slot_map, c->ws_counts, c->ws_info, c->st_q,
                     c->st_k, c->st_v, c->st_o, c->st_units, c->attn_part_o, c->attn_part_ml, c->cp_words, c->attn_live_idx, c->attn_live_mask,
-                    c->attn_n_live, c->mig_plan, c->dec_counter};
+                    c->attn_n_live, c->mig_plan, c->dec_counter, c->mc_moves, c->mc_class};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);

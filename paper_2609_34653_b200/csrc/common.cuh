@@ -26,6 +26,8 @@ struct omnitide_ctx {
     void* inplace_v;
     size_t inplace_rows;
     int32_t* mig_plan;            // [8] plan of the ordered-suffix migration, allocated on first use
+    int32_t* mc_moves;            // [2 s_cap] (source, destination) pairs of the class-aware migration, allocated on first use
+    uint8_t* mc_class;            // [s_cap] class bytes of its moved entries
     unsigned long long* cp_words; // [SMs] per-CTA count words of the compaction kernel, tagged with cp_epoch
     uint32_t cp_epoch;            // launches of the compaction kernel on this context so far
     // work buffers of omnitide_chunk_step
@@ -81,6 +83,7 @@ struct omnitide_ctx {
 static inline bool omni_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 // internal entry points implemented per file
+omni_status omni_inplace_staging(omnitide_ctx* ctx);   // allocates inplace_k / inplace_v (s_cap rows each) on first use
 omni_status omni_attention_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q, int t, const void* k_hist,
                               const void* v_hist, const int32_t* n_hist_dev, int n_hist_max, const void* k_chunk,
                               const void* v_chunk, float scale, void* o_out, int out_dtype, float* lse_out,

@@ -929,7 +929,7 @@ __global__ void __launch_bounds__(256) suffix_finish_kernel(uint8_t* mask, int32
 }
 
 // Staging rows of the in-place mode, allocated on the first in-place call on a context (synchronous).
-static omni_status omni_inplace_staging(omnitide_ctx* ctx) {
+omni_status omni_inplace_staging(omnitide_ctx* ctx) {
     if (ctx->inplace_rows >= (size_t)ctx->g.s_cap) return OMNI_OK;
     if (ctx->inplace_k) cudaFree(ctx->inplace_k);
     if (ctx->inplace_v) cudaFree(ctx->inplace_v);

@@ -46,6 +46,7 @@ def test_struct_layouts_match_the_header():
     assert ctypes.sizeof(binding.SelectParams) == 20
     assert ctypes.sizeof(binding.StructuralParams) == 28
     assert ctypes.sizeof(binding.CompactInfo) == 32
+    assert ctypes.sizeof(binding.ClassInfo) == 32
 
 
 def test_create_without_gpu_fails_loudly(lib_path):

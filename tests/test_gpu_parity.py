@@ -761,6 +761,129 @@ def test_migrate_suffix_bit_exact(H, ob, S, page, theta, pattern, seed):
     ctx.close()
 
 
+# ------------------------------------------------------------------ class-aware selective migration
+def _class_case(rng, S, page, pattern):
+    """A layout after a structural retention round: a must-keep head, older units reduced to short marked prefixes
+    (selected-history), unmarked survivors, recent units whole (recent-context)."""
+    keep = np.zeros(S, np.uint8)
+    cls = np.zeros(S, np.uint8)
+    head = min(S // 8, 3 * page + 5)
+    keep[:head] = 1                                              # must-keep, class 0
+    recent0 = S - S // 6
+    pos = head
+    while pos < recent0:
+        n = int(rng.integers(40, 700))
+        end = min(recent0, pos + n)
+        r = rng.random()
+        if pattern == "random":
+            m = rng.random(end - pos) < 0.3
+            keep[pos:end] = m
+            cls[pos:end] = np.where(m, rng.choice([1, 2]) | np.where(rng.random(end - pos) < 0.7, 0x80, 0), 0)
+        elif r < 0.65:                                           # sink prefix of a partially evicted unit
+            pre = min(end - pos, int(rng.choice([4, 8, 24])))
+            keep[pos:pos + pre] = 1
+            cls[pos:pos + pre] = 1 | 0x80
+        elif r < 0.8:                                            # kept whole: not a candidate
+            keep[pos:end] = 1
+            cls[pos:end] = 1
+        pos = end
+    keep[recent0:] = 1
+    cls[recent0:] = 2
+    if pattern == "no_holes":
+        keep[:] = 1
+        cls[head:recent0] = 1 | 0x80
+    return keep, np.where(keep == 1, cls, 0).astype(np.uint8)
+
+
+@pytest.mark.parametrize("S,page,sub,pattern,promote,seed", [
+    (1000, 16, 8, "random", 1, 0),
+    (5000, 64, 32, "sinks", 1, 1),
+    (16384, 64, 32, "random", 1, 2),
+    (3000, 256, 64, "sinks", 0, 3),
+    (2048, 64, 64, "no_holes", 1, 4),      # no empty slot anywhere: no plan
+    (80000, 64, 32, "sinks", 1, 5),
+    (80000, 16, 16, "random", 1, 6),
+    (777, 16, 2, "random", 1, 7),
+    (37, 16, 4, "random", 1, 8),
+])
+def test_migrate_class_bit_exact(H, ob, S, page, sub, pattern, promote, seed):
+    """omnipage_migrate_class equals the oracle: the plan move by move, the accept decision and its four counts, the new
+    mask, classes and page labels, and every live row of the cache, bit for bit."""
+    rng = np.random.default_rng(500 + seed)
+    keep, cls = _class_case(rng, S, page, pattern)
+    rowshape = (2, 128)
+    raw = rng.integers(0, 256, size=(2, S, rowshape[0] * rowshape[1] * 2), dtype=np.uint8)
+    k = torch.from_numpy(raw[0]).cuda().view(torch.bfloat16).view(S, *rowshape).contiguous()
+    v = torch.from_numpy(raw[1]).cuda().view(torch.bfloat16).view(S, *rowshape).contiguous()
+    exp = oc.migrate_class(raw[0], raw[1], keep, cls, page, sub, promote=bool(promote))
+    ctx = ob.Context(8, 2, 128, "bf16", S + 64, 8, 16)
+    mask = torch.zeros((S + 48,), dtype=torch.uint8, device="cuda")
+    mask[:S] = torch.from_numpy(keep).cuda()
+    mask[S:S + 40] = 1                                        # stale bytes beyond the span
+    sc = torch.zeros((S + 48,), dtype=torch.uint8, device="cuda")
+    sc[:S] = torch.from_numpy(cls).cuda()
+    n_pages = -(-S // page)
+    moves = torch.full((2 * (S + 48),), -5, dtype=torch.int32, device="cuda")
+    labels = torch.full((n_pages + 4,), 77, dtype=torch.uint8, device="cuda")
+    info = torch.full((8,), -5, dtype=torch.int32, device="cuda")
+    ctx.migrate_class(k, v, mask, sc, H.i32(S), S + 40, page, sub, promote, moves, labels, info)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    acc, n_moves, n_cand, pb, pa, sb, sa, _ = info.cpu().tolist()
+    assert bool(acc) == exp["accepted"] and n_moves == len(exp["moves"]) and n_cand == exp["n_candidates"]
+    assert (pb, pa, sb, sa) == (exp["pages_before"], exp["pages_after"], exp["subblocks_before"], exp["subblocks_after"])
+    if exp["accepted"]:
+        assert moves[:2 * n_moves].cpu().numpy().reshape(-1, 2).tolist() == [list(m) for m in exp["moves"]]
+    new_mask = mask[:S].cpu().numpy()
+    assert np.array_equal(new_mask, exp["keep_mask"]) and bool((mask[S:S + 40] == 1).all())
+    live = new_mask == 1
+    assert np.array_equal(sc[:S].cpu().numpy()[live], exp["slot_class"][live])
+    vacated = (keep == 1) & ~live
+    assert not sc[:S].cpu().numpy()[vacated].any()
+    assert np.array_equal(labels[:n_pages].cpu().numpy(), exp["page_class"]) and bool((labels[n_pages:] == 77).all())
+    assert np.array_equal(H.bytes_of(k).reshape(S, -1)[live], exp["k"][live])
+    assert np.array_equal(H.bytes_of(v).reshape(S, -1)[live], exp["v"][live])
+    if pattern == "no_holes":
+        assert not exp["accepted"] and n_moves == 0
+    elif S >= 777:
+        assert exp["accepted"] and n_moves > 0          # the cases are meant to exercise the move path
+    ctx.close()
+
+
+def test_migrate_class_then_attention(H, ob, cfg2):
+    """Attention over the class-migrated layout equals attention over the layout with its original holes: the migration
+    changes where entries are stored, not the history (Section 6.2)."""
+    w = cfg2
+    N, T = w.n_hist, w.t
+    plan = oc.plan_structural(w.units, 0, 6000, 2, (24, 8, 0), 64)
+    keep = plan["keep_mask"]
+    kept_len = plan["unit_kept_len"]
+    cls = np.zeros(N, np.uint8)
+    for u, (st, ln) in enumerate(zip(w.units[:, oc.U_START].tolist(), w.units[:, oc.U_LEN].tolist())):
+        part = 0 < kept_len[u] < ln
+        cls[st:st + ln] = (1 | 0x80) if part else 2
+    cls = np.where(keep == 1, cls, 0).astype(np.uint8)
+    o_ref, _ = oc.chunk_attention_masked(w.q, w.k_hist, w.v_hist, keep, w.k_chunk, w.v_chunk)
+    exp = oc.migrate_class(None, None, keep, cls, w.page_size, w.page_size // 2)
+    ctx = H.make_ctx(w)
+    q, kc, vc = (ob.to_device(a, "bf16") for a in (w.q, w.k_chunk, w.v_chunk))
+    k, v = ob.to_device(w.k_hist, "bf16").clone(), ob.to_device(w.v_hist, "bf16").clone()
+    mask = torch.zeros((N + 16,), dtype=torch.uint8, device="cuda")
+    mask[:N] = torch.from_numpy(keep).cuda()
+    sc = torch.from_numpy(cls).cuda()
+    info = torch.zeros((8,), dtype=torch.int32, device="cuda")
+    ctx.migrate_class(k, v, mask, sc, None, N, w.page_size, w.page_size // 2, 1, None, None, info)
+    o = torch.zeros((T, w.h_q, w.d), dtype=torch.float32, device="cuda")
+    ctx.chunk_attention_masked(q, T, k, v, mask, H.i32(N), N, kc, vc, 0.0, o, ob.DTYPE_FP32)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    got = info.cpu().tolist()
+    assert bool(got[0]) == exp["accepted"] and got[1] == len(exp["moves"]) and got[4] == exp["pages_after"]
+    assert np.array_equal(mask[:N].cpu().numpy(), exp["keep_mask"])
+    _check_attention(o.cpu().numpy(), None, o_ref, None)
+    ctx.close()
+
+
 def test_native_suffix_eager_layouts_attend_alike(H, ob, cfg2):
     """The three layouts of the paper's ablation (native holes, ordered-suffix migration, eager pack) present the same
     live rows: attention over each of them matches the oracle, and the spans shrink in that order."""
