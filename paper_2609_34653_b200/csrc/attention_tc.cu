@@ -434,12 +434,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     mx3 = tc::max3(mx3, __uint_as_float(sa[i + 6]), __uint_as_float(sa[i + 7]));
                 }
 #pragma unroll
-                for (int i = 4; i < 32; i += 8) {
+                for (int i = 4; i < 28; i += 8) {
                     mx0 = tc::max3(mx0, __uint_as_float(sb[i]), __uint_as_float(sb[i + 1]));
                     mx1 = tc::max3(mx1, __uint_as_float(sb[i + 2]), __uint_as_float(sb[i + 3]));
                     mx2 = tc::max3(mx2, __uint_as_float(sb[i + 4]), __uint_as_float(sb[i + 5]));
                     mx3 = tc::max3(mx3, __uint_as_float(sb[i + 6]), __uint_as_float(sb[i + 7]));
                 }
+                mx0 = tc::max3(mx0, __uint_as_float(sb[28]), __uint_as_float(sb[29]));
+                mx1 = tc::max3(mx1, __uint_as_float(sb[30]), __uint_as_float(sb[31]));
                 const float bm = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
                 if ((warp & 3) == 0) TRACE(w, 1);
 
