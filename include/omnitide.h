@@ -433,6 +433,31 @@ omni_status omnitide_chunk_step_host(omnitide_ctx* ctx, void* stream,
                                      void* o_host, int32_t out_dtype, omni_compact_info* info_out);
 
 /*
+ * The same pass for a caller that streams chunks: the call only enqueues.  The context keeps two sets of staging
+ * buffers and runs the uploads of call n on a copy stream under the kernels of call n - 1, and the download of
+ * call n on a second copy stream under the kernels of call n + 1; the kernels themselves run on `stream` in call
+ * order (call n + 1 reads the cache state call n wrote).  Arguments as omnitide_chunk_step_host.
+ * The host input buffers of a call may be rewritten, and o_host read, only after omnitide_host_wait (or a
+ * synchronisation of the whole device); pinned host memory is needed for the copies to overlap.  Staging is
+ * allocated on the first call (synchronously).
+ */
+omni_status omnitide_chunk_step_host_pipelined(omnitide_ctx* ctx, void* stream,
+                                               const void* q_host, const void* k_chunk_host, const void* v_chunk_host,
+                                               int32_t t, const omni_unit* chunk_units_host, int32_t n_chunk_units,
+                                               const void* k_cache, const void* v_cache,
+                                               const int32_t* n_hist_dev, int32_t n_hist_max,
+                                               const omni_unit* units, const int32_t* n_units_dev, int32_t n_units_max,
+                                               const float* w_modality, const omni_select_params* params,
+                                               int32_t page_size, float scale,
+                                               void* k_cache_out, void* v_cache_out, omni_unit* units_out,
+                                               int32_t* n_hist_out, int32_t* n_units_out,
+                                               void* o_host, int32_t out_dtype, omni_compact_info* info_out);
+
+/* Blocks until every upload and download enqueued by the host entry points of this context has completed
+ * (the kernels on the caller's stream are the caller's to synchronise). */
+omni_status omnitide_host_wait(omnitide_ctx* ctx);
+
+/*
  * Unit scoring for callers that cannot allocate.  (The paper has no counterpart: this is a
  * packaging variant of omnitide_score_units, same formula, computed by the fp32 CUDA-core kernel.)
  *

@@ -54,7 +54,7 @@ class ClassInfo(C.Structure):
 EXPORTS = [
     "omnitide_create", "omnitide_destroy", "omnitide_poll_status", "omnitide_last_error",
     "omnitide_score_units", "omnitide_select_units", "omnitide_plan_structural", "omnipage_compact", "omnipage_migrate_suffix", "omnipage_migrate_class", "omnipage_compact_units", "omnipage_compact_units_rope", "omnipage_compact_units_batched", "omnipage_append",
-    "omnitide_chunk_attention", "omnitide_chunk_attention_masked", "omnitide_chunk_step", "omnitide_chunk_step_host", "omnitide_chunk_step_structural",
+    "omnitide_chunk_attention", "omnitide_chunk_attention_masked", "omnitide_chunk_step", "omnitide_chunk_step_host", "omnitide_chunk_step_host_pipelined", "omnitide_host_wait", "omnitide_chunk_step_structural",
     "omnitide_set_option", "omnitide_launch_count", "omnitide_score_units_noalloc",
 ]
 NOALLOC_MAX_UNITS = 1024
@@ -97,6 +97,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.omnitide_chunk_step_structural.argtypes = [vp, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp, i32, vp, vp, i32,
                                                    C.POINTER(StructuralParams), i32, f32, vp, vp, vp, vp, vp, vp, i32, vp]
     lib.omnitide_chunk_step_host.argtypes = step
+    lib.omnitide_chunk_step_host_pipelined.argtypes = step
+    lib.omnitide_host_wait.argtypes = [vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if name not in ("omnitide_last_error", "omnitide_launch_count"):
@@ -304,6 +306,12 @@ class Context:
 
     def chunk_step_host(self, *a, info_out=None):
         self._step(self.lib.omnitide_chunk_step_host, "omnitide_chunk_step_host", _host_ptr, *a, info_out)
+
+    def chunk_step_host_pipelined(self, *a, info_out=None):
+        self._step(self.lib.omnitide_chunk_step_host_pipelined, "omnitide_chunk_step_host_pipelined", _host_ptr, *a, info_out)
+
+    def host_wait(self):
+        self._check(self.lib.omnitide_host_wait(self._ctx), "omnitide_host_wait")
 
 
 def score_units_noalloc(h_q, h_kv, d, dtype, q, t, k_cache, n_hist, units, n_units, w_modality, scale, scores_out,

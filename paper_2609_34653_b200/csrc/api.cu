@@ -22,6 +22,15 @@ void free_all(omnitide_ctx* c) {
                     c->attn_n_live, c->mig_plan, c->dec_counter, c->mc_moves, c->mc_class};
     for (void* p : ptrs)
         if (p) cudaFree(p);
+    for (int b = 0; b < 2; ++b) {
+        void* pl[] = {c->pl_q[b], c->pl_k[b], c->pl_v[b], c->pl_o[b], c->pl_units[b]};
+        for (void* p : pl)
+            if (p) cudaFree(p);
+        cudaEvent_t evs[] = {c->pl_ev_q[b], c->pl_ev_kv[b], c->pl_ev_done[b], c->pl_ev_out[b]};
+        for (cudaEvent_t e : evs)
+            if (e) cudaEventDestroy(e);
+    }
+    if (c->pl_out) cudaStreamDestroy(c->pl_out);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     if (c->ev_kv) cudaEventDestroy(c->ev_kv);
     if (c->aux_stream) cudaStreamDestroy(c->aux_stream);
@@ -325,5 +334,82 @@ extern "C" omni_status omnitide_chunk_step_host(omnitide_ctx* ctx, void* stream,
     if (s) return s;
     const size_t o_bytes = (size_t)t * ctx->g.h_q * ctx->g.d * (out_dtype == OMNI_DTYPE_FP32 ? 4 : 2);
     OMNI_CUDA(ctx, cudaMemcpyAsync(o_host, ctx->st_o, o_bytes, cudaMemcpyDeviceToHost, st));
+    return OMNI_OK;
+}
+
+// Staging, stream and events of the pipelined host entry point (synchronous allocation on the first call).
+static omni_status pipeline_init(omnitide_ctx* ctx) {
+    if (ctx->pl_out) return OMNI_OK;
+    const omni_geometry& g = ctx->g;
+    const size_t q_elems = (size_t)g.t_cap * g.h_q * g.d;
+    for (int b = 0; b < 2; ++b) {
+        OMNI_CUDA(ctx, cudaMalloc(&ctx->pl_q[b], q_elems * ctx->es));
+        OMNI_CUDA(ctx, cudaMalloc(&ctx->pl_k[b], (size_t)g.t_cap * ctx->row_bytes));
+        OMNI_CUDA(ctx, cudaMalloc(&ctx->pl_v[b], (size_t)g.t_cap * ctx->row_bytes));
+        OMNI_CUDA(ctx, cudaMalloc(&ctx->pl_o[b], q_elems * 4));
+        OMNI_CUDA(ctx, cudaMalloc(reinterpret_cast<void**>(&ctx->pl_units[b]), 64 * sizeof(omni_unit)));
+        OMNI_CUDA(ctx, cudaEventCreateWithFlags(&ctx->pl_ev_q[b], cudaEventDisableTiming));
+        OMNI_CUDA(ctx, cudaEventCreateWithFlags(&ctx->pl_ev_kv[b], cudaEventDisableTiming));
+        OMNI_CUDA(ctx, cudaEventCreateWithFlags(&ctx->pl_ev_done[b], cudaEventDisableTiming));
+        OMNI_CUDA(ctx, cudaEventCreateWithFlags(&ctx->pl_ev_out[b], cudaEventDisableTiming));
+    }
+    OMNI_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->pl_out, cudaStreamNonBlocking));
+    return OMNI_OK;
+}
+
+extern "C" omni_status omnitide_chunk_step_host_pipelined(omnitide_ctx* ctx, void* stream, const void* q_host,
+                                                          const void* k_chunk_host, const void* v_chunk_host, int32_t t,
+                                                          const omni_unit* chunk_units_host, int32_t n_chunk_units,
+                                                          const void* k_cache, const void* v_cache, const int32_t* n_hist_dev,
+                                                          int32_t n_hist_max, const omni_unit* units, const int32_t* n_units_dev,
+                                                          int32_t n_units_max, const float* w_modality,
+                                                          const omni_select_params* params, int32_t page_size, float scale,
+                                                          void* k_cache_out, void* v_cache_out, omni_unit* units_out,
+                                                          int32_t* n_hist_out, int32_t* n_units_out, void* o_host,
+                                                          int32_t out_dtype, omni_compact_info* info_out) {
+    if (!ctx) return OMNI_ERR_INVALID_ARG;
+    if (!q_host || !k_chunk_host || !v_chunk_host || !o_host || (n_chunk_units > 0 && !chunk_units_host))
+        OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "chunk_step_host_pipelined: null pointer");
+    if (t <= 0 || t > ctx->g.t_cap) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "chunk_step_host_pipelined: t %d outside (0, t_cap]", t);
+    if (n_chunk_units < 0 || n_chunk_units > 64) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "chunk_step_host_pipelined: more than 64 chunk units");
+    const omni_status pi = pipeline_init(ctx);
+    if (pi) return pi;
+    cudaStream_t st = static_cast<cudaStream_t>(stream), in = ctx->aux_stream, out = ctx->pl_out;
+    const int b = (int)(ctx->pl_calls & 1);
+    const size_t q_bytes = (size_t)t * ctx->g.h_q * ctx->g.d * ctx->es;
+    const size_t kv_bytes = (size_t)t * ctx->row_bytes;
+    // uploads: behind the compute of the call before last, which read this buffer; ahead of everything else, so
+    // that they run under the previous call's kernels
+    OMNI_CUDA(ctx, cudaStreamWaitEvent(in, ctx->pl_ev_done[b], 0));
+    OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->pl_q[b], q_host, q_bytes, cudaMemcpyHostToDevice, in));
+    OMNI_CUDA(ctx, cudaEventRecord(ctx->pl_ev_q[b], in));
+    OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->pl_k[b], k_chunk_host, kv_bytes, cudaMemcpyHostToDevice, in));
+    OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->pl_v[b], v_chunk_host, kv_bytes, cudaMemcpyHostToDevice, in));
+    if (n_chunk_units)
+        OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->pl_units[b], chunk_units_host, sizeof(omni_unit) * n_chunk_units,
+                                       cudaMemcpyHostToDevice, in));
+    OMNI_CUDA(ctx, cudaEventRecord(ctx->pl_ev_kv[b], in));
+    // compute: behind Q and behind the download of the call before last, which read this output buffer
+    OMNI_CUDA(ctx, cudaStreamWaitEvent(st, ctx->pl_ev_q[b], 0));
+    OMNI_CUDA(ctx, cudaStreamWaitEvent(st, ctx->pl_ev_out[b], 0));
+    omni_status s = chunk_step_impl(ctx->pl_ev_kv[b], ctx, stream, ctx->pl_q[b], ctx->pl_k[b], ctx->pl_v[b], t, ctx->pl_units[b],
+                                    n_chunk_units, k_cache, v_cache, n_hist_dev, n_hist_max, units, n_units_dev, n_units_max,
+                                    w_modality, params, page_size, scale, k_cache_out, v_cache_out, units_out,
+                                    n_hist_out, n_units_out, ctx->pl_o[b], out_dtype, info_out);
+    if (s) return s;
+    OMNI_CUDA(ctx, cudaEventRecord(ctx->pl_ev_done[b], st));
+    // download on its own stream, under the next call's kernels
+    const size_t o_bytes = (size_t)t * ctx->g.h_q * ctx->g.d * (out_dtype == OMNI_DTYPE_FP32 ? 4 : 2);
+    OMNI_CUDA(ctx, cudaStreamWaitEvent(out, ctx->pl_ev_done[b], 0));
+    OMNI_CUDA(ctx, cudaMemcpyAsync(o_host, ctx->pl_o[b], o_bytes, cudaMemcpyDeviceToHost, out));
+    OMNI_CUDA(ctx, cudaEventRecord(ctx->pl_ev_out[b], out));
+    ctx->pl_calls++;
+    return OMNI_OK;
+}
+
+extern "C" omni_status omnitide_host_wait(omnitide_ctx* ctx) {
+    if (!ctx) return OMNI_ERR_INVALID_ARG;
+    OMNI_CUDA(ctx, cudaStreamSynchronize(ctx->aux_stream));
+    if (ctx->pl_out) OMNI_CUDA(ctx, cudaStreamSynchronize(ctx->pl_out));
     return OMNI_OK;
 }

@@ -42,6 +42,11 @@ struct omnitide_ctx {
     void* st_q; void* st_k; void* st_v; void* st_o; omni_unit* st_units;
     cudaStream_t aux_stream;      // carries the K/V chunk upload of chunk_step_host beside the scoring kernels
     cudaEvent_t ev_fork, ev_kv;
+    // double-buffered staging of omnitide_chunk_step_host_pipelined, allocated on first use
+    void* pl_q[2]; void* pl_k[2]; void* pl_v[2]; void* pl_o[2]; omni_unit* pl_units[2];
+    cudaStream_t pl_out;          // carries the downloads; the uploads ride on aux_stream
+    cudaEvent_t pl_ev_q[2], pl_ev_kv[2], pl_ev_done[2], pl_ev_out[2];
+    int64_t pl_calls;             // pipelined calls so far: call n uses buffer n & 1
     // attention split-KV partials
     float* attn_part_o;           // allocated on first use
     float* attn_part_ml;

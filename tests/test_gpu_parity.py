@@ -485,6 +485,67 @@ def test_chunk_step_small_mixed_and_host_entry(H, ob):
         _check_step(H, ob, w, _run_step(H, ob, w, host=True))
 
 
+def test_chunk_step_host_pipelined_stream(H, ob):
+    """Five chunks through omnitide_chunk_step_host_pipelined back to back, nothing waited for in between: every output
+    and the final cache equal, bit for bit, what the device entry point gives one call at a time.  Each chunk has its own
+    host buffers and values, so a staging buffer reused too early or a download taken too early shows."""
+    w = wl.small_mixed(31, d=128, n_units=10, max_len=350, t=280)
+    N, T, U = w.n_hist, w.t, len(w.units)
+    n_steps = 5
+    s_cap, u_cap = N + n_steps * T + 64, U + n_steps * len(w.chunk_units) + 4
+    rng = np.random.default_rng(5)
+    tdt = torch.bfloat16
+    params = ob.select_params(w.budget, w.n_recent_events, w.modality_cap)
+    chunks = []
+    for i in range(n_steps):
+        conv = lambda a: torch.from_numpy(a + 0.25 * rng.standard_normal(a.shape).astype(a.dtype)).to(tdt).contiguous()
+        cu = np.ascontiguousarray(w.chunk_units, dtype=np.int32).copy()
+        cu[:, oc.U_EVENT] += i                                  # later chunks are later events
+        chunks.append((conv(w.q), conv(w.k_chunk), conv(w.v_chunk), cu))
+
+    def run(pipelined):
+        ctx = ob.Context(w.h_q, w.h_kv, w.d, w.dtype, s_cap, u_cap, T)
+        caches = [[torch.zeros((s_cap, w.h_kv, w.d), dtype=tdt, device="cuda") for _ in range(2)] for _ in range(2)]
+        caches[0][0][:N] = ob.to_device(w.k_hist, w.dtype)
+        caches[0][1][:N] = ob.to_device(w.v_hist, w.dtype)
+        units = [ob.units_to_device(w.units, u_cap), torch.zeros((u_cap, 6), dtype=torch.int32, device="cuda")]
+        n_hist = [H.i32(N), H.i32(-1)]
+        n_units = [H.i32(U), H.i32(-1)]
+        outs, pinned = [], []
+        for i, (q, kc, vc, cu) in enumerate(chunks):
+            a, b = i & 1, (i + 1) & 1
+            if pipelined:
+                o = torch.empty((T, w.h_q, w.d), dtype=torch.float32).pin_memory()
+                pinned.append((q.pin_memory(), kc.pin_memory(), vc.pin_memory()))      # alive until host_wait
+                ctx.chunk_step_host_pipelined(*pinned[-1], T, cu, len(cu), caches[a][0], caches[a][1],
+                                              n_hist[a], s_cap - T, units[a], n_units[a], u_cap - len(cu), w.w_modality, params,
+                                              w.page_size, 0.0, caches[b][0], caches[b][1], units[b], n_hist[b], n_units[b], o,
+                                              ob.DTYPE_FP32)
+            else:
+                o = torch.empty((T, w.h_q, w.d), dtype=torch.float32, device="cuda")
+                ctx.chunk_step(q.cuda(), kc.cuda(), vc.cuda(), T, torch.from_numpy(cu).cuda(), len(cu), caches[a][0], caches[a][1],
+                               n_hist[a], s_cap - T, units[a], n_units[a], u_cap - len(cu), w.w_modality, params, w.page_size, 0.0,
+                               caches[b][0], caches[b][1], units[b], n_hist[b], n_units[b], o, ob.DTYPE_FP32)
+                torch.cuda.synchronize()
+            outs.append(o)
+        if pipelined:
+            ctx.host_wait()
+        torch.cuda.synchronize()
+        assert ctx.poll_status() == 0
+        last = n_steps & 1
+        nh = int(n_hist[last].item())
+        res = ([o.cpu().numpy().copy() for o in outs], nh, H.bytes_of(caches[last][0][:nh]).copy(), H.bytes_of(caches[last][1][:nh]).copy(),
+               units[last].cpu().numpy().copy(), int(n_units[last].item()))
+        ctx.close()
+        return res
+
+    ref, got = run(False), run(True)
+    assert got[1] == ref[1] and got[5] == ref[5]
+    for i in range(n_steps):
+        assert np.array_equal(got[0][i], ref[0][i]), f"output of chunk {i}"
+    assert np.array_equal(got[2], ref[2]) and np.array_equal(got[3], ref[3]) and np.array_equal(got[4][:got[5]], ref[4][:ref[5]])
+
+
 def test_chunk_step_config2(H, ob, cfg2):
     res = _run_step(H, ob, cfg2)
     _check_step(H, ob, cfg2, res)
