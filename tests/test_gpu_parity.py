@@ -1009,3 +1009,35 @@ def test_decode_attention_many_lengths(H, ob, h_q, h_kv):
     torch.cuda.synchronize()
     assert np.array_equal(o16.float().cpu().numpy(), wl.round_to_bf16(o.cpu().numpy()))
     ctx.close()
+
+
+@pytest.mark.parametrize("h_q,h_kv", [(32, 8), (8, 1), (64, 8), (8, 8), (4, 2)])
+def test_decode_attention_staged_long_histories(H, ob, h_q, h_kv):
+    """The same against a long cache bound (the split count is at its maximum): actual lengths from empty to the bound,
+    around the multiples of the split count and of the batch a warp takes per step."""
+    rng = np.random.default_rng(h_q * 100 + h_kv)
+    n_max = 21000
+    units = wl.make_units([(n_max, 0, 0)], group_of_first=None)
+    chunk_units = wl.make_units([(1, 0, 1)], group_of_first=None)
+    q, kh, vh, kc, vc = wl.random_layer_inputs(rng, units, chunk_units, h_q, h_kv, 128, "bf16")
+    ctx = ob.Context(h_q, h_kv, 128, "bf16", n_max + 64, 8, 4)
+    khd, vhd = ob.to_device(kh, "bf16"), ob.to_device(vh, "bf16")
+    qd, kcd, vcd = ob.to_device(q, "bf16"), ob.to_device(kc, "bf16"), ob.to_device(vc, "bf16")
+    n_split = min(64, max(1, 148 // h_kv))
+    lengths = [0, 1, 127, 128, 129, n_split - 1, n_split, n_split * 128 - 1, n_split * 128, n_split * 128 + 1, n_split * 384 - 1,
+               n_split * 384, n_split * 384 + 1, 8191, 16384, n_max - 1, n_max] + [int(x) for x in rng.integers(1, n_max, size=10)]
+    for n in lengths:
+        n = min(n, n_max)
+        o = torch.full((1, h_q, 128), float("nan"), dtype=torch.float32, device="cuda")
+        lse = torch.full((1, h_q), float("nan"), dtype=torch.float32, device="cuda")
+        ctx.chunk_attention(qd, 1, khd, vhd, H.i32(n), n_max, kcd, vcd, 0.0, o, ob.DTYPE_FP32, lse)
+        torch.cuda.synchronize()
+        assert ctx.poll_status() == 0
+        o_ref, lse_ref = oc.chunk_attention(q, kh[:n], vh[:n], kc, vc)
+        _check_attention(o.cpu().numpy(), lse.cpu().numpy(), o_ref, lse_ref)
+    o16 = torch.zeros((1, h_q, 128), dtype=torch.bfloat16, device="cuda")
+    ctx.chunk_attention(qd, 1, khd, vhd, H.i32(9999), n_max, kcd, vcd, 0.0, o16, ob.DTYPE_BF16)
+    ctx.chunk_attention(qd, 1, khd, vhd, H.i32(9999), n_max, kcd, vcd, 0.0, o, ob.DTYPE_FP32)
+    torch.cuda.synchronize()
+    assert np.array_equal(o16.float().cpu().numpy(), wl.round_to_bf16(o.cpu().numpy()))
+    ctx.close()
