@@ -911,6 +911,45 @@ def test_migrate_class_bit_exact(H, ob, S, page, sub, pattern, promote, seed):
     ctx.close()
 
 
+def test_migrate_class_argument_and_device_errors(H, ob):
+    """Host-side refusals (null pointers, a subblock that does not divide the page, a span above the capacity) and the
+    device-side one (a class value outside 0..2 sets OMNI_DEV_BAD_UNITS and moves nothing)."""
+    S = 512
+    ctx = ob.Context(8, 2, 128, "bf16", S + 64, 8, 16)
+    k = torch.zeros((S, 2, 128), dtype=torch.bfloat16, device="cuda")
+    v = torch.zeros_like(k)
+    mask = torch.ones(S + 16, dtype=torch.uint8, device="cuda")
+    mask[10:200] = 0
+    mask[230:256] = 0                                      # 30 entries left in page 3: moving them to page 0 empties it
+    cls = torch.full((S + 16,), 1 | 0x80, dtype=torch.uint8, device="cuda")
+    info = torch.full((8,), -5, dtype=torch.int32, device="cuda")
+    with pytest.raises(ob.OmniTideError):
+        ctx.migrate_class(k, v, None, cls, None, S, 64, 32, 1, None, None, info)
+    with pytest.raises(ob.OmniTideError):
+        ctx.migrate_class(k, v, mask, cls, None, S, 64, 48, 1, None, None, info)        # 48 does not divide 64
+    with pytest.raises(ob.OmniTideError):
+        ctx.migrate_class(k, v, mask, cls, None, S + 4096, 64, 32, 1, None, None, info)  # above s_cap
+    with pytest.raises(ob.OmniTideError):
+        ctx.migrate_class(k, v, mask, cls, None, S, 64, 32, 1, None, None, None)        # the outcome has to go somewhere
+    assert int(info[0].item()) == -5                       # nothing was launched
+    cls[300] = 3
+    before = mask.clone()
+    ctx.migrate_class(k, v, mask, cls, None, S, 64, 32, 1, None, None, info)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() & ob.DEV_BAD_UNITS
+    assert info.cpu().tolist() == [0] * 8 and torch.equal(mask, before)
+    # a device span above the host bound is refused on the device
+    cls[300] = 1
+    ctx.migrate_class(k, v, mask, cls, H.i32(S + 1), S, 64, 32, 1, None, None, info)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() & ob.DEV_BAD_COUNT and torch.equal(mask, before)
+    # and the same call with a valid span works afterwards: the context is still usable
+    ctx.migrate_class(k, v, mask, cls, H.i32(S), S, 64, 32, 1, None, None, info)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0 and info.cpu().tolist()[:2] == [1, 30] and not bool(mask[192:256].any())
+    ctx.close()
+
+
 def test_migrate_class_then_attention(H, ob, cfg2):
     """Attention over the class-migrated layout equals attention over the layout with its original holes: the migration
     changes where entries are stored, not the history (Section 6.2)."""
