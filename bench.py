@@ -171,6 +171,22 @@ def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=6
     hist_bound, units_bound = 16, 1
     o = torch.empty((t_cap, h_q, d), dtype=torch.float32, device="cuda")
     rows = []
+    shared = structural == "shared"
+    if shared:
+        # the paper's executor: ONE plan and ONE source -> destination map per chunk for the caches of all layers
+        ptrs = lambda ts: torch.tensor([t_.data_ptr() for t_ in ts], dtype=torch.int64, device="cuda")
+        pk = [ptrs([L["k"][i] for L in layers]) for i in range(2)]
+        pv = [ptrs([L["v"][i] for L in layers]) for i in range(2)]
+        sh_units = [layers[0]["units"][0], layers[0]["units"][1]]          # the unit table is the same for every layer
+        sh_n_units = [layers[0]["n_units"][0], layers[0]["n_units"][1]]
+        sh_n_hist = [layers[0]["n_hist"][0], layers[0]["n_hist"][1]]
+        sh_keep = torch.zeros(u_cap + 16, dtype=torch.uint8, device="cuda")
+        sh_klen = torch.zeros(u_cap + 16, dtype=torch.int32, device="cuda")
+        sh_nk, sh_nuk = torch.zeros(1, dtype=torch.int32, device="cuda"), torch.zeros(1, dtype=torch.int32, device="cuda")
+        sh_kept_units = torch.zeros((u_cap, 6), dtype=torch.int32, device="cuda")
+        dummy_units = torch.zeros((u_cap, 6), dtype=torch.int32, device="cuda")
+        dummy_cnt = [torch.zeros(1, dtype=torch.int32, device="cuda") for _ in range(2)]
+        sh_info = layers[0]["info"]
     for c, cu in enumerate(sched):
         T = int(cu[:, 1].sum())
         cu_dev = ob.units_to_device(cu)
@@ -182,7 +198,20 @@ def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=6
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         e0.record()
-        for l, L in enumerate(layers):
+        if shared:
+            ctx.plan_structural(sh_units[a], sh_n_units[a], units_bound, sparams, sh_keep, sh_klen, None, hist_bound, sh_nk,
+                                sh_kept_units, sh_nuk)
+            ctx.compact_units_batched(pk[a], pv[a], pk[b], pv[b], n_layers, sh_units[a], sh_n_units[a], units_bound, sh_keep,
+                                      hist_bound, page, sh_kept_units, sh_nuk, None, sh_info, None, unit_kept_len=sh_klen)
+            for l, L in enumerate(layers):
+                q, kc, vc = ins[l]
+                ctx.chunk_attention(q, T, L["k"][b], L["v"][b], sh_nk, hist_bound, kc, vc, 0.0, o, ob.DTYPE_FP32)
+                if l == 0:      # the shared unit table and counts advance once
+                    sh_units[b].copy_(sh_kept_units)
+                    ctx.append(L["k"][b], L["v"][b], sh_nk, kc, vc, T, sh_units[b], sh_nuk, cu_dev, len(cu), sh_n_hist[b], sh_n_units[b])
+                else:
+                    ctx.append(L["k"][b], L["v"][b], sh_nk, kc, vc, T, dummy_units, sh_nuk, cu_dev, len(cu), dummy_cnt[0], dummy_cnt[1])
+        for l, L in enumerate(layers if not shared else []):
             q, kc, vc = ins[l]
             if structural:
                 ctx.chunk_step_structural(q, kc, vc, T, cu_dev, len(cu), L["k"][a], L["v"][a], L["n_hist"][a], hist_bound,
@@ -195,12 +224,12 @@ def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=6
         e1.record()
         torch.cuda.synchronize()
         assert ctx.poll_status() == 0, "device status word not clean inside the stream loop"
-        infos = torch.stack([L["info"] for L in layers]).cpu().numpy()
-        n_hist_new = int(max(int(L["n_hist"][b].item()) for L in layers))
+        infos = torch.stack([L["info"] for L in (layers[:1] if shared else layers)]).cpu().numpy()
+        n_hist_new = int(max(int(L["n_hist"][b].item()) for L in (layers[:1] if shared else layers)))
         rows.append(dict(ms=e0.elapsed_time(e1), hist=hist_bound, t=T, kept=float(infos[:, 0].mean()),
                          span=float(infos[:, 1].mean()) * page, evicting=bool((infos[:, 0] < hist_bound).any())))
         hist_bound = n_hist_new
-        units_bound = int(max(int(L["n_units"][b].item()) for L in layers))
+        units_bound = int(max(int(L["n_units"][b].item()) for L in (layers[:1] if shared else layers)))
     launches = ctx.launch_count()
     ctx.close()
     # steady state: every chunk from the first retention round on (with watermarks most chunks have no round)
@@ -214,7 +243,8 @@ def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=6
             "span_slots_mean": float(np.mean([r["span"] for r in steady])),
             "span_over_kept": float(np.mean([r["span"] / max(r["kept"], 1.0) for r in steady])),
             "retention_rounds": int(sum(1 for r in steady if r["evicting"])),
-            "gpu_launches": int(launches), "selection": "structural (score-free)" if structural else
+            "gpu_launches": int(launches), "selection": ("structural (score-free), one plan and one batched compaction for all layers" if shared
+                                                          else "structural (score-free)") if structural else
             (f"scored by the last {score_window} queries of the chunk" if score_window else "scored by every query of the chunk"),
             "note": "36 layer steps per chunk timed with CUDA events; chunks counted from the first retention round on"}
 
@@ -686,6 +716,9 @@ def main():
         loop_s = run_stream_loop(ob, torch, args.loop_chunks, rank, structural=True)
         loop_s["ms_per_chunk"] = max_over_ranks([loop_s["ms_per_chunk"]], world, "cuda")[0]
         line["stream_loop_structural"] = loop_s
+        loop_sh = run_stream_loop(ob, torch, args.loop_chunks, rank, structural="shared")
+        loop_sh["ms_per_chunk"] = max_over_ranks([loop_sh["ms_per_chunk"]], world, "cuda")[0]
+        line["stream_loop_structural_shared"] = loop_sh
         loop_w = run_stream_loop(ob, torch, args.loop_chunks, rank, score_window=128)
         loop_w["ms_per_chunk"] = max_over_ranks([loop_w["ms_per_chunk"]], world, "cuda")[0]
         line["stream_loop_window128"] = loop_w

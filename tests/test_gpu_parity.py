@@ -1080,3 +1080,68 @@ def test_decode_attention_staged_long_histories(H, ob, h_q, h_kv):
     torch.cuda.synchronize()
     assert np.array_equal(o16.float().cpu().numpy(), wl.round_to_bf16(o.cpu().numpy()))
     ctx.close()
+
+
+def test_shared_plan_over_layers_equals_per_layer_steps(H, ob, cfg2):
+    """One structural plan and one batched compaction for the caches of two layers, then attention and append per layer
+    (the paper's executor: one map shared by all layers, Section 6.2), against omnitide_chunk_step_structural run on each
+    layer by itself: outputs, caches, unit table and counts bit for bit."""
+    w = cfg2
+    N, T, U = w.n_hist, w.t, len(w.units)
+    s_cap, u_cap = N + T + 64, U + len(w.chunk_units) + 4
+    sp = ob.structural_params(6000, 4000, 2, (24, 8, 0), 64)
+    rng = np.random.default_rng(8)
+    tdt = torch.bfloat16
+    mk = lambda a: torch.from_numpy(wl.round_to_bf16(a + 0.5 * rng.standard_normal(a.shape).astype(np.float32))).to(tdt).cuda()
+    layers = [dict(k=mk(w.k_hist), v=mk(w.v_hist), q=mk(w.q), kc=mk(w.k_chunk), vc=mk(w.v_chunk)) for _ in range(2)]
+    cu = ob.units_to_device(w.chunk_units)
+
+    def fresh_cache(L):
+        k = torch.zeros((s_cap, w.h_kv, w.d), dtype=tdt, device="cuda")
+        v = torch.zeros_like(k)
+        k[:N], v[:N] = L["k"], L["v"]
+        return k, v
+
+    # ---- reference: the fused per-layer entry point
+    ref = []
+    ctx = ob.Context(w.h_q, w.h_kv, w.d, w.dtype, s_cap, u_cap, T)
+    for L in layers:
+        k_in, v_in = fresh_cache(L)
+        k_out, v_out = torch.zeros_like(k_in), torch.zeros_like(v_in)
+        units_out = torch.zeros((u_cap, 6), dtype=torch.int32, device="cuda")
+        nh, nu = H.i32(-1), H.i32(-1)
+        o = torch.zeros((T, w.h_q, w.d), dtype=torch.float32, device="cuda")
+        ctx.chunk_step_structural(L["q"], L["kc"], L["vc"], T, cu, len(w.chunk_units), k_in, v_in, H.i32(N), N,
+                                  ob.units_to_device(w.units, u_cap), H.i32(U), U, sp, w.page_size, 0.0, k_out, v_out, units_out,
+                                  nh, nu, o, ob.DTYPE_FP32)
+        torch.cuda.synchronize()
+        ref.append(dict(o=o.cpu().numpy(), nh=int(nh.item()), nu=int(nu.item()), k=k_out, v=v_out, units=units_out.cpu().numpy()))
+    assert ctx.poll_status() == 0 and ref[0]["nh"] < N + T                     # the plan evicts
+    # ---- one plan, one batched compaction, then per layer attention + append
+    ins = [fresh_cache(L) for L in layers]
+    outs = [(torch.zeros_like(a), torch.zeros_like(b)) for a, b in ins]
+    ptrs = lambda ts: torch.tensor([t_.data_ptr() for t_ in ts], dtype=torch.int64, device="cuda")
+    units_in = ob.units_to_device(w.units, u_cap)
+    keep = torch.zeros(u_cap + 16, dtype=torch.uint8, device="cuda")
+    klen = torch.zeros(u_cap + 16, dtype=torch.int32, device="cuda")
+    n_kept, n_uk = H.i32(-1), H.i32(-1)
+    kept_units = torch.zeros((u_cap, 6), dtype=torch.int32, device="cuda")
+    info = torch.zeros(8, dtype=torch.int32, device="cuda")
+    ctx.plan_structural(units_in, H.i32(U), U, sp, keep, klen, None, N, n_kept, kept_units, n_uk)
+    ctx.compact_units_batched(ptrs([a for a, _ in ins]), ptrs([b for _, b in ins]), ptrs([a for a, _ in outs]),
+                              ptrs([b for _, b in outs]), 2, units_in, H.i32(U), U, keep, N, w.page_size, kept_units, n_uk, None,
+                              info, None, unit_kept_len=klen)
+    for i, L in enumerate(layers):
+        o = torch.zeros((T, w.h_q, w.d), dtype=torch.float32, device="cuda")
+        ctx.chunk_attention(L["q"], T, outs[i][0], outs[i][1], n_kept, N, L["kc"], L["vc"], 0.0, o, ob.DTYPE_FP32)
+        table = kept_units.clone()
+        nh, nu = H.i32(-1), H.i32(-1)
+        ctx.append(outs[i][0], outs[i][1], n_kept, L["kc"], L["vc"], T, table, n_uk, cu, len(w.chunk_units), nh, nu)
+        torch.cuda.synchronize()
+        assert ctx.poll_status() == 0
+        assert (int(nh.item()), int(nu.item())) == (ref[i]["nh"], ref[i]["nu"])
+        assert np.array_equal(o.cpu().numpy(), ref[i]["o"])
+        n_new = ref[i]["nh"]
+        assert torch.equal(outs[i][0][:n_new], ref[i]["k"][:n_new]) and torch.equal(outs[i][1][:n_new], ref[i]["v"][:n_new])
+        assert np.array_equal(table[:ref[i]["nu"]].cpu().numpy(), ref[i]["units"][:ref[i]["nu"]])
+    ctx.close()
