@@ -701,9 +701,17 @@ def main():
         assert ctx.poll_status() == 0, "device status word not clean after the per-layer compaction loop"
         pl_ms = max_over_ranks([float(np.mean([a_.elapsed_time(b_) for a_, b_ in bevs]))], world, "cuda")[0] / L
         pl_gbs = work["compact_bytes"] / (pl_ms * 1e-3) / 1e9
-        line["kernels"]["compact"]["back_to_back"] = {
-            "ms_per_launch": pl_ms, "achieved": pl_gbs, "frac": pl_gbs / peaks["hbm_gbs"], "launches_per_event_pair": L,
-            "note": "omnipage_compact_units on the caches of successive layers, the launches replayed from one CUDA graph inside one event pair"}
+        # the per-layer kernel is reported by its average launch duration over this region (the model runs it once per layer,
+        # back to back); the figure of one launch between its own two events stays beside it
+        cpk = line["kernels"]["compact"]
+        cpk["single_launch"] = {"ms": cpk["ms"], "achieved": cpk["achieved"], "frac": cpk["frac"],
+                                "note": "one launch between its own two CUDA events; an empty kernel measures 5-6 us there"}
+        cpk.update(ms=pl_ms, achieved=pl_gbs, frac=pl_gbs / peaks["hbm_gbs"], frac_of_nominal=pl_gbs / NOMINAL["hbm_gbs"],
+                   launches_per_event_pair=L,
+                   timing=f"average launch duration over {L} launches on the caches of successive layers, replayed from one CUDA graph "
+                          "inside one event pair (the step total above uses the single-launch time)")
+        line["compaction_single_launch_gbs"] = line["compaction_gbs"]
+        line["compaction_gbs"] = pl_gbs * world
         line["compaction_batched_gbs"] = b_gbs * world
         del k_src, v_src, k_dst, v_dst
     ctx.close()

@@ -309,6 +309,10 @@ __global__ void __launch_bounds__(CP_THREADS, 1) compact_pack_kernel(const Compa
     __shared__ int abort_flag;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int G = gridDim.x;
+    // Launched as a programmatic dependent, the grid is scheduled while the kernel before it drains; nothing is read
+    // before that kernel has completed and its writes are visible.  The next launch of this kind may be scheduled at once.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // ---- prologue: every load whose address needs no device-side count is issued before anything waits ----
     const int part_bytes = a.part_groups * 512;
@@ -1086,7 +1090,16 @@ static omni_status compact_units_impl(const omni_rope_params* rope, omnitide_ctx
     const size_t smem = smem_lists_al + (size_t)a.n_slots * CP_WARPS * ctx->row_bytes;
     if (smem > 48 * 1024)
         OMNI_CUDA(ctx, cudaFuncSetAttribute(compact_units_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    compact_units_kernel<false><<<grid, CP_THREADS, smem, st>>>(a);
+    {
+        // programmatic stream serialisation: the launch latency of this kernel hides behind the tail of the previous one
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(CP_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        OMNI_CUDA(ctx, cudaLaunchKernelEx(&cfg, compact_units_kernel<false>, a));
+    }
     OMNI_CHECK_LAUNCH(ctx, "compact_units_kernel");
     if (in_place) {
         copy_rows_kernel<<<ctx->sm_count * 4, 256, 0, st>>>(
