@@ -107,9 +107,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int b0 = split * bps, b1 = min(nkb, b0 + bps);
     const int nb = b1 - b0;
     if (nb <= 0) return;
-    bool active[NT];
+    uint32_t active_bits = 0;                  // bit tt: tile slot tt of this CTA holds a (row tile, head) pair
 #pragma unroll
-    for (int tt = 0; tt < NT; ++tt) active[tt] = row_of(tt) < p.n_row_tiles;
+    for (int tt = 0; tt < NT; ++tt) active_bits |= (uint32_t)(row_of(tt) < p.n_row_tiles) << tt;
+    auto is_active = [&](int tt) { return ((active_bits >> tt) & 1u) != 0; };
 
     for (int u = threadIdx.x; u < n_units; u += SC_THREADS) unit_end[u] = p.units[u].start + p.units[u].len;
     if (threadIdx.x == 0) {
@@ -136,10 +137,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             tc::tma_prefetch_desc(&tm_q);
             tc::tma_prefetch_desc(&tm_k);
             int n_active = 0;
-            for (int tt = 0; tt < NT; ++tt) n_active += (int)active[tt];
+            for (int tt = 0; tt < NT; ++tt) n_active += (int)is_active(tt);
             tc::mbar_expect_tx(tc::smem_u32(&bars->q_full), n_active * TILE_BYTES);
             for (int tt = 0; tt < NT; ++tt) {
-                if (!active[tt]) continue;
+                if (!is_active(tt)) continue;
                 const int row0 = row_of(tt) * BLK, head = head_of(tt);
                 tc::tma_load_2d(q_smem + tt * TILE_BYTES, &tm_q, head * HD, row0, tc::smem_u32(&bars->q_full));
                 tc::tma_load_2d(q_smem + tt * TILE_BYTES + HALF_BYTES, &tm_q, head * HD + 64, row0, tc::smem_u32(&bars->q_full));
@@ -165,20 +166,21 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
     } else if (warp == 4 * NT) {
         if (lane == 0) {
+            const uint64_t q_desc0 = tc::umma_smem_desc(q_smem, 16, 1024), k_desc0 = tc::umma_smem_desc(k_smem, 16, 1024);
             bool ok = tc::mbar_wait(tc::smem_u32(&bars->q_full), 0, abort_flag);
             for (int j = 0; j < nb && ok; ++j) {
                 const int stage = j % NSTAGE;
                 ok = tc::mbar_wait(tc::smem_u32(&bars->k_full[stage]), (j / NSTAGE) & 1, abort_flag);
                 for (int tt = 0; tt < NT && ok; ++tt) {
-                    if (!active[tt]) continue;
+                    if (!is_active(tt)) continue;
                     ok = tc::mbar_wait(tc::smem_u32(&bars->s_empty[tt]), (j & 1) ^ 1, abort_flag);
                     tc::tcgen05_fence_after();
-                    const uint32_t a0 = q_smem + tt * TILE_BYTES, bb = k_smem + stage * TILE_BYTES;
+                    // descriptors differ from the tile's first one only in the address field (16-byte units; no carry out of it)
+                    const uint64_t a_desc = q_desc0 + (uint64_t)((tt * TILE_BYTES) >> 4), b_desc = k_desc0 + (uint64_t)((stage * TILE_BYTES) >> 4);
 #pragma unroll
                     for (int kk = 0; kk < HD / 16; ++kk) {
                         const uint32_t off = (kk >> 2) * HALF_BYTES + (kk & 3) * 32;
-                        tc::umma_ss(tmem + tt * 128, tc::umma_smem_desc(a0 + off, 16, 1024),
-                                    tc::umma_smem_desc(bb + off, 16, 1024), IDESC_QK, kk > 0, 1u);
+                        tc::umma_ss(tmem + tt * 128, a_desc + (off >> 4), b_desc + (off >> 4), IDESC_QK, kk > 0, 1u);
                     }
                     tc::umma_commit(tc::smem_u32(&bars->s_full[tt]));
                 }
@@ -187,7 +189,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
     } else {
         const int tt = warp >> 2;
-        if (active[tt]) {
+        if (is_active(tt)) {
             const int r = (warp & 3) * 32 + lane;
             const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
             const int tile = head_of(tt) * p.n_row_tiles + row_of(tt);
