@@ -289,10 +289,15 @@ __device__ __forceinline__ uint4 mask_at(const uint8_t* mask, int pos, int s) {
 __global__ void __launch_bounds__(CP_THREADS, 1) compact_pack_kernel(const CompactArgs a_in) {
     CompactArgs a = a_in;
     int span_off = 0;
+    bool empty_span = false;
     if (a_in.span_off_dev) {
         const int s_all = a_in.s_span_dev ? __ldg(a_in.s_span_dev) : a_in.s_span_max;
         span_off = __ldg(a_in.span_off_dev);
-        if (span_off < 0 || span_off > s_all) span_off = max(0, min(s_all, a_in.s_span_max));   // nothing to pack: an empty span
+        if (span_off < 0 || span_off >= s_all) {
+            // nothing to pack: an empty span at an offset that keeps the 16-byte mask loads and slot-map stores aligned
+            empty_span = true;
+            span_off = max(0, min(s_all, a_in.s_span_max)) & ~15;
+        }
         a.mask += span_off;
         if (a.k_src) { a.k_src += (size_t)span_off * a.row_bytes; a.v_src += (size_t)span_off * a.row_bytes; }
         if (a.slot_map) a.slot_map += span_off;
@@ -309,10 +314,6 @@ __global__ void __launch_bounds__(CP_THREADS, 1) compact_pack_kernel(const Compa
     __shared__ int abort_flag;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int G = gridDim.x;
-    // Launched as a programmatic dependent, the grid is scheduled while the kernel before it drains; nothing is read
-    // before that kernel has completed and its writes are visible.  The next launch of this kind may be scheduled at once.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // ---- prologue: every load whose address needs no device-side count is issued before anything waits ----
     const int part_bytes = a.part_groups * 512;
@@ -322,6 +323,7 @@ __global__ void __launch_bounds__(CP_THREADS, 1) compact_pack_kernel(const Compa
     uint4 mv = make_uint4(0, 0, 0, 0);                                // its first group stays in registers
     if (wg0 < wg1 && my_base + wg0 * 512 + lane * 16 < a.s_span_max) mv = ld_mask(a.mask, (my_base + wg0 * 512) / 16 + lane);
     int s = a.s_span_dev ? __ldg(a.s_span_dev) - span_off : a.s_span_max;
+    if (empty_span) s = 0;
     int nu = 0, u_len = 0, u_group = -1;
     if (a.units_kept) {
         nu = a.n_units_kept_dev ? __ldg(a.n_units_kept_dev) : a.n_units_max;
@@ -1090,16 +1092,7 @@ static omni_status compact_units_impl(const omni_rope_params* rope, omnitide_ctx
     const size_t smem = smem_lists_al + (size_t)a.n_slots * CP_WARPS * ctx->row_bytes;
     if (smem > 48 * 1024)
         OMNI_CUDA(ctx, cudaFuncSetAttribute(compact_units_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    {
-        // programmatic stream serialisation: the launch latency of this kernel hides behind the tail of the previous one
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(CP_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
-        OMNI_CUDA(ctx, cudaLaunchKernelEx(&cfg, compact_units_kernel<false>, a));
-    }
+    compact_units_kernel<false><<<grid, CP_THREADS, smem, st>>>(a);
     OMNI_CHECK_LAUNCH(ctx, "compact_units_kernel");
     if (in_place) {
         copy_rows_kernel<<<ctx->sm_count * 4, 256, 0, st>>>(
