@@ -249,6 +249,71 @@ def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=6
             "note": "36 layer steps per chunk timed with CUDA events; chunks counted from the first retention round on"}
 
 
+def run_sweep(ob, torch, peaks, tensor_peak, rank, reps=3):
+    """The stress grid: 131,072-token history of 2,304-token frames and 25 tok/s audio, heavy-tailed per-head key scales
+    (Student-t, nu = 3), chunk sizes {256, 1024, 4096} x retention ratios {5, 12.5, 25, 50 %} x page sizes {16, 64, 256}.
+    Per cell: scoring, selection, unit-granular compaction and chunk attention, each between its own CUDA events (mean
+    of `reps` after one warm-up); K/V of the cell are 0.5 GB, larger than L2."""
+    from paper_2609_34653_b200 import workloads as wl
+    h_q, h_kv, d, n_hist = 32, 8, 128, 131072
+    gen = torch.Generator(device="cuda").manual_seed(7000 + rank)
+    t_scale = torch.distributions.StudentT(torch.tensor(3.0)).sample((h_kv,)).abs().clamp(0.05, 20.0).cuda()
+    k_in = (torch.randn((n_hist + 64, h_kv, d), generator=gen, device="cuda") * t_scale[None, :, None]).to(torch.bfloat16)
+    v_in = torch.randn((n_hist + 64, h_kv, d), generator=gen, device="cuda").to(torch.bfloat16)
+    k_out, v_out = torch.empty_like(k_in), torch.empty_like(v_in)
+    cells = []
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    for t in (256, 1024, 4096):
+        q = torch.randn((t, h_q, d), generator=gen, device="cuda").to(torch.bfloat16)
+        kc = (torch.randn((t, h_kv, d), generator=gen, device="cuda") * t_scale[None, :, None]).to(torch.bfloat16)
+        vc = torch.randn((t, h_kv, d), generator=gen, device="cuda").to(torch.bfloat16)
+        o = torch.empty((t, h_q, d), dtype=torch.float32, device="cuda")
+        for ratio in (0.05, 0.125, 0.25, 0.5):
+            for page in (16, 64, 256):
+                w = wl.sweep_cell(t, ratio, page, cell=len(cells), draw_values=False)
+                U = len(w.units)
+                ctx = ob.Context(h_q, h_kv, d, "bf16", n_hist + 64, U + 8, t)
+                units = ob.units_to_device(w.units, U + 8)
+                n_units_dev = torch.tensor([U], dtype=torch.int32, device="cuda")
+                n_hist_dev = torch.tensor([n_hist], dtype=torch.int32, device="cuda")
+                scores = torch.zeros(U + 8, dtype=torch.float32, device="cuda")
+                keep = torch.zeros(U + 24, dtype=torch.uint8, device="cuda")
+                n_kept, n_uk = torch.zeros(1, dtype=torch.int32, device="cuda"), torch.zeros(1, dtype=torch.int32, device="cuda")
+                units_out = torch.zeros((U + 8, 6), dtype=torch.int32, device="cuda")
+                info = torch.zeros(8, dtype=torch.int32, device="cuda")
+                params = ob.select_params(w.budget, w.n_recent_events, w.modality_cap)
+                acc = {"score": 0.0, "select": 0.0, "compact": 0.0, "attention": 0.0}
+                for i in range(1 + reps):
+                    e = [ev() for _ in range(5)]
+                    e[0].record()
+                    ctx.score_units(q, t, k_in, n_hist_dev, n_hist, units, n_units_dev, U, w.w_modality, 0.0, scores)
+                    e[1].record()
+                    ctx.select_units(units, n_units_dev, U, scores, params, keep, None, n_hist, n_kept, units_out, n_uk)
+                    e[2].record()
+                    ctx.compact_units(k_in, v_in, k_out, v_out, units, n_units_dev, U, keep, n_hist, page, units_out, n_uk, None, info, None)
+                    e[3].record()
+                    ctx.chunk_attention(q, t, k_out, v_out, n_kept, n_hist, kc, vc, 0.0, o, ob.DTYPE_FP32)
+                    e[4].record()
+                    torch.cuda.synchronize()
+                    if i:
+                        for j, name in enumerate(acc):
+                            acc[name] += e[j].elapsed_time(e[j + 1]) / reps
+                assert ctx.poll_status() == 0, "device status word not clean in the sweep"
+                kept = int(n_kept.item())
+                span = int(info[1].item()) * page
+                ctx.close()
+                att_flop = 4.0 * d * h_q * (t * kept + t * (t + 1) / 2.0)
+                cp_bytes = 2.0 * kept * 2 * h_kv * d * 2 + 25.0 * U
+                att_tf, cp_gbs = att_flop / (acc["attention"] * 1e-3) / 1e12, cp_bytes / (acc["compact"] * 1e-3) / 1e9
+                cells.append({"t": t, "ratio": ratio, "page": page, "kept": kept, "span": span,
+                              "attention_ms": acc["attention"], "attention_tflops": att_tf, "attention_frac": att_tf / tensor_peak,
+                              "compact_ms": acc["compact"], "compact_gbs": cp_gbs, "compact_frac": cp_gbs / peaks["hbm_gbs"],
+                              "score_ms": acc["score"], "select_ms": acc["select"]})
+    return {"cells": cells, "history": n_hist,
+            "note": "per-cell kernel times between their own CUDA events; fractions of the measured sustained bf16 peak and of the "
+                    "measured copy bandwidth; short kernels carry the 5-6 us an event pair costs"}
+
+
 def run_reference(args, rank, world):
     """CPU oracle timed on a bounded sample of the same workload (rank 0 only)."""
     if rank != 0:
@@ -295,6 +360,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--mask-compaction", action="store_true",
                     help="time omnipage_compact (token keep mask + slot map) instead of the unit-granular entry point")
+    ap.add_argument("--no-sweep", dest="sweep", action="store_false", help="skip the 36-cell stress grid (131,072-token history)")
     ap.add_argument("--no-ablation", dest="ablation", action="store_false",
                     help="skip the native / class-aware / ordered-suffix / eager layout ablation")
     ap.add_argument("--batch-layers", type=int, default=36,
@@ -717,6 +783,8 @@ def main():
     ctx.close()
     del sets
     torch.cuda.empty_cache()
+    if args.sweep:
+        line["sweep"] = run_sweep(ob, torch, peaks, tensor_peak, rank)
     if args.loop_chunks > 0:
         loop = run_stream_loop(ob, torch, args.loop_chunks, rank)
         loop["ms_per_chunk"] = max_over_ranks([loop["ms_per_chunk"]], world, "cuda")[0]
