@@ -145,7 +145,9 @@ def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=6
     region) and the physical span against the kept count."""
     from paper_2609_34653_b200 import workloads as wl
     sched = wl.loop_schedule(n_chunks)
-    h_q, h_kv, d, t_cap, u_cap = 32, 8, 128, 2432, 96
+    # the score-free plan keeps a short prefix of every old span, so its unit table grows with the stream (about two
+    # units per surviving event); the scored selection drops whole units and stays small
+    h_q, h_kv, d, t_cap, u_cap = 32, 8, 128, 2432, (768 if structural else 96)
     s_cap = ((budget + 2 * t_cap + 255) // 256) * 256
     ctx = ob.Context(h_q, h_kv, d, "bf16", s_cap, u_cap, t_cap)
     if score_window:
@@ -365,7 +367,7 @@ def main():
                     help="skip the native / class-aware / ordered-suffix / eager layout ablation")
     ap.add_argument("--batch-layers", type=int, default=36,
                     help="layers packed by one launch of the cross-layer batched compaction (0: skip it)")
-    ap.add_argument("--loop-chunks", type=int, default=40, help="chunks of the 36-layer stream loop (0: skip it)")
+    ap.add_argument("--loop-chunks", type=int, default=400, help="chunks of the 36-layer stream loop (0: skip it)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
