@@ -137,7 +137,8 @@ def whole_job(per_replica_value, world):
     return per_replica_value * world
 
 
-def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=64, structural=False, score_window=0):
+def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=64, structural=False, score_window=0,
+                    high_watermark=0):
     """The 36-layer stream loop (frames of {640, 1280, 2304} tokens plus 2 s of audio at 10-25 tok/s per
     chunk): per chunk and per layer one omnitide_chunk_step on a device-resident cache.  Returns the
     mean milliseconds per chunk over the chunks whose history already exceeds the budget (CUDA events
@@ -148,10 +149,14 @@ def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=6
     # the score-free plan keeps a short prefix of every old span, so its unit table grows with the stream (about two
     # units per surviving event); the scored selection drops whole units and stays small
     h_q, h_kv, d, t_cap, u_cap = 32, 8, 128, 2432, (768 if structural else 96)
-    s_cap = ((budget + 2 * t_cap + 255) // 256) * 256
+    s_cap = ((max(budget, high_watermark) + 2 * t_cap + 255) // 256) * 256
     ctx = ob.Context(h_q, h_kv, d, "bf16", s_cap, u_cap, t_cap)
     if score_window:
         ctx.set_option(ob.OPT_SCORE_WINDOW, score_window)
+    if high_watermark:
+        # hysteresis for the scored pass: a retention round (scoring included) only when the history exceeds the
+        # high watermark; it trims to the budget (the low watermark)
+        ctx.set_option(ob.OPT_HIGH_WATERMARK, high_watermark)
     gen = torch.Generator(device="cuda").manual_seed(4000 + rank)
     randn = lambda *shape: torch.randn(*shape, generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
     prefix = wl.loop_prefix_units()
@@ -229,7 +234,7 @@ def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=6
         infos = torch.stack([L["info"] for L in (layers[:1] if shared else layers)]).cpu().numpy()
         n_hist_new = int(max(int(L["n_hist"][b].item()) for L in (layers[:1] if shared else layers)))
         rows.append(dict(ms=e0.elapsed_time(e1), hist=hist_bound, t=T, kept=float(infos[:, 0].mean()),
-                         span=float(infos[:, 1].mean()) * page, evicting=bool((infos[:, 0] < hist_bound).any())))
+                         span=float(infos[:, 1].mean()) * page, evicting=(hist_bound > high_watermark) if high_watermark else bool((infos[:, 0] < hist_bound).any())))
         hist_bound = n_hist_new
         units_bound = int(max(int(L["n_units"][b].item()) for L in (layers[:1] if shared else layers)))
     launches = ctx.launch_count()
@@ -237,7 +242,9 @@ def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=6
     # steady state: every chunk from the first retention round on (with watermarks most chunks have no round)
     first = next((i for i, r in enumerate(rows) if r["evicting"]), len(rows) // 2)
     steady = rows[first:] or rows[-1:]
-    return {"ms_per_chunk": float(np.mean([r["ms"] for r in steady])), "layers": n_layers, "chunks": len(rows),
+    ms = np.array([r["ms"] for r in steady])
+    return {"ms_per_chunk": float(ms.mean()), "ms_per_chunk_p50": float(np.percentile(ms, 50)),
+            "ms_per_chunk_p99": float(np.percentile(ms, 99)), "layers": n_layers, "chunks": len(rows),
             "chunks_timed": len(steady), "budget": budget, "page": page,
             "mean_chunk_tokens": float(np.mean([r["t"] for r in steady])),
             "mean_history_tokens": float(np.mean([r["hist"] for r in steady])),
@@ -247,7 +254,8 @@ def run_stream_loop(ob, torch, n_chunks, rank, n_layers=36, budget=12288, page=6
             "retention_rounds": int(sum(1 for r in steady if r["evicting"])),
             "gpu_launches": int(launches), "selection": ("structural (score-free), one plan and one batched compaction for all layers" if shared
                                                           else "structural (score-free)") if structural else
-            (f"scored by the last {score_window} queries of the chunk" if score_window else "scored by every query of the chunk"),
+            ((f"scored by the last {score_window} queries of the chunk" if score_window else "scored by every query of the chunk")
+             + (f", rounds only above {high_watermark} history tokens" if high_watermark else "")),
             "note": "36 layer steps per chunk timed with CUDA events; chunks counted from the first retention round on"}
 
 
@@ -800,6 +808,10 @@ def main():
         loop_w = run_stream_loop(ob, torch, args.loop_chunks, rank, score_window=128)
         loop_w["ms_per_chunk"] = max_over_ranks([loop_w["ms_per_chunk"]], world, "cuda")[0]
         line["stream_loop_window128"] = loop_w
+        # the paper's 2500 / 1800 watermark ratio around the same budget
+        loop_h = run_stream_loop(ob, torch, args.loop_chunks, rank, high_watermark=int(12288 / 0.72))
+        loop_h["ms_per_chunk"] = max_over_ranks([loop_h["ms_per_chunk"]], world, "cuda")[0]
+        line["stream_loop_watermarks"] = loop_h
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import omni_oracle as oc
         import threadpoolctl

@@ -491,8 +491,13 @@ omni_status omnitide_score_units_noalloc(void* stream, int32_t h_q, int32_t h_kv
  * kernels even where the tensor-core kernels apply (a second implementation for cross-checks).
  * OMNI_OPT_SCORE_WINDOW = W > 0 makes omnitide_chunk_step (and its host form) score the history with the last W
  * queries of the chunk only, a trailing observation window as in the score-based methods the paper cites (Section 3);
- * 0 (default) scores with every query.  A caller of omnitide_score_units gets the same by passing that row range. */
-enum { OMNI_OPT_FORCE_CUDA_CORES = 1, OMNI_OPT_SCORE_WINDOW = 2 };
+ * 0 (default) scores with every query.  A caller of omnitide_score_units gets the same by passing that row range.
+ * OMNI_OPT_HIGH_WATERMARK = H > 0 gives omnitide_chunk_step (and its host forms) the paper's hysteresis (Section 5.1:
+ * retention starts only above a high watermark and trims to the low one, here the selection budget): a call whose
+ * n_hist_max is at most H launches no scoring kernel and keeps every unit (the history is copied whole to the output
+ * cache); a call whose bound exceeds H runs the full pass.  The decision is the host's, from the bound it was given,
+ * so a caller that wants rounds to be rare passes a tight n_hist_max.  0 (default): every call runs the full pass. */
+enum { OMNI_OPT_FORCE_CUDA_CORES = 1, OMNI_OPT_SCORE_WINDOW = 2, OMNI_OPT_HIGH_WATERMARK = 3 };
 omni_status omnitide_set_option(omnitide_ctx* ctx, int32_t option, int32_t value);
 
 /* Number of kernels this library has launched on this context since creation (for accounting). */

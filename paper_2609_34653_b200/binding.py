@@ -20,6 +20,7 @@ DEV_TIMEOUT, DEV_BAD_UNITS, DEV_BAD_COUNT = 1, 2, 4
 DTYPE_BF16, DTYPE_FP32 = 0, 1
 OPT_FORCE_CUDA_CORES = 1
 OPT_SCORE_WINDOW = 2
+OPT_HIGH_WATERMARK = 3
 _STATUS_NAMES = {1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "CUDA_ERROR", 4: "TIMEOUT", 5: "CAPACITY"}
 
 

@@ -138,6 +138,11 @@ extern "C" omni_status omnitide_set_option(omnitide_ctx* ctx, int32_t option, in
         ctx->score_window = value;
         return OMNI_OK;
     }
+    if (option == OMNI_OPT_HIGH_WATERMARK) {
+        if (value < 0) OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "high watermark must be >= 0");
+        ctx->high_watermark = value;
+        return OMNI_OK;
+    }
     OMNI_FAIL(ctx, OMNI_ERR_INVALID_ARG, "unknown option %d", option);
 }
 
@@ -232,9 +237,19 @@ static omni_status chunk_step_impl(cudaEvent_t chunk_kv_ready, omnitide_ctx* ctx
         t_score = ctx->score_window;
         q_score = static_cast<const char*>(q) + (size_t)(t - t_score) * ctx->g.h_q * ctx->g.d * ctx->es;
     }
-    s = omnitide_score_units(ctx, stream, q_score, t_score, k_cache, n_hist_dev, n_hist_max, units, n_units_dev, n_units_max,
-                             w_modality, scale, ctx->ws_scores, nullptr);
-    if (s) return s;
+    // hysteresis (Section 5.1): a history that cannot exceed the high watermark has no retention round -- no scoring
+    // pass, and the selection keeps every unit (an unbounded budget makes the stale scores irrelevant)
+    omni_select_params keep_all;
+    if (ctx->high_watermark > 0 && n_hist_max <= ctx->high_watermark) {
+        keep_all = *params;
+        keep_all.budget = INT32_MAX;
+        keep_all.modality_cap[0] = keep_all.modality_cap[1] = keep_all.modality_cap[2] = -1;
+        params = &keep_all;
+    } else {
+        s = omnitide_score_units(ctx, stream, q_score, t_score, k_cache, n_hist_dev, n_hist_max, units, n_units_dev, n_units_max,
+                                 w_modality, scale, ctx->ws_scores, nullptr);
+        if (s) return s;
+    }
     // the keep decision stays per unit between the two steps: no token mask, no slot map inside the pass
     s = omnitide_select_units(ctx, stream, units, n_units_dev, n_units_max, ctx->ws_scores, params, ctx->ws_unit_keep,
                               nullptr, n_hist_max, n_kept, units_out, n_units_kept);

@@ -61,6 +61,7 @@ struct omnitide_ctx {
     int64_t launches;
     bool force_cuda_cores;        // OMNI_OPT_FORCE_CUDA_CORES
     int score_window;             // OMNI_OPT_SCORE_WINDOW: trailing queries that score in omnitide_chunk_step (0: all)
+    int high_watermark;           // OMNI_OPT_HIGH_WATERMARK: omnitide_chunk_step runs a retention round only above it (0: always)
     char err[256];
 };
 

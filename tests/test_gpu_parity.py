@@ -692,6 +692,56 @@ def test_chunk_step_with_observation_window(H, ob, cfg2):
     ctx.close()
 
 
+@pytest.mark.parametrize("above", [False, True])
+def test_chunk_step_with_high_watermark(H, ob, cfg2, above):
+    """OMNI_OPT_HIGH_WATERMARK: a call whose history bound is at most the watermark keeps the whole history (the
+    selection rule with a budget that covers everything, Section 5.1 hysteresis) and launches no scoring kernel;
+    above it the pass is the ordinary one."""
+    w = cfg2
+    N, T, U = w.n_hist, w.t, len(w.units)
+    ctx = ob.Context(w.h_q, w.h_kv, w.d, w.dtype, N + T + 64, U + 8, T)
+    kc_in = torch.zeros((N + T + 64, w.h_kv, w.d), dtype=torch.bfloat16, device="cuda")
+    vc_in = torch.zeros_like(kc_in)
+    kc_in[:N], vc_in[:N] = ob.to_device(w.k_hist, "bf16"), ob.to_device(w.v_hist, "bf16")
+    kc_out, vc_out = torch.zeros_like(kc_in), torch.zeros_like(vc_in)
+    units_out = torch.zeros((U + 8, 6), dtype=torch.int32, device="cuda")
+    n_hist_out, n_units_out = H.i32(-1), H.i32(-1)
+    o = torch.zeros((T, w.h_q, w.d), dtype=torch.float32, device="cuda")
+    def step():
+        before = ctx.launch_count()
+        ctx.chunk_step(ob.to_device(w.q, "bf16"), ob.to_device(w.k_chunk, "bf16"), ob.to_device(w.v_chunk, "bf16"), T,
+                       ob.units_to_device(w.chunk_units), len(w.chunk_units), kc_in, vc_in, H.i32(N), N,
+                       ob.units_to_device(w.units, U + 8), H.i32(U), U, w.w_modality,
+                       ob.select_params(w.budget, w.n_recent_events, w.modality_cap), w.page_size, 0.0, kc_out, vc_out,
+                       units_out, n_hist_out, n_units_out, o, ob.DTYPE_FP32)
+        torch.cuda.synchronize()
+        assert ctx.poll_status() == 0
+        return ctx.launch_count() - before
+    ctx.set_option(ob.OPT_HIGH_WATERMARK, 0)
+    launches_full = step()
+    ctx.set_option(ob.OPT_HIGH_WATERMARK, N - 1 if above else N)
+    launches = step()
+    if above:
+        s_gpu, _ = H.gpu_score(ctx, w)
+        sel = oc.select_units(w.units, s_gpu, w.budget, w.n_recent_events, w.modality_cap)
+        assert sel["n_kept"] < N
+    else:
+        sel = oc.select_units(w.units, np.zeros(U, np.float32), N, w.n_recent_events, (-1, -1, -1))
+        assert sel["n_kept"] == N                                   # a budget that covers the history keeps all of it
+        assert launches < launches_full                             # no scoring kernels
+    nk = sel["n_kept"]
+    nu = int(n_units_out.item()) - len(w.chunk_units)
+    assert np.array_equal(units_out[:nu].cpu().numpy(), sel["units_out"])
+    assert int(n_hist_out.item()) == nk + T
+    exp = oc.compact_pack(H.bytes_of(kc_in[:N]).reshape(N, -1), H.bytes_of(vc_in[:N]).reshape(N, -1), sel["keep_mask"], w.page_size)
+    assert np.array_equal(H.bytes_of(kc_out[:nk]).reshape(nk, -1), exp["k"][:nk])
+    assert np.array_equal(H.bytes_of(vc_out[:nk]).reshape(nk, -1), exp["v"][:nk])
+    keep = sel["keep_mask"].astype(bool)
+    o_ref, _ = oc.chunk_attention(w.q, w.k_hist[keep], w.v_hist[keep], w.k_chunk, w.v_chunk)
+    _check_attention(o.cpu().numpy(), None, o_ref, None)
+    ctx.close()
+
+
 def dataclasses_replace_q(w, W):
     import dataclasses
     return dataclasses.replace(w, q=np.ascontiguousarray(w.q[-W:]))
