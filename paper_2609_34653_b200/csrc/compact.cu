@@ -542,26 +542,22 @@ struct CompactUnitsArgs {
 // Positions are slot indices, so the shift of row r is (d0 + r) - src_list[r].  The whole warp takes part: lane 0
 // drives the bulk copies, and once a K row has landed in shared memory every lane rotates the pairs
 // (i, i + rope_dims / 2) of its dimensions i = lane, lane + 32, ... in all heads, in place, before the row is stored.
+// A warp takes the K and the V row of the same destination rows (every warp rotates as much as any other) and keeps
+// the sines and cosines of the last shift: the rows of a kept run share theirs.
 // Angles are formed and reduced to one turn in double (a shift of 1e5 positions times a float frequency would lose
 // the phase), the rotation itself runs in fp32 and the result is rounded to bf16 (nearest even).
 __device__ __forceinline__ void move_rows_rope(const CompactUnitsArgs& a, const int* src_list, const int d0, const int n_rows,
                                                char* rowbuf, uint64_t (*cbar)[CP_MAX_SLOTS], int* abort_flag_p) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    const int n_copies = 2 * n_rows;
-    const int mcp = n_copies > wid ? (n_copies - wid + CP_WARPS - 1) / CP_WARPS : 0;
+    // copy q of this warp: row wid + (q / 2) * CP_WARPS, its K row for even q and its V row for odd q, so that every
+    // warp has the same share of rotations
+    const int my_rows = n_rows > wid ? (n_rows - wid + CP_WARPS - 1) / CP_WARPS : 0;
+    const int mcp = 2 * my_rows;
     char* gbuf0 = rowbuf + (size_t)(wid * a.n_slots) * a.row_bytes;
     const uint32_t buf0 = tc::smem_u32(gbuf0);
     const int half = a.rope_dims >> 1, n_heads = (a.row_bytes >> 1) / a.rope_head_dim;
-    double inv_freq[4];                                      // rope_dims <= 256: at most four frequencies per lane
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const int i = lane + 32 * j;
-        inv_freq[j] = i < half ? exp2(-(2.0 * i / a.rope_dims) * a.rope_log2_base) : 0.0;
-    }
-    auto src_of = [&](int q) {
-        const int i = wid + q * CP_WARPS;
-        return ((i & 1) ? a.v_src : a.k_src) + (size_t)src_list[i >> 1] * a.row_bytes;
-    };
+    auto row_of = [&](int q) { return wid + (q >> 1) * CP_WARPS; };
+    auto src_of = [&](int q) { return ((q & 1) ? a.v_src : a.k_src) + (size_t)src_list[row_of(q)] * a.row_bytes; };
     auto issue_load = [&](int q) {
         const int slot = q % a.n_slots;
         const uint32_t bar = tc::smem_u32(&cbar[wid][slot]);
@@ -570,29 +566,61 @@ __device__ __forceinline__ void move_rows_rope(const CompactUnitsArgs& a, const 
     };
     if (lane == 0)
         for (int q = 0; q < mcp && q < a.n_slots; ++q) issue_load(q);
+    // the frequencies (double: a shift of 1e5 positions times a float frequency would lose the phase) are formed
+    // while the first rows are in flight; rope_dims <= 256: at most four per lane
+    double inv_freq[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int i = lane + 32 * j;
+        inv_freq[j] = 0.0;
+        if (32 * j < half) inv_freq[j] = i < half ? exp2(-(2.0 * i / a.rope_dims) * a.rope_log2_base) : 0.0;
+    }
     bool ok = true;
+    int delta_of_trig = 0;                                   // the shift cs[] / sn[] were computed for (0: none yet)
+    float cs[4], sn[4];
     for (int q = 0; q < mcp && ok; ++q) {
         const int slot = q % a.n_slots;
         ok = __all_sync(0xffffffffu, tc::mbar_wait(tc::smem_u32(&cbar[wid][slot]), (q / a.n_slots) & 1, abort_flag_p));
         if (!ok) break;
-        const int i_copy = wid + q * CP_WARPS, row = i_copy >> 1;
+        const int row = row_of(q);
         const int delta = (d0 + row) - src_list[row];
-        if (!(i_copy & 1) && delta != 0) {
+        if (!(q & 1) && delta != 0) {
+            if (delta != delta_of_trig) {                    // the rows of a kept run share their shift
+                delta_of_trig = delta;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    // the phase is reduced to one turn in double (three operations), then the fast fp32 sine and
+                    // cosine (absolute error about 2^-21, far below the bf16 step of the result) do the rest
+                    const double turns = (double)delta * inv_freq[j] * 0.15915494309189535;
+                    __sincosf((float)((turns - rint(turns)) * 6.283185307179586), &sn[j], &cs[j]);
+                }
+            }
             __nv_bfloat16* r = reinterpret_cast<__nv_bfloat16*>(gbuf0 + (size_t)slot * a.row_bytes);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int i = lane + 32 * j;
                 if (i < half) {
-                    // the phase is reduced to one turn in double (three operations), then the fast fp32 sine and
-                    // cosine (absolute error about 2^-21, far below the bf16 step of the result) do the rest
-                    const double turns = (double)delta * inv_freq[j] * 0.15915494309189535;
-                    float c, sn;
-                    __sincosf((float)((turns - rint(turns)) * 6.283185307179586), &sn, &c);
-                    for (int h = 0; h < n_heads; ++h) {
+                    const float c = cs[j], s_ = sn[j];
+                    int h = 0;
+                    for (; h + 4 <= n_heads; h += 4) {       // four heads at a time: eight independent loads in flight
+                        __nv_bfloat16* px = r + h * a.rope_head_dim + i;
+                        float x[4], y[4];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            x[k] = __bfloat162float(px[k * a.rope_head_dim]);
+                            y[k] = __bfloat162float(px[k * a.rope_head_dim + half]);
+                        }
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            px[k * a.rope_head_dim] = __float2bfloat16_rn(x[k] * c - y[k] * s_);
+                            px[k * a.rope_head_dim + half] = __float2bfloat16_rn(x[k] * s_ + y[k] * c);
+                        }
+                    }
+                    for (; h < n_heads; ++h) {
                         __nv_bfloat16* px = r + h * a.rope_head_dim + i;
                         const float x = __bfloat162float(px[0]), y = __bfloat162float(px[half]);
-                        px[0] = __float2bfloat16_rn(x * c - y * sn);
-                        px[half] = __float2bfloat16_rn(x * sn + y * c);
+                        px[0] = __float2bfloat16_rn(x * c - y * s_);
+                        px[half] = __float2bfloat16_rn(x * s_ + y * c);
                     }
                 }
             }
@@ -600,7 +628,7 @@ __device__ __forceinline__ void move_rows_rope(const CompactUnitsArgs& a, const 
         }
         __syncwarp();
         if (lane == 0) {
-            const char* dst_base = (i_copy & 1) ? a.v_dst : a.k_dst;
+            const char* dst_base = (q & 1) ? a.v_dst : a.k_dst;
             bulk_store(const_cast<char*>(dst_base) + (size_t)(d0 + row) * a.row_bytes, buf0 + slot * a.row_bytes, a.row_bytes);
             if (q >= 1 && q - 1 + a.n_slots < mcp) {
                 asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
