@@ -15,7 +15,7 @@ namespace {
 constexpr int DEC_THREADS = 256;
 constexpr int DEC_WARPS = DEC_THREADS / 32;
 constexpr int DEC_D = 128;
-constexpr int DEC_BATCH = 4;              // key pairs in flight per warp
+constexpr int DEC_BATCH = 2;              // key pairs per batch per warp; the next batch is loaded under the arithmetic of this one
 constexpr int DEC_CTAS_PER_SM = 2;        // splits are sized for about two CTAs per SM in all
 constexpr int DEC_MAX_SPLIT = 64;         // the weights of the final merge live in shared memory (2 * G * 64 floats)
 
@@ -83,20 +83,29 @@ __global__ void __launch_bounds__(DEC_THREADS, (G <= 4 ? 2 : 1)) decode_attentio
     auto v_ptr = [&](int key) {
         return key < n_hist ? p.v_hist + (size_t)key * row + (size_t)kvh * DEC_D + sub * 8 : p.v_chunk + (size_t)kvh * DEC_D + sub * 8;
     };
-    // the trip count depends on the warp only: both half-warps take part in every full-mask shuffle below
+    // the trip count depends on the warp only: both half-warps take part in every full-mask shuffle below.
+    // The loads of batch n + 1 are issued before the arithmetic of batch n (a warp has only three or four batches:
+    // without this every one of them pays a full memory round trip).
+    uint4 kk_next[DEC_BATCH], vv_next[DEC_BATCH];
+    auto load_batch = [&](int base) {
+#pragma unroll
+        for (int b = 0; b < DEC_BATCH; ++b) {
+            const int key = base + half + b * DEC_WARPS * 2;
+            kk_next[b] = make_uint4(0, 0, 0, 0);
+            vv_next[b] = make_uint4(0, 0, 0, 0);
+            if (key < k1) {
+                kk_next[b] = __ldg(reinterpret_cast<const uint4*>(k_ptr(key)));
+                vv_next[b] = __ldg(reinterpret_cast<const uint4*>(v_ptr(key)));
+            }
+        }
+    };
+    if (k0 + warp * 2 < k1) load_batch(k0 + warp * 2);
     for (int base = k0 + warp * 2; base < k1; base += DEC_WARPS * 2 * DEC_BATCH) {
         const int key0 = base + half;
         uint4 kk[DEC_BATCH], vv[DEC_BATCH];
 #pragma unroll
-        for (int b = 0; b < DEC_BATCH; ++b) {
-            const int key = key0 + b * DEC_WARPS * 2;
-            kk[b] = make_uint4(0, 0, 0, 0);
-            vv[b] = make_uint4(0, 0, 0, 0);
-            if (key < k1) {
-                kk[b] = __ldg(reinterpret_cast<const uint4*>(k_ptr(key)));
-                vv[b] = __ldg(reinterpret_cast<const uint4*>(v_ptr(key)));
-            }
-        }
+        for (int b = 0; b < DEC_BATCH; ++b) { kk[b] = kk_next[b]; vv[b] = vv_next[b]; }
+        if (base + DEC_WARPS * 2 * DEC_BATCH < k1) load_batch(base + DEC_WARPS * 2 * DEC_BATCH);
         // scores of the batch first (an invalid key scores -inf), then ONE rescale per head for the whole batch
         float kf[DEC_BATCH][8];
 #pragma unroll
