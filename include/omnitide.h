@@ -496,7 +496,9 @@ omni_status omnitide_score_units_noalloc(void* stream, int32_t h_q, int32_t h_kv
  * retention starts only above a high watermark and trims to the low one, here the selection budget): a call whose
  * n_hist_max is at most H launches no scoring kernel and keeps every unit (the history is copied whole to the output
  * cache); a call whose bound exceeds H runs the full pass.  The decision is the host's, from the bound it was given,
- * so a caller that wants rounds to be rare passes a tight n_hist_max.  0 (default): every call runs the full pass. */
+ * so a caller that wants rounds to be rare passes a tight n_hist_max.  0 (default): every call runs the full pass.
+ * (Scoring only every k-th chunk is the same mechanism driven by the caller: a watermark of INT32_MAX on the other
+ * chunks, the real one, or 0, on every k-th.) */
 enum { OMNI_OPT_FORCE_CUDA_CORES = 1, OMNI_OPT_SCORE_WINDOW = 2, OMNI_OPT_HIGH_WATERMARK = 3 };
 omni_status omnitide_set_option(omnitide_ctx* ctx, int32_t option, int32_t value);
 
