@@ -716,8 +716,64 @@ __global__ void __launch_bounds__(256) attention_merge_kernel(const AttnParams p
     __syncthreads();
     const int n_parts = s_n;
     if (n_parts == 0) return;                                // no item is cut at this boundary (or an earlier boundary owns it)
+    // launched as a programmatic dependent of the main kernel: everything above ran beside it (it reads only what
+    // earlier kernels wrote); the partials exist once the main grid has completed
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int qt = s_qt, head = s_head;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (n_parts <= 2) {
+        // the usual case (an item cut once): the loads of the warp's four rows are issued together, one round trip
+        const bool packed = p.pack_shift >= 0;
+        float2 ml[4][2];
+        float4 o[4][2];
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+            const int r = blockIdx.y * 32 + warp * 4 + q4;
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                ml[q4][i] = make_float2(-INFINITY, 0.f);
+                o[q4][i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (i < n_parts) {
+                    const size_t pslot = (size_t)s_slot[i];
+                    ml[q4][i] = p.part_ml[pslot * BQ + r];
+                    o[q4][i] = *reinterpret_cast<const float4*>(p.part_o + (pslot * BQ + r) * HD + lane * 4);
+                }
+            }
+        }
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+            const int r = blockIdx.y * 32 + warp * 4 + q4;
+            const int row = packed ? (r >> p.pack_shift) : qt * BQ + r;
+            const int out_head = packed ? (head << p.pack_shift) + (r & ((1 << p.pack_shift) - 1)) : head;
+            if (row >= p.t) continue;
+            float M = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+                if (ml[q4][i].y > 0.f) M = fmaxf(M, ml[q4][i].x);
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            float L = 0.f;
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                if (!(ml[q4][i].y > 0.f)) continue;
+                const float wgt = tc::ex2_approx((ml[q4][i].x - M) * p.scale_log2);
+                acc.x += wgt * o[q4][i].x; acc.y += wgt * o[q4][i].y; acc.z += wgt * o[q4][i].z; acc.w += wgt * o[q4][i].w;
+                L += wgt * ml[q4][i].y;
+            }
+            const float inv = 1.f / L;
+            const size_t off = ((size_t)row * p.h_q + out_head) * HD + lane * 4;
+            if (p.out_dtype == OMNI_DTYPE_FP32) {
+                *reinterpret_cast<float4*>(static_cast<float*>(p.o_out) + off) =
+                    make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+            } else {
+                uint2 v;
+                v.x = tc::pack_bf16x2(acc.x * inv, acc.y * inv);
+                v.y = tc::pack_bf16x2(acc.z * inv, acc.w * inv);
+                *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.o_out) + off) = v;
+            }
+            if (p.lse_out && lane == 0) p.lse_out[(size_t)row * p.h_q + out_head] = M * p.scale + logf(L);
+        }
+        return;
+    }
     for (int q4 = 0; q4 < 4; ++q4) {
         const int r = blockIdx.y * 32 + warp * 4 + q4;       // row of the tile
         const bool packed = p.pack_shift >= 0;
@@ -817,8 +873,18 @@ omni_status omni_attention_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q,
     OMNI_CHECK_LAUNCH(ctx, "attention_tc_kernel");
     if (n_cta > 1) {
         // one CTA row per boundary between two shares: only an item cut there has partials to merge
-        attention_merge_kernel<<<dim3(n_cta - 1, 4), 256, (n_cta + 2) * sizeof(int) + (n_cta + 1) * sizeof(long long), st>>>(p, n_cta);
-        OMNI_CHECK_LAUNCH(ctx, "attention_merge_kernel");
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(n_cta - 1, 4);
+        cfg.blockDim = dim3(256);
+        cfg.dynamicSmemBytes = (n_cta + 2) * sizeof(int) + (n_cta + 1) * sizeof(long long);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;       // its prologue and its launch run under the main kernel
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        OMNI_CUDA(ctx, cudaLaunchKernelEx(&cfg, attention_merge_kernel, p, n_cta));
+        ++ctx->launches;
     }
     return OMNI_OK;
 }
