@@ -86,6 +86,7 @@ class ClockSampler:
         self.thread = None
         self.stop_flag = False
         self.sm, self.mx, self.reasons = [], [], set()
+        self.ts, self.bits = [], []          # NVML path: time of every sample and its reason bits
 
     def _nvml_handle(self):
         import pynvml
@@ -105,6 +106,8 @@ class ClockSampler:
                 self.sm.append(float(pynvml.nvmlDeviceGetClockInfo(handle, pynvml.NVML_CLOCK_SM)))
                 self.mx.append(float(pynvml.nvmlDeviceGetMaxClockInfo(handle, pynvml.NVML_CLOCK_SM)))
                 bits = int(pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(handle))
+                self.ts.append(time.perf_counter())
+                self.bits.append(bits)
                 for name, bit in self.REASONS:
                     if bits & bit:
                         self.reasons.add(name)
@@ -132,13 +135,21 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
-    def stop(self):
+    def stop(self, skip_seconds=0.0):
+        """skip_seconds: drop the samples of the first part of the window (NVML path; the driver refreshes its readings
+        about every 100 ms, so the first ones still show the state before the load)."""
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
         source = None
         if self.thread is not None:
             self.stop_flag = True
             self.thread.join(timeout=2)
             source = "nvml, 5 ms period"
+            if skip_seconds > 0 and self.ts:
+                keep = [i for i, t_ in enumerate(self.ts) if t_ - self.ts[0] >= skip_seconds]
+                if keep:
+                    self.sm = [self.sm[i] for i in keep]
+                    self.mx = [self.mx[i] for i in keep]
+                    self.reasons = {name for i in keep for name, bit in self.REASONS if self.bits[i] & bit}
         elif self.proc is not None:
             time.sleep(0.15)
             self.proc.terminate()
@@ -414,6 +425,8 @@ def main():
     ap.add_argument("--workload", default="long_stream")
     ap.add_argument("--sets", type=int, default=8, help="distinct cache sets rotated so the working set exceeds L2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sustained-seconds", type=float, default=1.0,
+                    help="also run the step back to back for about this long (power-capped steady state; 0: skip)")
     ap.add_argument("--mask-compaction", action="store_true",
                     help="time omnipage_compact (token keep mask + slot map) instead of the unit-granular entry point")
     ap.add_argument("--no-sweep", dest="sweep", action="store_false", help="skip the 36-cell stress grid (131,072-token history)")
@@ -540,6 +553,26 @@ def main():
     torch.cuda.synchronize()
     event_pair_floor_ms = float(np.mean([a_.elapsed_time(b_) for a_, b_ in floor_evs]))
 
+    # ---- the same step back to back for about a second: the GPU settles at the clock its power cap allows for this
+    # mix of kernels, and the driver's clock readings (refreshed about every 100 ms) have time to show it.  The
+    # per-kernel times are those of the second half of the run.
+    sustained = None
+    if args.sustained_seconds > 0:
+        n_s = max(args.steps, int(np.ceil(args.sustained_seconds * 1e3 / max(total_ms / args.steps, 1e-3))))
+        evs_s = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(n_s)]
+        sampler_s = ClockSampler(local_rank)
+        barrier()
+        sampler_s.start()
+        for i in range(n_s):
+            one_step(sets[i % R], evs_s[i])
+        barrier()
+        clocks_s = sampler_s.stop(skip_seconds=min(0.4, 0.5 * args.sustained_seconds))
+        assert ctx.poll_status() == 0, "device status word not clean after the sustained run"
+        half = range(n_s // 2, n_s)
+        per_s = {n: float(np.mean([evs_s[i][j].elapsed_time(evs_s[i][j + 1]) for i in half])) for j, n in enumerate(names)}
+        step_s = evs_s[n_s // 2][0].elapsed_time(evs_s[n_s - 1][5]) / len(half)
+        sustained = {"steps": n_s, "ms_per_step": step_s, "per_kernel_ms": per_s, "clocks": clocks_s}
+
     # ---- end to end through the host-buffer entry point: chunk H2D and output D2H inside the timed region
     hq = torch.from_numpy(w.q).to(tdt).contiguous().pin_memory()
     hk = torch.from_numpy(w.k_chunk).to(tdt).contiguous().pin_memory()
@@ -647,6 +680,25 @@ def main():
                                 "ms_per_chunk": e2e_ms, "entry": "omnitide_chunk_step_host",
                                 "note": "the caller waits for the output in host memory after every step"}},
     }
+    if sustained is not None:
+        st_ms, sa_ms, ss_ms, sc_ms_ = max_over_ranks([sustained["ms_per_step"], sustained["per_kernel_ms"]["attention"],
+                                                      sustained["per_kernel_ms"]["score"], sustained["per_kernel_ms"]["compact"]],
+                                                     world, "cuda")
+        s_att_tf = work["attn_flop"] / (sa_ms * 1e-3) / 1e12
+        s_texp = work["score_exp"] / (ss_ms * 1e-3) / 1e12
+        s_mhz = sustained["clocks"].get("sm_mhz") or SM_MAX_MHZ
+        line["sustained"] = {
+            "steps": sustained["steps"], "ms_per_step": st_ms, "clocks": sustained["clocks"],
+            "attention": {"ms": sa_ms, "achieved": s_att_tf * world, "unit": "TFLOP/s", "peak": tensor_peak,
+                          "frac": s_att_tf / tensor_peak},
+            "score": {"ms": ss_ms, "achieved": s_texp, "unit": "Texp/s", "frac": s_texp / xu_peak,
+                      "frac_at_sampled_clock": s_texp / (XU_PER_CLK_PER_SM * N_SM * s_mhz * 1e6 / 1e12)},
+            "compact": {"ms": sc_ms_, "achieved": cp_bytes / (sc_ms_ * 1e-3) / 1e9, "unit": "GB/s",
+                        "frac": cp_bytes / (sc_ms_ * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+            "note": "the step back to back for about a second, kernel times of the second half: the regime the sustained "
+                    "matmul peak was measured in (power cap active, SM clock below its maximum); the figures above this "
+                    "object come from the short timed region the command line asked for"}
+
     # ---- decode-phase attention: one new token against the compacted history (split-KV decode kernel), cache sets rotated
     d_reps = max(8, min(args.steps, 40))
     devs = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(d_reps)]
