@@ -85,6 +85,7 @@ struct AttnParams {
 
 struct Barriers {
     uint64_t q_full;
+    uint64_t q_free;            // every QK^T of the part has completed: the Q tile may be overwritten
     uint64_t kv_full[NSTAGE];
     uint64_t kv_empty[NSTAGE];
     uint64_t s_full;            // S of the next block is complete
@@ -194,6 +195,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
     if (threadIdx.x == 0) {
         tc::mbar_init(tc::smem_u32(&bars->q_full), 1);
+        tc::mbar_init(tc::smem_u32(&bars->q_free), 1);
         for (int s = 0; s < NSTAGE; ++s) {
             tc::mbar_init(tc::smem_u32(&bars->kv_full[s]), 1);
             tc::mbar_init(tc::smem_u32(&bars->kv_empty[s]), 1);
@@ -253,8 +255,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 issued = idx + 1;
             };
             while (ok && it.next(part)) {
-                // the Q tile is free once every MMA of the previous part has completed
-                if (part_idx > 0) ok = tc::mbar_wait(tc::smem_u32(&bars->o_done), (part_idx - 1) & 1, abort_flag);
+                // the Q tile is free once every QK^T of the previous part has completed (its last softmax, its last PVs
+                // and its epilogue still run: the next part's Q and first K tiles land under them)
+                if (part_idx > 0) ok = tc::mbar_wait(tc::smem_u32(&bars->q_free), (part_idx - 1) & 1, abort_flag);
                 if (!ok) break;
                 kvh = packed ? part.head : part.head / (p.h_q / p.h_kv);
                 tc::mbar_expect_tx(tc::smem_u32(&bars->q_full), TILE_BYTES);
@@ -319,6 +322,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     TRACE(2, 2); TRACE(2, 3); TRACE(2, 4);
                     TRACE_NEXT();
                 }
+                if (ok) tc::umma_commit(tc::smem_u32(&bars->q_free));
                 // the softmax warpgroups must have seen the previous part's o_done before this part's is
                 // committed (a waiter may lag one mbarrier phase, never two)
                 if (ok && part_idx > 0) ok = wait(&bars->o_free, (part_idx - 1) & 1);
