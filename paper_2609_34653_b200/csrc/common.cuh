@@ -60,7 +60,7 @@ struct omnitide_ctx {
     void* encode_tiled;           // cuTensorMapEncodeTiled, resolved through the runtime
     int64_t launches;
     bool force_cuda_cores;        // OMNI_OPT_FORCE_CUDA_CORES
-    int sc_split_items, sc_split_nkb, sc_split_best;   // the scoring kernel's last split decision (work items, key blocks -> splits)
+    int sc_split_items, sc_split_nkb, sc_split_best, sc_split_bps;   // the scoring kernel's last split decision (work items, key blocks -> splits)
     int score_window;             // OMNI_OPT_SCORE_WINDOW: trailing queries that score in omnitide_chunk_step (0: all)
     int high_watermark;           // OMNI_OPT_HIGH_WATERMARK: omnitide_chunk_step runs a retention round only above it (0: always)
     char err[256];

@@ -44,6 +44,7 @@ struct ScoreParams {
     float2* part;             // [tile][seg_cap][128]
     int seg_cap;
     int ctas_per_kv, n_row_tiles, n_splits;                   // CTAs per KV head and split: ceil(n_row_tiles * G / NT)
+    int bps;                                                  // key blocks per split (the last split of a history may be shorter)
     int32_t* status;
 };
 
@@ -107,7 +108,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         return;
     }
     const int nkb = (n_hist + BLK - 1) / BLK;
-    const int bps = blocks_per_split(nkb, p.n_splits);
+    const int bps = p.bps;
     const int b0 = split * bps, b1 = min(nkb, b0 + bps);
     const int nb = b1 - b0;
     if (nb <= 0) return;
@@ -321,7 +322,7 @@ __global__ void __launch_bounds__(128) score_combine_kernel(const ScoreParams p,
     const int n_hist = p.units[n_units - 1].start + p.units[n_units - 1].len;
     if (n_hist > p.n_hist_max) return;
     const int nkb = (n_hist + BLK - 1) / BLK;
-    const int bps = blocks_per_split(nkb, p.n_splits);
+    const int bps = p.bps;
     // first and last split of every unit, once per CTA
     int* s_first = cmb_smem;                                  // [n_units]
     int* s_last = cmb_smem + p.n_units_max;                   // [n_units]
@@ -427,44 +428,50 @@ omni_status omni_score_tc(omnitide_ctx* ctx, cudaStream_t st, const void* q, int
     // cost of a choice = the makespan when the hardware hands the CTAs out in block order to the SMs as they free up
     // (one CTA per SM; a CTA costs its key blocks plus a start-up allowance: Q load, pipeline fill, partial writes).
     // The CTAs of a split have equal length, so the simulation keeps (load, SM count) groups in ascending order.
-    // Whole-wave counting misleads here: 16 splits of a 625-block history are 16.4 waves, but the short last pieces
-    // fill the partial wave and the launch is 2-3 % faster than with 11 splits (measured, and what this model says).
+    // Whole-wave counting misleads here: for a 625-block history it picks 11 even splits (11.3 waves), while 10 splits
+    // of 66 blocks with a last one of 31 (10.3 waves, the short pieces filling the partial wave) are 4 % faster
+    // (measured, and what this model says).
     if (ctx->sc_split_items != base_items || ctx->sc_split_nkb != nkb_max) {
         constexpr int STARTUP_BLOCKS = 3;
-        int best = 1;
+        int best = 1, best_bps = nkb_max;
         long long best_cost = -1;
         std::vector<std::pair<long long, int>> groups;
         for (int ks = 1; ks <= 32 && (ks == 1 || nkb_max / ks >= 8); ++ks) {
-            const int bps = blocks_per_split(nkb_max, ks);
-            groups.assign(1, std::make_pair(0ll, ctx->sm_count));
-            long long makespan = 0;
-            for (int sp = 0; sp < ks; ++sp) {
-                const int len = std::min(nkb_max, (sp + 1) * bps) - sp * bps;
-                if (len <= 0) break;
-                const long long job = len + STARTUP_BLOCKS;
-                int left = base_items;
-                while (left > 0) {
-                    const long long a = groups.front().first;
-                    const int take = std::min(groups.front().second, left);
-                    groups.front().second -= take;
-                    if (groups.front().second == 0) groups.erase(groups.begin());
-                    const long long b = a + job;
-                    auto pos = groups.begin();
-                    while (pos != groups.end() && pos->first < b) ++pos;
-                    if (pos != groups.end() && pos->first == b) pos->second += take;
-                    else groups.insert(pos, std::make_pair(b, take));
-                    makespan = std::max(makespan, b);
-                    left -= take;
+            // ks - 1 pieces of bps blocks and a shorter last one: a last piece of about half a piece fills the
+            // partial last wave best, so sizes a little above the even one are tried too
+            const int even = blocks_per_split(nkb_max, ks);
+            for (int bps = even; bps < even + 12 && (ks == 1 ? bps == even : (long long)(ks - 1) * bps < nkb_max); ++bps) {
+                groups.assign(1, std::make_pair(0ll, ctx->sm_count));
+                long long makespan = 0;
+                for (int sp = 0; sp < ks; ++sp) {
+                    const int len = std::min(nkb_max, (sp + 1) * bps) - sp * bps;
+                    const long long job = len + STARTUP_BLOCKS;
+                    int left = base_items;
+                    while (left > 0) {
+                        const long long a = groups.front().first;
+                        const int take = std::min(groups.front().second, left);
+                        groups.front().second -= take;
+                        if (groups.front().second == 0) groups.erase(groups.begin());
+                        const long long b = a + job;
+                        auto pos = groups.begin();
+                        while (pos != groups.end() && pos->first < b) ++pos;
+                        if (pos != groups.end() && pos->first == b) pos->second += take;
+                        else groups.insert(pos, std::make_pair(b, take));
+                        makespan = std::max(makespan, b);
+                        left -= take;
+                    }
                 }
+                if (best_cost < 0 || makespan < best_cost) { best_cost = makespan; best = ks; best_bps = bps; }
             }
-            if (best_cost < 0 || makespan < best_cost) { best_cost = makespan; best = ks; }
         }
         ctx->sc_split_items = base_items;
         ctx->sc_split_nkb = nkb_max;
         ctx->sc_split_best = best;
+        ctx->sc_split_bps = best_bps;
     }
     const int best = ctx->sc_split_best;
     p.n_splits = best;
+    p.bps = ctx->sc_split_bps;
     const int smem = SMEM_FIXED + n_units_max * (int)sizeof(int);
     if (smem > 227 * 1024) OMNI_FAIL(ctx, OMNI_ERR_CAPACITY, "score: too many units for one CTA's shared memory");
     OMNI_CUDA(ctx, cudaFuncSetAttribute(score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
